@@ -1,0 +1,174 @@
+/*
+ * pvq.h - C ABI of the B200 (sm_100a) group-wise Pyramid Vector Quantization codec.
+ *
+ * A rows x cols matrix (row-major) is cut into groups of N contiguous values
+ * along each row, G = cols / N groups per row (Sec. 3.3 Step 0).  Each group is
+ * stored as
+ *   - one direction code: the Fischer index (Algorithm 2) of the point of the
+ *     pyramid P(N,K) = { y in Z^N : sum |y_i| = K } nearest to the group's
+ *     direction (Sec. 2.5), an unsigned integer in [0, N(N,K) - 1] kept as W
+ *     little-endian 32-bit words, W = ceil(ceil(log2 N(N,K)) / 32);
+ *   - one amplitude index of scale_bits bits: the quantile bin of the group's
+ *     share of the row energy, u = ||x_g||^2 / ||x_row||^2, under
+ *     Beta(N/2, N(G-1)/2) (Sec. 3.4, Sec. 3.3 Step 5);
+ * and each row stores its norm ||x_row||_2 once (fp32), which Step 5 says has
+ * to be kept for dequantisation.
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers owned by the caller; the library
+ *     never allocates, frees or keeps them.  Everything else is host memory.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and
+ *     return without synchronising; outputs are valid once the stream reaches
+ *     that point.  The device current at the call must own all pointers.
+ *   - Every function returns a pvq_status; nothing is thrown across the ABI and
+ *     no argument error reaches a kernel.
+ *   - Inputs must be finite.  NaN or Inf gives unspecified codes but never an
+ *     out-of-bounds access.
+ *
+ * Storage formats (also the persistent format of an encoded matrix)
+ *   codes      uint32  codes[(r*G + g)*W + w], w = 0 the least significant word.
+ *   scale_idx  bytes   one LSB-first bit stream per row: group g occupies bits
+ *                      [g*b, (g+1)*b) of the row, b = scale_bits; the row stride
+ *                      is pvq_scale_row_stride(G, b) = ceil(G*b/8) rounded up to 4.
+ *   row_norm   float   row_norm[r].
+ *   count table uint32 table[(n*(K+1) + k)*W + w] = word w of N(n,k) for
+ *                      n = 0..N-1 (dimensions left after a position) and
+ *                      k = 0..K; pvq_count_table_bytes(N,K) bytes, 16-byte
+ *                      aligned.
+ *   edges      float   2^b - 1 ascending bin edges of u.
+ *   levels     float   2^b values sqrt(PPF((q + 1/2) / 2^b)): the factor that
+ *                      multiplies row_norm to give the dequantised amplitude.
+ */
+#ifndef PVQ_H_
+#define PVQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PVQ_OK = 0,
+    PVQ_ERR_INVALID_ARG = 1,     /* null pointer, non-positive size, cols % N != 0, ... */
+    PVQ_ERR_UNSUPPORTED = 2,     /* (N, K, W) or G outside what the kernels are built for */
+    PVQ_ERR_ALIGNMENT = 3,       /* a pointer or leading dimension breaks the stated alignment */
+    PVQ_ERR_TABLE_TOO_SMALL = 4, /* buffer smaller than the size the call needs */
+    PVQ_ERR_CUDA = 5             /* a CUDA call failed; see pvq_last_cuda_error() */
+} pvq_status;
+
+#define PVQ_DTYPE_F32 0
+#define PVQ_DTYPE_BF16 1
+
+/* bit 0 of the decode status word: some code was >= N(N,K) */
+#define PVQ_STATUS_INVALID_CODE 1u
+
+typedef void* pvq_stream_t; /* a cudaStream_t */
+
+/* Human-readable name of a status.  Never NULL. */
+const char* pvq_strerror(int status);
+
+/* cudaError_t (as int) of the last failed CUDA call made by this library on the
+ * calling thread; 0 if none. */
+int pvq_last_cuda_error(void);
+
+/* ---- host-side parameter helpers (exact integer arithmetic, no GPU) ---------- */
+
+/* ceil(log2 N(N,K)): bits of one direction code (Sec. 3.3 Step 7).  N >= 1, K >= 0. */
+int pvq_index_bits(int N, int K, int* bits_out);
+
+/* Sec. 3.3 Step 2: the largest K with N(N,K) <= 2^index_bits (the comparison is made
+ * on the integers).  *K_out = 0 when not even one pulse fits. */
+int pvq_max_pulses(int N, int index_bits, int* K_out);
+
+/* W = ceil(pvq_index_bits / 32), at least 1. */
+int pvq_code_words(int N, int K, int* W_out);
+
+/* Bytes of the device count table for (N,K): N * (K+1) * W * 4.  0 on bad arguments. */
+size_t pvq_count_table_bytes(int N, int K);
+
+/* Row stride in bytes of the packed amplitude indices. */
+size_t pvq_scale_row_stride(int64_t G, int scale_bits);
+
+/* ---- set-up kernels (cold path) --------------------------------------------------- */
+
+/* Fill d_table with N(n,k), n = 0..N-1, k = 0..K (Sec. 2.4 recurrence; built a row at a
+ * time with a parallel prefix sum over k as in App. C.2 / Algorithm 4, by one thread
+ * block).  `bytes` is the size of d_table and must be at least
+ * pvq_count_table_bytes(N,K).  Requires 1 <= N <= 256, 1 <= K <= 1023, W <= 12. */
+int pvq_build_count_table(int N, int K, uint32_t* d_table, size_t bytes, pvq_stream_t stream);
+
+/* Fill d_edges (2^b - 1 floats) and d_levels (2^b floats) for group size N, G groups per
+ * row and b = scale_bits (Sec. 3.4: quantize = floor(CDF * 2^b), dequantize =
+ * PPF((q + 1/2) / 2^b), Beta(N/2, N(G-1)/2)).  Computed in fp64 on the device and rounded
+ * once to fp32.  Requires N even, G >= 2, 1 <= b <= 8.  Either pointer may be NULL. */
+int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, float* d_levels,
+                             pvq_stream_t stream);
+
+/* ---- hot path --------------------------------------------------------------------- */
+
+/* Encode (Sec. 3.3 Steps 3, 4, 5, 7; Algorithms 1 and 2).
+ *   d_x        rows x cols values of `dtype`, leading dimension ld (elements); 16-byte
+ *              aligned, ld a multiple of 8 (bf16) or 4 (fp32) elements.
+ *   N, K       group size (power of two, 8..64) and pulses; cols % N == 0; G >= 2.
+ *   d_table    from pvq_build_count_table(N, K, ...).
+ *   d_edges    2^scale_bits - 1 bin edges.
+ *   d_codes    out, rows*G*W words.      d_scale_idx  out, rows * stride bytes.
+ *   d_row_norm out, rows floats.
+ * Arithmetic: fp32 with one rounding per operation; sums over a group and over the
+ * groups of a row use a balanced tree over contiguous halves (row: zero-padded to a
+ * power of two).  Amplitude index q = #{ j : u >= edges[j] }.  Direction: scale to the
+ * l1 ball of radius K, floor, then hand out the missing pulses one at a time to the
+ * largest residual, lowest index first among equals; a group with zero l1 norm maps to
+ * (K,0,...,0). */
+int pvq_encode(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+               int scale_bits, const uint32_t* d_table, const float* d_edges, uint32_t* d_codes,
+               uint8_t* d_scale_idx, float* d_row_norm, pvq_stream_t stream);
+
+/* Decode to bf16 (Algorithm 3; Sec. 2.4 projection on the sphere; Sec. 3.4 dequantize).
+ *   out[r][g*N + i] = bf16( y_i * (row_norm[r] * levels[q]) / sqrt(sum y^2) ), rounded to
+ *   nearest even, with y the pyramid point of the code.
+ *   d_out      rows x cols bf16, leading dimension ld_out (elements, multiple of 8),
+ *              16-byte aligned.
+ *   d_status   optional device word; PVQ_STATUS_INVALID_CODE is OR-ed into it when a code
+ *              is >= N(N,K) (that group decodes to zeros).  May be NULL. */
+int pvq_decode(const uint32_t* d_codes, const uint8_t* d_scale_idx, const float* d_row_norm,
+               int64_t rows, int64_t cols, int N, int K, int scale_bits, const uint32_t* d_table,
+               const float* d_levels, void* d_out, int64_t ld_out, uint32_t* d_status,
+               pvq_stream_t stream);
+
+/* Fused encode -> decode of activations (Sec. 2.2, Sec. 4.3: on-the-fly quantisation):
+ * each group is encoded to its integer code and decoded again inside one kernel, the code
+ * living in registers; only d_x is read and d_out written.  Same arguments and arithmetic
+ * as pvq_encode followed by pvq_decode. */
+int pvq_roundtrip(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+                  int scale_bits, const uint32_t* d_table, const float* d_edges,
+                  const float* d_levels, void* d_out, int64_t ld_out, pvq_stream_t stream);
+
+/* One matrix of a batched call.  Pointers are device pointers with the meaning and
+ * alignment of the corresponding pvq_encode / pvq_decode arguments; d_edges / d_levels
+ * belong to this matrix's G. */
+typedef struct {
+    const void* d_x;      /* encode input (unused by decode) */
+    void* d_out;          /* decode output (unused by encode) */
+    uint32_t* d_codes;
+    uint8_t* d_scale_idx;
+    float* d_row_norm;
+    const float* d_edges;
+    const float* d_levels;
+    int64_t rows, cols, ld, ld_out;
+} pvq_matrix_desc;
+
+/* Encode / decode `count` matrices (1..32) that share dtype, N, K, scale_bits and the
+ * count table with ONE kernel launch (all seven matrices of a decoder layer at once).
+ * `descs` is a host array, copied into the launch; it may be freed on return. */
+int pvq_encode_batched(const pvq_matrix_desc* descs, int count, int dtype, int N, int K,
+                       int scale_bits, const uint32_t* d_table, pvq_stream_t stream);
+int pvq_decode_batched(const pvq_matrix_desc* descs, int count, int N, int K, int scale_bits,
+                       const uint32_t* d_table, uint32_t* d_status, pvq_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PVQ_H_ */

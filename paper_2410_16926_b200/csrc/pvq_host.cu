@@ -1,0 +1,324 @@
+// Host side of the C ABI: argument checks, exact integer helpers for choosing
+// K (Sec. 3.3 Step 2), and translation of the public calls into kernel launches.
+#include <algorithm>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <utility>
+#include <vector>
+
+#include "pvq_internal.cuh"
+
+namespace pvq {
+
+static thread_local int g_last_cuda_error = 0;
+
+int set_cuda_error(cudaError_t e) {
+    g_last_cuda_error = static_cast<int>(e);
+    return PVQ_ERR_CUDA;
+}
+
+bool is_aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// ------------------------------------------------------------------ big ints
+// Unsigned integers of up to kLimbs 32-bit limbs; only what choosing K needs.
+namespace {
+
+constexpr int kLimbs = 48;
+
+struct BigU {
+    uint32_t w[kLimbs];
+    BigU() { std::memset(w, 0, sizeof w); }
+    explicit BigU(uint32_t v) {
+        std::memset(w, 0, sizeof w);
+        w[0] = v;
+    }
+    // *this += o; false when the sum overflows kLimbs
+    bool add(const BigU& o) {
+        uint64_t c = 0;
+        for (int i = 0; i < kLimbs; ++i) {
+            uint64_t s = static_cast<uint64_t>(w[i]) + o.w[i] + c;
+            w[i] = static_cast<uint32_t>(s);
+            c = s >> 32;
+        }
+        return c == 0;
+    }
+    int bit_length() const {
+        for (int i = kLimbs - 1; i >= 0; --i)
+            if (w[i]) return 32 * i + (32 - __builtin_clz(w[i]));
+        return 0;
+    }
+    bool is_pow2() const {
+        int ones = 0;
+        for (int i = 0; i < kLimbs; ++i) ones += __builtin_popcount(w[i]);
+        return ones == 1;
+    }
+    // ceil(log2 v) for v >= 1
+    int ceil_log2() const { return is_pow2() ? bit_length() - 1 : bit_length(); }
+};
+
+// col[n] = N(n,k) for n = 0..N, advanced from k to k+1 with
+// N(n,k+1) = N(n-1,k+1) + N(n,k) + N(n-1,k)   (Sec. 2.4).
+struct CountColumn {
+    std::vector<BigU> col;
+    int k = 0;
+    explicit CountColumn(int N) : col(static_cast<size_t>(N) + 1, BigU(1u)) {}  // N(n,0) = 1
+    bool advance() {
+        std::vector<BigU> nxt(col.size());
+        nxt[0] = BigU(0u);  // N(0,k>=1) = 0
+        for (size_t n = 1; n < col.size(); ++n) {
+            nxt[n] = nxt[n - 1];
+            if (!nxt[n].add(col[n]) || !nxt[n].add(col[n - 1])) return false;
+        }
+        col.swap(nxt);
+        ++k;
+        return true;
+    }
+};
+
+}  // namespace
+
+static int index_bits_exact(int N, int K) {
+    if (N < 1 || N > 4096 || K < 0 || K > 65535) return -1;
+    CountColumn c(N);
+    for (int k = 0; k < K; ++k)
+        if (!c.advance()) return -1;
+    return c.col[static_cast<size_t>(N)].ceil_log2();
+}
+
+// W for (N,K); memoised, since every hot call asks for it.
+int code_words_for(int N, int K) {
+    static std::mutex mu;
+    static std::map<std::pair<int, int>, int> memo;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find({N, K});
+    if (it != memo.end()) return it->second;
+    int bits = index_bits_exact(N, K);
+    int W = bits < 0 ? 0 : std::max(1, (bits + 31) / 32);
+    memo[{N, K}] = W;
+    return W;
+}
+
+}  // namespace pvq
+
+using namespace pvq;
+
+// -------------------------------------------------------------- public: misc
+
+extern "C" const char* pvq_strerror(int status) {
+    switch (status) {
+        case PVQ_OK: return "PVQ_OK";
+        case PVQ_ERR_INVALID_ARG: return "PVQ_ERR_INVALID_ARG: bad pointer, size or parameter";
+        case PVQ_ERR_UNSUPPORTED: return "PVQ_ERR_UNSUPPORTED: no kernel for this (N, K, G)";
+        case PVQ_ERR_ALIGNMENT: return "PVQ_ERR_ALIGNMENT: pointer or leading dimension not aligned";
+        case PVQ_ERR_TABLE_TOO_SMALL: return "PVQ_ERR_TABLE_TOO_SMALL: buffer smaller than required";
+        case PVQ_ERR_CUDA: return "PVQ_ERR_CUDA: a CUDA call failed (pvq_last_cuda_error)";
+        default: return "unknown pvq status";
+    }
+}
+
+extern "C" int pvq_last_cuda_error(void) { return g_last_cuda_error; }
+
+extern "C" int pvq_index_bits(int N, int K, int* bits_out) {
+    if (!bits_out) return PVQ_ERR_INVALID_ARG;
+    int b = index_bits_exact(N, K);
+    if (b < 0) return PVQ_ERR_INVALID_ARG;
+    *bits_out = b;
+    return PVQ_OK;
+}
+
+extern "C" int pvq_max_pulses(int N, int index_bits, int* K_out) {
+    if (!K_out || N < 1 || N > 4096 || index_bits < 1 || index_bits > 32 * (kLimbs - 2))
+        return PVQ_ERR_INVALID_ARG;
+    CountColumn c(N);
+    int K = 0;
+    for (;;) {
+        if (!c.advance()) break;
+        const BigU& v = c.col[static_cast<size_t>(N)];
+        // v <= 2^index_bits  <=>  bit_length <= index_bits, or v == 2^index_bits exactly
+        int bl = v.bit_length();
+        bool fits = bl <= index_bits || (bl == index_bits + 1 && v.is_pow2());
+        if (!fits) break;
+        K = c.k;
+        if (K >= 65535) break;
+    }
+    *K_out = K;
+    return PVQ_OK;
+}
+
+extern "C" int pvq_code_words(int N, int K, int* W_out) {
+    if (!W_out) return PVQ_ERR_INVALID_ARG;
+    int W = code_words_for(N, K);
+    if (W == 0) return PVQ_ERR_INVALID_ARG;
+    *W_out = W;
+    return PVQ_OK;
+}
+
+extern "C" size_t pvq_count_table_bytes(int N, int K) {
+    int W = code_words_for(N, K);
+    if (W == 0 || N < 1 || K < 1) return 0;
+    return static_cast<size_t>(N) * (static_cast<size_t>(K) + 1) * static_cast<size_t>(W) * 4u;
+}
+
+extern "C" size_t pvq_scale_row_stride(int64_t G, int scale_bits) {
+    if (G < 1 || scale_bits < 1 || scale_bits > 8) return 0;
+    size_t bytes = static_cast<size_t>((G * scale_bits + 7) / 8);
+    return (bytes + 3u) & ~static_cast<size_t>(3u);
+}
+
+// ------------------------------------------------------ public: hot-path calls
+
+namespace {
+
+struct Common {
+    int N, K, W, scale_bits;
+};
+
+int check_common(int N, int K, int scale_bits, const uint32_t* d_table, Common* out) {
+    if (N < 2 || (N & (N - 1)) != 0 || K < 1) return PVQ_ERR_INVALID_ARG;
+    if (scale_bits < 1 || scale_bits > 8) return PVQ_ERR_INVALID_ARG;
+    if (!d_table) return PVQ_ERR_INVALID_ARG;
+    if (N < 8 || N > 64 || K > kMaxPulses) return PVQ_ERR_UNSUPPORTED;
+    int W = code_words_for(N, K);
+    if (W == 0) return PVQ_ERR_INVALID_ARG;
+    if (W > kMaxWords) return PVQ_ERR_UNSUPPORTED;
+    if (!is_aligned(d_table, 16)) return PVQ_ERR_ALIGNMENT;
+    out->N = N;
+    out->K = K;
+    out->W = W;
+    out->scale_bits = scale_bits;
+    return PVQ_OK;
+}
+
+// Fills the geometry of one matrix; `need` says which pointers the call uses.
+enum { NEED_X = 1, NEED_OUT = 2, NEED_CODES = 4, NEED_EDGES = 8, NEED_LEVELS = 16 };
+
+int fill_matrix(const pvq_matrix_desc& d, int need, int dtype, const Common& c, MatrixArgs* m) {
+    if (d.rows < 1 || d.cols < 1 || d.cols % c.N != 0) return PVQ_ERR_INVALID_ARG;
+    const int64_t G = d.cols / c.N;
+    if (G < 2) return PVQ_ERR_UNSUPPORTED;  // the quantile codebook needs two groups (beta > 0)
+    if (G > 1024) return PVQ_ERR_UNSUPPORTED;
+    if (d.rows * G >= (int64_t(1) << 31)) return PVQ_ERR_UNSUPPORTED;
+    if (need & NEED_X) {
+        if (!d.d_x || d.ld < d.cols) return PVQ_ERR_INVALID_ARG;
+        const int vec = dtype == PVQ_DTYPE_BF16 ? 8 : 4;
+        if (!is_aligned(d.d_x, 16) || d.ld % vec != 0) return PVQ_ERR_ALIGNMENT;
+    }
+    if (need & NEED_OUT) {
+        if (!d.d_out || d.ld_out < d.cols) return PVQ_ERR_INVALID_ARG;
+        if (!is_aligned(d.d_out, 16) || d.ld_out % 8 != 0) return PVQ_ERR_ALIGNMENT;
+    }
+    if (need & NEED_CODES) {
+        if (!d.d_codes || !d.d_scale_idx || !d.d_row_norm) return PVQ_ERR_INVALID_ARG;
+        if (!is_aligned(d.d_codes, 4) || !is_aligned(d.d_scale_idx, 4) || !is_aligned(d.d_row_norm, 4))
+            return PVQ_ERR_ALIGNMENT;
+    }
+    if ((need & NEED_EDGES) && !d.d_edges) return PVQ_ERR_INVALID_ARG;
+    if ((need & NEED_LEVELS) && !d.d_levels) return PVQ_ERR_INVALID_ARG;
+    m->x = d.d_x;
+    m->out = d.d_out;
+    m->codes = d.d_codes;
+    m->scale_idx = d.d_scale_idx;
+    m->row_norm = d.d_row_norm;
+    m->edges = d.d_edges;
+    m->levels = d.d_levels;
+    m->rows = d.rows;
+    m->cols = d.cols;
+    m->ld = d.ld;
+    m->ld_out = d.ld_out;
+    m->G = static_cast<int>(G);
+    m->sstride = static_cast<int>(pvq_scale_row_stride(G, c.scale_bits));
+    m->rows_per_tile = 1;
+    m->tile_begin = 0;
+    return PVQ_OK;
+}
+
+int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int N, int K, int scale_bits,
+              const uint32_t* d_table, uint32_t* d_status, int kind /*0 enc,1 dec,2 fused*/,
+              pvq_stream_t stream) {
+    if (!descs || count < 1 || count > kMaxBatch) return PVQ_ERR_INVALID_ARG;
+    if (kind != 1 && dtype != PVQ_DTYPE_F32 && dtype != PVQ_DTYPE_BF16) return PVQ_ERR_INVALID_ARG;
+    Common c;
+    int st = check_common(N, K, scale_bits, d_table, &c);
+    if (st != PVQ_OK) return st;
+    BatchArgs a;
+    std::memset(&a, 0, sizeof a);
+    a.count = count;
+    a.K = K;
+    a.scale_bits = scale_bits;
+    a.table = d_table;
+    a.status = d_status;
+    for (int i = 0; i < count; ++i) {
+        st = fill_matrix(descs[i], need, dtype, c, &a.m[i]);
+        if (st != PVQ_OK) return st;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (kind == 1) return launch_decode(a, c.N, c.W, s);
+    return launch_encode(a, dtype, c.N, c.W, kind == 2, s);
+}
+
+}  // namespace
+
+extern "C" int pvq_encode(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+                          int scale_bits, const uint32_t* d_table, const float* d_edges, uint32_t* d_codes,
+                          uint8_t* d_scale_idx, float* d_row_norm, pvq_stream_t stream) {
+    pvq_matrix_desc d;
+    std::memset(&d, 0, sizeof d);
+    d.d_x = d_x;
+    d.d_codes = d_codes;
+    d.d_scale_idx = d_scale_idx;
+    d.d_row_norm = d_row_norm;
+    d.d_edges = d_edges;
+    d.rows = rows;
+    d.cols = cols;
+    d.ld = ld;
+    return run_batch(&d, 1, NEED_X | NEED_CODES | NEED_EDGES, dtype, N, K, scale_bits, d_table, nullptr, 0,
+                     stream);
+}
+
+extern "C" int pvq_decode(const uint32_t* d_codes, const uint8_t* d_scale_idx, const float* d_row_norm,
+                          int64_t rows, int64_t cols, int N, int K, int scale_bits, const uint32_t* d_table,
+                          const float* d_levels, void* d_out, int64_t ld_out, uint32_t* d_status,
+                          pvq_stream_t stream) {
+    pvq_matrix_desc d;
+    std::memset(&d, 0, sizeof d);
+    d.d_out = d_out;
+    d.d_codes = const_cast<uint32_t*>(d_codes);
+    d.d_scale_idx = const_cast<uint8_t*>(d_scale_idx);
+    d.d_row_norm = const_cast<float*>(d_row_norm);
+    d.d_levels = d_levels;
+    d.rows = rows;
+    d.cols = cols;
+    d.ld_out = ld_out;
+    return run_batch(&d, 1, NEED_OUT | NEED_CODES | NEED_LEVELS, PVQ_DTYPE_BF16, N, K, scale_bits, d_table,
+                     d_status, 1, stream);
+}
+
+extern "C" int pvq_roundtrip(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+                             int scale_bits, const uint32_t* d_table, const float* d_edges,
+                             const float* d_levels, void* d_out, int64_t ld_out, pvq_stream_t stream) {
+    pvq_matrix_desc d;
+    std::memset(&d, 0, sizeof d);
+    d.d_x = d_x;
+    d.d_out = d_out;
+    d.d_edges = d_edges;
+    d.d_levels = d_levels;
+    d.rows = rows;
+    d.cols = cols;
+    d.ld = ld;
+    d.ld_out = ld_out;
+    return run_batch(&d, 1, NEED_X | NEED_OUT | NEED_EDGES | NEED_LEVELS, dtype, N, K, scale_bits, d_table,
+                     nullptr, 2, stream);
+}
+
+extern "C" int pvq_encode_batched(const pvq_matrix_desc* descs, int count, int dtype, int N, int K,
+                                  int scale_bits, const uint32_t* d_table, pvq_stream_t stream) {
+    return run_batch(descs, count, NEED_X | NEED_CODES | NEED_EDGES, dtype, N, K, scale_bits, d_table,
+                     nullptr, 0, stream);
+}
+
+extern "C" int pvq_decode_batched(const pvq_matrix_desc* descs, int count, int N, int K, int scale_bits,
+                                  const uint32_t* d_table, uint32_t* d_status, pvq_stream_t stream) {
+    return run_batch(descs, count, NEED_OUT | NEED_CODES | NEED_LEVELS, PVQ_DTYPE_BF16, N, K, scale_bits,
+                     d_table, d_status, 1, stream);
+}

@@ -1,0 +1,175 @@
+// Set-up kernels: the count table N(n,k) (Sec. 2.4, App. C.2 / Algorithm 4) and
+// the amplitude codebook (Sec. 3.4).  Both are cold: they run once per (N,K)
+// or per (N,G,b).
+#include "mp_uint.cuh"
+#include "pvq_internal.cuh"
+
+namespace pvq {
+
+// ------------------------------------------------------------- count table
+//
+// One thread block, thread k owns column k and keeps N(n,k) in registers while
+// the block walks the rows n = 0, 1, ...:
+//   a_k = N(n-1,k) + N(n-1,k-1)   (the diagonal term, from the neighbour's value)
+//   N(n,k) = sum_{i<=k} a_i, a_0 = 1   (inclusive prefix sum over k)
+// which is the recurrence N(n,k) = N(n-1,k) + N(n,k-1) + N(n-1,k-1) unrolled
+// along k.  The prefix sum is a Hillis-Steele scan through shared memory.  A
+// table of this size never needs more than one block, so there is no
+// inter-block barrier.
+template <int W>
+__global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, uint32_t* __restrict__ table) {
+    extern __shared__ uint32_t sm[];  // two buffers of (K+1) entries of W words
+    const int k = threadIdx.x;
+    const int KP = K + 1;
+    uint32_t* buf0 = sm;
+    uint32_t* buf1 = sm + static_cast<size_t>(KP) * W;
+    const bool live = k < KP;
+
+    mp<W> v;  // N(n,k) for the current row
+    mp_zero(v);
+    if (k == 0) v.w[0] = 1u;  // row 0: N(0,0) = 1, N(0,k>=1) = 0
+
+    for (int n = 0; n < N; ++n) {
+        if (live) {
+#pragma unroll
+            for (int w = 0; w < W; ++w) table[(static_cast<size_t>(n) * KP + k) * W + w] = v.w[w];
+#pragma unroll
+            for (int w = 0; w < W; ++w) buf0[k * W + w] = v.w[w];
+        }
+        __syncthreads();
+        // a_k = N(n,k) + N(n,k-1) for the next row; a_0 = 1
+        if (live) {
+            if (k == 0) {
+                mp_zero(v);
+                v.w[0] = 1u;
+            } else {
+                mp<W> left = mp_load<W>(buf0 + (k - 1) * W);
+                mp_add<W>(v, left);
+            }
+        }
+        __syncthreads();
+        // inclusive scan of a over k
+        uint32_t* src = buf0;
+        uint32_t* dst = buf1;
+        for (int off = 1; off < KP; off <<= 1) {
+            if (live) {
+#pragma unroll
+                for (int w = 0; w < W; ++w) src[k * W + w] = v.w[w];
+            }
+            __syncthreads();
+            if (live && k >= off) {
+                mp<W> o = mp_load<W>(src + (k - off) * W);
+                mp_add<W>(v, o);
+            }
+            uint32_t* t = src;
+            src = dst;
+            dst = t;
+        }
+        __syncthreads();
+    }
+}
+
+template <int W>
+static int launch_count_table(int N, int K, uint32_t* d_table, cudaStream_t s) {
+    const int threads = ((K + 1 + 31) / 32) * 32;
+    const size_t smem = 2u * static_cast<size_t>(K + 1) * W * sizeof(uint32_t);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(count_table_kernel<W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+        if (e != cudaSuccess) return set_cuda_error(e);
+    }
+    count_table_kernel<W><<<1, threads, smem, s>>>(N, K, d_table);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
+}
+
+// ---------------------------------------------------------- scale codebook
+//
+// u = ||x_g||^2 / ||x_row||^2 ~ Beta(a, b) with a = N/2, b = N(G-1)/2, both
+// integers for even N.  For integer parameters the CDF is a binomial tail:
+//   I_x(a,b) = P[ Bin(n, x) >= a ],  n = a + b - 1
+//            = 1 - sum_{j<a} C(n,j) x^j (1-x)^(n-j),
+// a sum of a <= N/2 positive terms, evaluated in fp64.  The quantile is found
+// by bisection on x until the bracket is one fp64 spacing wide.
+__device__ double beta_cdf_int(double x, int a, int n) {
+    if (x <= 0.0) return 0.0;
+    if (x >= 1.0) return 1.0;
+    double t = exp(static_cast<double>(n) * log1p(-x));  // (1-x)^n
+    const double ratio = x / (1.0 - x);
+    double sum = 0.0;
+    for (int j = 0; j < a; ++j) {
+        sum += t;
+        t = t * (static_cast<double>(n - j) / static_cast<double>(j + 1)) * ratio;
+    }
+    return 1.0 - sum;
+}
+
+__device__ double beta_ppf_int(double p, int a, int n) {
+    double lo = 0.0, hi = 1.0;
+    for (int it = 0; it < 1100; ++it) {
+        const double mid = 0.5 * (lo + hi);
+        if (mid <= lo || mid >= hi) break;
+        if (beta_cdf_int(mid, a, n) < p)
+            lo = mid;
+        else
+            hi = mid;
+    }
+    return 0.5 * (lo + hi);
+}
+
+__global__ void scale_codebook_kernel(int a, int n, int scale_bits, float* __restrict__ edges,
+                                      float* __restrict__ levels) {
+    const int L = 1 << scale_bits;
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < L - 1) {
+        if (edges) edges[t] = static_cast<float>(beta_ppf_int(static_cast<double>(t + 1) / L, a, n));
+    } else if (t < 2 * L - 1) {
+        const int q = t - (L - 1);
+        if (levels) levels[q] = static_cast<float>(sqrt(beta_ppf_int((q + 0.5) / L, a, n)));
+    }
+}
+
+}  // namespace pvq
+
+using namespace pvq;
+
+extern "C" int pvq_build_count_table(int N, int K, uint32_t* d_table, size_t bytes, pvq_stream_t stream) {
+    if (!d_table || N < 1 || K < 1) return PVQ_ERR_INVALID_ARG;
+    if (N > 256 || K > kMaxPulses) return PVQ_ERR_UNSUPPORTED;
+    const int W = code_words_for(N, K);
+    if (W == 0) return PVQ_ERR_INVALID_ARG;
+    if (W > kMaxWords) return PVQ_ERR_UNSUPPORTED;
+    if (!is_aligned(d_table, 16)) return PVQ_ERR_ALIGNMENT;
+    if (bytes < pvq_count_table_bytes(N, K)) return PVQ_ERR_TABLE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (W) {
+        case 1: return launch_count_table<1>(N, K, d_table, s);
+        case 2: return launch_count_table<2>(N, K, d_table, s);
+        case 3: return launch_count_table<3>(N, K, d_table, s);
+        case 4: return launch_count_table<4>(N, K, d_table, s);
+        case 5: return launch_count_table<5>(N, K, d_table, s);
+        case 6: return launch_count_table<6>(N, K, d_table, s);
+        case 7: return launch_count_table<7>(N, K, d_table, s);
+        case 8: return launch_count_table<8>(N, K, d_table, s);
+        case 9: return launch_count_table<9>(N, K, d_table, s);
+        case 10: return launch_count_table<10>(N, K, d_table, s);
+        case 11: return launch_count_table<11>(N, K, d_table, s);
+        case 12: return launch_count_table<12>(N, K, d_table, s);
+        default: return PVQ_ERR_UNSUPPORTED;
+    }
+}
+
+extern "C" int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, float* d_levels,
+                                        pvq_stream_t stream) {
+    if (N < 2 || (N & 1) || G < 2 || scale_bits < 1 || scale_bits > 8) return PVQ_ERR_INVALID_ARG;
+    if (!d_edges && !d_levels) return PVQ_ERR_INVALID_ARG;
+    const int64_t n64 = static_cast<int64_t>(N) * G / 2 - 1;  // a + b - 1
+    if (n64 > (int64_t(1) << 30)) return PVQ_ERR_UNSUPPORTED;
+    const int L = 1 << scale_bits;
+    const int threads = 64;
+    const int blocks = (2 * L - 1 + threads - 1) / threads;
+    scale_codebook_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(
+        N / 2, static_cast<int>(n64), scale_bits, d_edges, d_levels);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
+}

@@ -1,0 +1,253 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle
+on the same seeded inputs.  Codes, amplitude indices, row norms and decoded bf16
+values must match bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import beta_codebook as bc
+from oracle import pvq_oracle as po
+from paper_2410_16926_b200 import inputs, pvq
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def as_u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def bf16_bits(t):
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def to_device(x_np, kind):
+    if kind == "bf16":
+        return torch.from_numpy(x_np.view(np.int16)).to(DEV).view(torch.bfloat16)
+    return torch.from_numpy(x_np).to(DEV)
+
+
+class Codec:
+    """Device tables for one (N, index_bits, G, scale_bits); the codebook is the oracle's,
+    so that parity of the hot path does not hinge on two ways of computing quantiles."""
+
+    def __init__(self, N, index_bits, G, b, K=None):
+        self.N, self.G, self.b = N, G, b
+        self.K = pvq.max_pulses(N, index_bits) if K is None else K
+        self.W = pvq.code_words(N, self.K)
+        self.table = pvq.build_count_table(N, self.K)
+        self.edges_np = bc.edges_f32(N, G, b)
+        self.levels_np = bc.levels_amp_f32(N, G, b)
+        self.edges = torch.from_numpy(self.edges_np).to(DEV)
+        self.levels = torch.from_numpy(self.levels_np).to(DEV)
+
+
+def check_encode(cd, x_np, kind, x_dev=None):
+    x_dev = to_device(x_np, kind) if x_dev is None else x_dev
+    codes, sidx, rnorm = pvq.encode(x_dev, cd.N, cd.K, cd.b, cd.table, cd.edges)
+    torch.cuda.synchronize()
+    o_codes, o_sidx, o_rnorm = po.encode(x_np, cd.N, cd.K, cd.b, cd.edges_np, W=cd.W)
+    assert np.array_equal(rnorm.cpu().numpy().view(np.uint32), o_rnorm.view(np.uint32)), "row norms"
+    assert np.array_equal(sidx.cpu().numpy(), o_sidx), "amplitude indices"
+    bad = np.argwhere(as_u32(codes) != o_codes)
+    assert bad.size == 0, "codes differ first at (row, group, word) %s" % (bad[0],)
+    return (codes, sidx, rnorm), (o_codes, o_sidx, o_rnorm)
+
+
+def check_decode(cd, enc_dev, enc_np):
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = pvq.decode(*enc_dev, cd.N, cd.K, cd.b, cd.table, cd.levels, status=status)
+    torch.cuda.synchronize()
+    o_out, o_status = po.decode(*enc_np, cd.N, cd.K, cd.b, cd.levels_np)
+    assert int(status.item()) == o_status
+    bad = np.argwhere(bf16_bits(out) != o_out)
+    assert bad.size == 0, "decoded values differ first at %s" % (bad[0],)
+    return out
+
+
+# ------------------------------------------------------------------ set-up kernels
+
+@pytest.mark.parametrize("N,K", [(8, 6), (8, 40), (16, 18), (32, 22), (32, 50), (64, 96), (32, 1), (128, 187)])
+def test_count_table_word_for_word(N, K):
+    W = pvq.code_words(N, K)
+    t = pvq.build_count_table(N, K)
+    torch.cuda.synchronize()
+    ref = po.count_table(N, K, W)[:N]          # rows n = 0..N-1
+    assert np.array_equal(as_u32(t), ref)
+
+
+@pytest.mark.parametrize("N,G,b", [(32, 16, 8), (32, 128, 4), (32, 448, 8), (64, 448, 6), (32, 128, 8),
+                                   (8, 2, 3), (16, 5, 1)])
+def test_scale_codebook_against_scipy(N, G, b):
+    edges, levels = pvq.build_scale_codebook(N, G, b)
+    torch.cuda.synchronize()
+    e, l = edges.cpu().numpy(), levels.cpu().numpy()
+    re_, rl = bc.edges_f32(N, G, b), bc.levels_amp_f32(N, G, b)
+    # fp64 quantiles from two unrelated algorithms, each rounded once to fp32: at most one ulp apart
+    assert np.all(np.abs(e.view(np.int32) - re_.view(np.int32)) <= 1)
+    assert np.all(np.abs(l.view(np.int32) - rl.view(np.int32)) <= 1)
+    assert np.mean(e.view(np.int32) == re_.view(np.int32)) > 0.98
+    assert np.all(np.diff(e) > 0)
+
+
+# ------------------------------------------------------------------------ hot path
+
+SMALL = [
+    # N, index_bits, rows, cols, scale_bits, dtype
+    (8, 24, 7, 64, 3, "f32"),
+    (8, 40, 5, 24, 5, "bf16"),       # G = 3
+    (16, 40, 33, 208, 4, "bf16"),    # G = 13
+    (32, 64, 70, 512, 8, "f32"),     # several tiles, ragged last tile
+    (32, 96, 37, 4096, 4, "bf16"),   # G = 128
+    (32, 96, 9, 14336, 8, "bf16"),   # G = 448: not a power of two
+    (32, 128, 12, 1024, 6, "bf16"),  # 4-word codes
+    (64, 192, 11, 3584, 6, "bf16"),  # N = 64, 6-word codes, G = 56
+    (64, 64, 6, 640, 2, "f32"),      # few pulses per position
+]
+
+
+@pytest.mark.parametrize("N,bits,rows,cols,b,kind", SMALL)
+def test_encode_decode_parity(N, bits, rows, cols, b, kind):
+    rng = np.random.default_rng(N * 1000 + rows)
+    x = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+    cd = Codec(N, bits, cols // N, b)
+    enc_dev, enc_np = check_encode(cd, x_np, kind)
+    check_decode(cd, enc_dev, enc_np)
+
+
+def test_heavy_tails_and_outliers():
+    rng = np.random.default_rng(42)
+    x = (rng.standard_t(2.0, size=(24, 1024)) * 0.05).astype(np.float32)
+    x[3, 100] = 1e4
+    x[5, :32] = 0.0
+    x_np = inputs.f32_to_bf16_bits(x)
+    cd = Codec(32, 96, 32, 8)
+    enc_dev, enc_np = check_encode(cd, x_np, "bf16")
+    check_decode(cd, enc_dev, enc_np)
+
+
+def test_degenerate_inputs():
+    N, rows, cols = 32, 12, 256
+    x = np.zeros((rows, cols), dtype=np.float32)
+    rng = np.random.default_rng(1)
+    x[1] = rng.standard_normal(cols)              # ordinary row
+    x[2, 40] = -3.0                               # one non-zero in the whole row
+    x[3, :32] = 1.0                               # all-equal group: every residual ties
+    x[3, 32:64] = -0.5
+    x[4] = rng.standard_normal(cols)
+    x[4, 64:96] = 0.0                             # zero group inside a non-zero row
+    x[5] = -0.0                                   # negative zeros only
+    x[6] = np.round(rng.standard_normal(cols) * 4) / 4      # many equal magnitudes
+    x[7] = rng.standard_normal(cols) * 1e-30      # tiny values
+    x[8] = rng.standard_normal(cols) * 1e15       # large but finite sums of squares
+    x[9, ::2] = 1.0
+    x[9, 1::2] = -1.0
+    x[10, 5] = 1e-45                              # smallest subnormal: K / l1 overflows
+    x[11] = rng.standard_normal(cols)
+    x[11, 31] = 100.0                             # all pulses of a group in its last position
+    cd = Codec(N, 64, cols // N, 8)
+    for kind in ("f32", "bf16"):
+        x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+        enc_dev, enc_np = check_encode(cd, x_np, kind)
+        check_decode(cd, enc_dev, enc_np)
+
+
+def test_leading_dimensions():
+    N, rows, cols, ld, ldo = 32, 10, 256, 320, 288
+    rng = np.random.default_rng(8)
+    x = inputs.f32_to_bf16_bits((rng.standard_normal((rows, cols))).astype(np.float32))
+    cd = Codec(N, 96, cols // N, 4)
+    big = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
+    big[:, :cols] = to_device(x, "bf16")
+    enc_dev, enc_np = check_encode(cd, x, "bf16", x_dev=big[:, :cols])
+    out_big = torch.full((rows, ldo), 7.0, dtype=torch.bfloat16, device=DEV)
+    pvq.decode(*enc_dev, cd.N, cd.K, cd.b, cd.table, cd.levels, out=out_big[:, :cols])
+    torch.cuda.synchronize()
+    o_out, _ = po.decode(*enc_np, cd.N, cd.K, cd.b, cd.levels_np)
+    assert np.array_equal(bf16_bits(out_big[:, :cols].contiguous()), o_out)
+    assert torch.all(out_big[:, cols:] == 7.0)       # nothing written past cols
+
+
+def test_invalid_codes_set_status_and_decode_to_zero():
+    cd = Codec(32, 64, 8, 8)
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((4, 256)).astype(np.float32)
+    enc_dev, enc_np = check_encode(cd, x, "f32")
+    codes = enc_np[0].copy()
+    codes[1, 3, :] = 0xFFFFFFFF                      # >= N(32,22)
+    total = po.code_to_int(po.count_table(32, cd.K, 3)[32, cd.K])
+    codes[2, 0, :] = po.int_to_code(total, 2)         # the first invalid value
+    codes[2, 1, :] = po.int_to_code(total - 1, 2)     # the last valid one
+    enc_np2 = (codes, enc_np[1], enc_np[2])
+    enc_dev2 = (torch.from_numpy(codes.view(np.int32)).to(DEV), enc_dev[1], enc_dev[2])
+    out = check_decode(cd, enc_dev2, enc_np2)
+    assert torch.all(out[1, 96:128] == 0) and torch.all(out[2, :32] == 0)
+    assert torch.any(out[2, 32:64] != 0)
+
+
+def test_fused_roundtrip_equals_encode_then_decode():
+    for (N, bits, rows, cols, b, kind) in [(32, 64, 40, 4096, 8, "bf16"), (16, 40, 9, 208, 4, "f32"),
+                                           (64, 192, 5, 3584, 6, "bf16")]:
+        rng = np.random.default_rng(rows)
+        x = rng.standard_normal((rows, cols)).astype(np.float32)
+        x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+        cd = Codec(N, bits, cols // N, b)
+        out = pvq.roundtrip(to_device(x_np, kind), cd.N, cd.K, cd.b, cd.table, cd.edges, cd.levels)
+        torch.cuda.synchronize()
+        enc = po.encode(x_np, cd.N, cd.K, cd.b, cd.edges_np, W=cd.W)
+        o_out, _ = po.decode(*enc, cd.N, cd.K, cd.b, cd.levels_np)
+        assert np.array_equal(bf16_bits(out), o_out)
+
+
+def test_batched_calls_match_single_calls():
+    wl = inputs.config3(scale_div=256)       # the seven matrices of a layer, 1/256 of the rows
+    N, b = wl.N, wl.scale_bits
+    K = pvq.max_pulses(N, wl.index_bits)
+    W = pvq.code_words(N, K)
+    table = pvq.build_count_table(N, K)
+    items, refs = [], []
+    books = {}
+    for m in wl.matrices:
+        G = m.cols // N
+        if G not in books:
+            books[G] = (bc.edges_f32(N, G, b), bc.levels_amp_f32(N, G, b))
+        e_np, l_np = books[G]
+        codes, sidx, rnorm = pvq.alloc_encoded(m.rows, G, W, b)
+        items.append(dict(x=to_device(m.data, "bf16"), codes=codes, scale_idx=sidx, row_norm=rnorm,
+                          edges=torch.from_numpy(e_np).to(DEV), levels=torch.from_numpy(l_np).to(DEV),
+                          out=torch.empty((m.rows, m.cols), dtype=torch.bfloat16, device=DEV), cols=m.cols))
+        enc = po.encode(m.data, N, K, b, e_np, W=W)
+        refs.append((enc, po.decode(*enc, N, K, b, l_np)[0]))
+    pvq.encode_batched(items, torch.bfloat16, N, K, b, table)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    pvq.decode_batched(items, N, K, b, table, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for it, (enc, out) in zip(items, refs):
+        assert np.array_equal(as_u32(it["codes"]), enc[0])
+        assert np.array_equal(it["scale_idx"].cpu().numpy(), enc[1])
+        assert np.array_equal(it["row_norm"].cpu().numpy().view(np.uint32), enc[2].view(np.uint32))
+        assert np.array_equal(bf16_bits(it["out"]), out)
+
+
+def test_library_codebook_end_to_end():
+    # With the library's own codebook the amplitude indices may differ from the oracle's only
+    # where u sits within an ulp of an edge; the direction codes do not depend on it.
+    N, G, b = 32, 128, 4
+    wl = inputs.config2(rows=64)
+    x_np = wl.matrices[0].data
+    K = pvq.max_pulses(N, 96)
+    table = pvq.build_count_table(N, K)
+    edges, levels = pvq.build_scale_codebook(N, G, b)
+    codes, sidx, rnorm = pvq.encode(to_device(x_np, "bf16"), N, K, b, table, edges)
+    torch.cuda.synchronize()
+    o_codes, o_sidx, o_rnorm = po.encode(x_np, N, K, b, bc.edges_f32(N, G, b))
+    assert np.array_equal(as_u32(codes), o_codes)
+    q = po.unpack_scale_idx(sidx.cpu().numpy(), G, b)
+    oq = po.unpack_scale_idx(o_sidx, G, b)
+    assert np.mean(q != oq) < 1e-3 and np.max(np.abs(q - oq)) <= 1
+    # uniform bin occupancy on Gaussian rows (Sec. 3.4): every 4-bit bin near 1/16
+    occ = np.bincount(q.ravel(), minlength=16) / q.size
+    assert np.all(np.abs(occ - 1 / 16) < 0.02)

@@ -1,0 +1,113 @@
+"""CPU-only checks of the C-ABI library: it loads, exports what include/pvq.h
+declares, its host helpers agree with the oracle, and bad arguments are turned
+into status codes before any CUDA work."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from oracle import pvq_oracle as po
+from paper_2410_16926_b200 import pvq
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "pvq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pvq_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = pvq.lib()
+    names = declared_functions()
+    assert len(names) >= 14
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(pvq.EXPORTS) == names
+
+
+def test_strerror():
+    for s in range(0, 7):
+        assert pvq.lib().pvq_strerror(s)
+    assert b"OK" in pvq.lib().pvq_strerror(0)
+
+
+@pytest.mark.parametrize("N,bits", [(32, 64), (32, 96), (64, 192), (16, 40), (8, 24), (128, 384)])
+def test_pulse_selection_matches_oracle(N, bits):
+    K = pvq.max_pulses(N, bits)
+    assert K == po.max_pulses(N, bits)
+    assert pvq.index_bits(N, K) == po.index_bits(N, K) <= bits
+    assert pvq.index_bits(N, K + 1) > bits
+    W = pvq.code_words(N, K)
+    assert W == (bits + 31) // 32
+    assert pvq.count_table_bytes(N, K) == N * (K + 1) * W * 4
+
+
+def test_index_bits_small_cases():
+    # N(2,7) = 28 -> 5 bits; N(1,k) = 2 -> 1 bit; N(n,0) = 1 -> 0 bits
+    assert pvq.index_bits(2, 7) == 5
+    assert pvq.index_bits(1, 9) == 1
+    assert pvq.index_bits(5, 0) == 0
+    for n in range(1, 12):
+        for k in range(0, 12):
+            assert pvq.index_bits(n, k) == po.index_bits(n, k)
+
+
+def test_scale_row_stride():
+    for G in (1, 2, 5, 16, 128, 448, 1000):
+        for b in range(1, 9):
+            assert pvq.scale_row_stride(G, b) == po.scale_row_stride(G, b)
+    assert pvq.scale_row_stride(128, 4) == 64
+    assert pvq.scale_row_stride(448, 6) == 336
+    assert pvq.scale_row_stride(5, 3) == 4
+
+
+def test_bad_arguments_are_rejected_without_a_gpu():
+    L = pvq.lib()
+    buf = (C.c_uint32 * 64)()
+    p = C.cast(buf, C.c_void_p)
+    INVALID, UNSUPPORTED, ALIGN, SMALL = 1, 2, 3, 4
+    # table builder
+    assert L.pvq_build_count_table(32, 22, None, 1 << 20, None) == INVALID
+    assert L.pvq_build_count_table(0, 22, p, 1 << 20, None) == INVALID
+    assert L.pvq_build_count_table(32, 22, p, 16, None) == SMALL
+    assert L.pvq_build_count_table(32, 5000, p, 1 << 30, None) == UNSUPPORTED
+    assert L.pvq_build_count_table(32, 22, C.c_void_p(p.value + 4), 1 << 20, None) == ALIGN
+    # codebook
+    assert L.pvq_build_scale_codebook(32, 1, 4, p, p, None) == INVALID
+    assert L.pvq_build_scale_codebook(32, 16, 9, p, p, None) == INVALID
+    assert L.pvq_build_scale_codebook(31, 16, 4, p, p, None) == INVALID
+    assert L.pvq_build_scale_codebook(32, 16, 4, None, None, None) == INVALID
+    # encode
+    enc = lambda x=p, dt=1, rows=4, cols=64, ld=64, N=32, K=22, b=8, tab=p, e=p, c=p, s=p, r=p: \
+        L.pvq_encode(x, dt, rows, cols, ld, N, K, b, tab, e, c, s, r, None)
+    assert enc(x=None) == INVALID
+    assert enc(cols=48) == INVALID          # not a multiple of N
+    assert enc(N=24) == INVALID             # not a power of two
+    assert enc(b=0) == INVALID
+    assert enc(dt=7) == INVALID
+    assert enc(ld=32) == INVALID            # ld < cols
+    assert enc(cols=32, ld=32) == UNSUPPORTED   # one group per row: no quantile codebook
+    assert enc(N=128, cols=256, ld=256) == UNSUPPORTED
+    assert enc(ld=68) == ALIGN
+    assert enc(x=C.c_void_p(p.value + 2)) == ALIGN
+    assert enc(tab=None) == INVALID
+    assert enc(e=None) == INVALID
+    assert enc(K=0) == INVALID
+    # decode
+    dec = lambda c=p, s=p, r=p, rows=4, cols=64, N=32, K=22, b=8, tab=p, lev=p, out=p, ldo=64: \
+        L.pvq_decode(c, s, r, rows, cols, N, K, b, tab, lev, out, ldo, None, None)
+    assert dec(out=None) == INVALID
+    assert dec(c=None) == INVALID
+    assert dec(lev=None) == INVALID
+    assert dec(ldo=60) == INVALID
+    assert dec(ldo=68) == ALIGN
+    assert dec(rows=0) == INVALID
+    # batched
+    assert L.pvq_encode_batched(None, 1, 1, 32, 22, 8, p, None) == INVALID
+    d = (pvq.MatrixDesc * 1)()
+    assert L.pvq_encode_batched(d, 0, 1, 32, 22, 8, p, None) == INVALID
+    assert L.pvq_encode_batched(d, 33, 1, 32, 22, 8, p, None) == INVALID
+    assert L.pvq_decode_batched(d, 1, 32, 22, 8, p, None, None) == INVALID   # empty descriptor
