@@ -168,6 +168,38 @@ int pvq_encode_batched(const pvq_matrix_desc* descs, int count, int dtype, int N
 int pvq_decode_batched(const pvq_matrix_desc* descs, int count, int N, int K, int scale_bits,
                        const uint32_t* d_table, uint32_t* d_status, pvq_stream_t stream);
 
+/* ---- for callers that cannot allocate device memory ---------------------------------- */
+
+/* Size of the count table that is built into the library image (see below). */
+#define PVQ_STATIC_TABLE_BYTES (160u * 1024u)
+
+/* pvq_decode without a caller-provided count table.  (The paper has no counterpart: this
+ * is a packaging variant of pvq_decode, with identical results.)
+ *
+ * For hosts where device allocation is off limits once set-up is over - a plug-in inside
+ * an engine that has already planned all of its memory, a control loop whose allocator is
+ * frozen, a process whose memory budget is enforced by refusing cudaMalloc - the table
+ * N(n,k) is kept in a fixed array inside the library (PVQ_STATIC_TABLE_BYTES per GPU that
+ * loads the library, held until the process exits).  This call allocates and frees
+ * nothing, on the device or through any allocating library routine; codes, amplitude
+ * indices, row norms, levels and the output are still the caller's buffers, with the
+ * meaning and alignment they have in pvq_decode.
+ *
+ *   - (N,K) whose table needs more than PVQ_STATIC_TABLE_BYTES (pvq_count_table_bytes
+ *     tells) is refused with PVQ_ERR_TABLE_TOO_SMALL.
+ *   - The first call on a device looks up the array's device address and fills the table
+ *     on `stream`; so does any later call whose (N,K) differs from the previous call's on
+ *     that device.  Make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps what the last call put
+ *     there.  Nothing in it has to start at zero (the fill overwrites every word decode
+ *     reads).  Two calls with different (N,K) whose work overlaps on the GPU - different
+ *     streams, no dependency between them - race on the array; calls with the same (N,K)
+ *     only read it and may overlap freely once the first has been enqueued. */
+int pvq_decode_static_table(const uint32_t* d_codes, const uint8_t* d_scale_idx, const float* d_row_norm,
+                            int64_t rows, int64_t cols, int N, int K, int scale_bits,
+                            const float* d_levels, void* d_out, int64_t ld_out, uint32_t* d_status,
+                            pvq_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -65,6 +65,7 @@ def lib():
         L.pvq_roundtrip.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, vp, vp, i64, vp]
         L.pvq_encode_batched.argtypes = [C.POINTER(MatrixDesc), i32, i32, i32, i32, i32, vp, vp]
         L.pvq_decode_batched.argtypes = [C.POINTER(MatrixDesc), i32, i32, i32, i32, vp, vp, vp]
+        L.pvq_decode_static_table.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, i64, vp, vp]
         _lib = L
     return _lib
 
@@ -72,7 +73,7 @@ def lib():
 EXPORTS = ["pvq_strerror", "pvq_last_cuda_error", "pvq_index_bits", "pvq_max_pulses", "pvq_code_words",
            "pvq_count_table_bytes", "pvq_scale_row_stride", "pvq_build_count_table",
            "pvq_build_scale_codebook", "pvq_encode", "pvq_decode", "pvq_roundtrip", "pvq_encode_batched",
-           "pvq_decode_batched"]
+           "pvq_decode_batched", "pvq_decode_static_table"]
 
 
 def _check(status, where):
@@ -185,6 +186,22 @@ def decode(codes, sidx, rnorm, N, K, scale_bits, table, levels, out=None, status
                             rows, cols, N, K, scale_bits, _ptr(table, torch.int32),
                             _ptr(levels, torch.float32), _ptr(out, torch.bfloat16), out.stride(0),
                             _ptr(status, torch.int32), _stream()), "pvq_decode")
+    return out
+
+
+def decode_static_table(codes, sidx, rnorm, N, K, scale_bits, levels, out=None, status=None):
+    """decode() for callers that must not allocate on the device: the count table is the
+    one built into the library.  `out` has to be passed by such a caller; it is only
+    created here when omitted."""
+    rows, G, _ = codes.shape
+    cols = G * N
+    if out is None:
+        out = torch.empty((rows, cols), dtype=torch.bfloat16, device=codes.device)
+    _check(lib().pvq_decode_static_table(_ptr(codes, torch.int32), _ptr(sidx, torch.uint8),
+                                         _ptr(rnorm, torch.float32), rows, cols, N, K, scale_bits,
+                                         _ptr(levels, torch.float32), _ptr(out, torch.bfloat16),
+                                         out.stride(0), _ptr(status, torch.int32), _stream()),
+           "pvq_decode_static_table")
     return out
 
 
