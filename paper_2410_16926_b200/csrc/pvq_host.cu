@@ -157,7 +157,7 @@ extern "C" int pvq_code_words(int N, int K, int* W_out) {
 extern "C" size_t pvq_count_table_bytes(int N, int K) {
     int W = code_words_for(N, K);
     if (W == 0 || N < 1 || K < 1) return 0;
-    return static_cast<size_t>(N) * (static_cast<size_t>(K) + 1) * static_cast<size_t>(W) * 4u;
+    return table_layout(N, K, W).total;
 }
 
 extern "C" size_t pvq_scale_row_stride(int64_t G, int scale_bits) {

@@ -37,9 +37,60 @@ struct BatchArgs {
     unsigned total_tiles;
     int K;
     int scale_bits;
-    const uint32_t* table;
+    const uint32_t* table;  // the blob written by pvq_build_count_table (see TableLayout)
     uint32_t* status;
+    int walk_phases;        // decode: how many of the walk tables are staged in shared memory (1..3)
 };
+
+// Layout of the table blob.  Section 0 is the count table as the paper defines it,
+// [n][k][W] words for n = 0..N-1, k = 0..K.  The other sections are the same numbers
+// rearranged for the kernels, so that a thread block can stage them with one flat copy:
+//
+//   bound       N(N,K) as 8 words (codes are valid below it)
+//   walk[0]     rows by position i (row i holds N(N-1-i, .)), `rowlen` entries of
+//               `top_words` words each, entry (i, col) = N(N-1-i, col), zero padded
+//   walk[1]     same with 2-word entries, values that need more than 2 words replaced by
+//               2^64-1 (present when top_words > 2)
+//   walk[2]     same with 1-word entries saturated at 2^32-1 (present when top_words > 1)
+//
+// rowlen is K+1 rounded up to an even number: consecutive positions on a diagonal of the
+// table, (i, col) and (i+1, col+1), are then an odd number of entries apart, so threads that
+// sit on neighbouring diagonals' cells read different shared-memory banks.
+struct TableLayout {
+    int rowlen;
+    int top_words;
+    uint32_t bound_off;
+    uint32_t walk_off[3];
+    uint32_t walk_bytes[3];
+    uint32_t total;
+};
+
+__host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
+    TableLayout L;
+    if (N > 64 || W > 6) {  // no hot-path kernel for these: the blob is the plain count table
+        L.rowlen = 0;
+        L.top_words = 0;
+        L.bound_off = 0;
+        for (int p = 0; p < 3; ++p) L.walk_off[p] = L.walk_bytes[p] = 0;
+        L.total = static_cast<uint32_t>(N) * (K + 1) * W * 4u;
+        return L;
+    }
+    L.rowlen = (K + 2) & ~1;
+    L.top_words = W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : W));
+    uint32_t off = static_cast<uint32_t>(N) * (K + 1) * W * 4u;
+    off = (off + 127u) & ~127u;
+    L.bound_off = off;
+    off += 128u;
+    const uint32_t entries = static_cast<uint32_t>(N) * L.rowlen;
+    const int words[3] = {L.top_words, L.top_words > 2 ? 2 : 0, L.top_words > 1 ? 1 : 0};
+    for (int p = 0; p < 3; ++p) {
+        L.walk_off[p] = off;
+        L.walk_bytes[p] = entries * words[p] * 4u;
+        off += (L.walk_bytes[p] + 127u) & ~127u;
+    }
+    L.total = off;
+    return L;
+}
 
 // host helpers (pvq_host.cu)
 int set_cuda_error(cudaError_t e);  // records e, returns PVQ_ERR_CUDA

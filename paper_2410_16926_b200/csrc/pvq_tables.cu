@@ -69,6 +69,60 @@ __global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, uint32_
     }
 }
 
+// The other sections of the blob (TableLayout): the same numbers re-laid for the decode walk,
+// narrow copies saturated at their width, and N(N,K) itself.
+template <int W>
+__global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) {
+    const TableLayout L = table_layout(N, K, W);
+    if (L.rowlen == 0) return;
+    const int KP = K + 1;
+    const int entries = N * L.rowlen;
+    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < entries; e += gridDim.x * blockDim.x) {
+        const int i = e / L.rowlen;
+        const int col = e - i * L.rowlen;
+        const bool pad = col > K;  // never read; filled with all ones
+        uint32_t v[W];
+#pragma unroll
+        for (int w = 0; w < W; ++w)
+            v[w] = pad ? 0xffffffffu : blob[(static_cast<size_t>(N - 1 - i) * KP + col) * W + w];
+        uint32_t* top = blob + L.walk_off[0] / 4 + static_cast<size_t>(e) * L.top_words;
+        for (int w = 0; w < L.top_words; ++w) top[w] = w < W ? v[w] : 0u;
+        if (L.walk_bytes[1]) {
+            uint32_t hi = 0;
+#pragma unroll
+            for (int w = 2; w < W; ++w) hi |= v[w];
+            uint32_t* t2 = blob + L.walk_off[1] / 4 + static_cast<size_t>(e) * 2;
+            t2[0] = hi ? 0xffffffffu : v[0];
+            t2[1] = hi ? 0xffffffffu : (W > 1 ? v[W > 1 ? 1 : 0] : 0u);
+        }
+        if (L.walk_bytes[2]) {
+            uint32_t hi = 0;
+#pragma unroll
+            for (int w = 1; w < W; ++w) hi |= v[w];
+            blob[L.walk_off[2] / 4 + e] = hi ? 0xffffffffu : v[0];
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        // N(N,K) = N(N-1,K) + 2 sum_{j=1..K} N(N-1,K-j)   (every point of P(N,K) by its first
+        // coordinate: 0, or +-j with K-j pulses left for the other N-1)
+        uint32_t acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const uint32_t* row = blob + static_cast<size_t>(N - 1) * KP * W;
+        for (int col = 0; col <= K; ++col) {
+            const int times = col == K ? 1 : 2;
+            for (int rep = 0; rep < times; ++rep) {
+                unsigned long long carry = 0;
+                for (int w = 0; w < 8; ++w) {
+                    const unsigned long long add = w < W ? row[col * W + w] : 0u;
+                    const unsigned long long sum = static_cast<unsigned long long>(acc[w]) + add + carry;
+                    acc[w] = static_cast<uint32_t>(sum);
+                    carry = sum >> 32;
+                }
+            }
+        }
+        for (int w = 0; w < 8; ++w) blob[L.bound_off / 4 + w] = acc[w];
+    }
+}
+
 template <int W>
 static int launch_count_table(int N, int K, uint32_t* d_table, cudaStream_t s) {
     const int threads = ((K + 1 + 31) / 32) * 32;
@@ -80,6 +134,11 @@ static int launch_count_table(int N, int K, uint32_t* d_table, cudaStream_t s) {
     }
     count_table_kernel<W><<<1, threads, smem, s>>>(N, K, d_table);
     cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return set_cuda_error(e);
+    if (table_layout(N, K, W).rowlen != 0) {
+        derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, d_table);
+        e = cudaGetLastError();
+    }
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 

@@ -136,11 +136,17 @@ def scale_row_stride(G, scale_bits):
 # ---- set-up ---------------------------------------------------------------------
 
 def build_count_table(N, K, device="cuda"):
-    """Device table uint32 [N][K+1][W] of N(n,k)."""
-    W = code_words(N, K)
-    t = torch.empty((N, K + 1, W), dtype=torch.int32, device=device)
+    """The device table blob of pvq_build_count_table (flat int32): the count table N(n,k)
+    followed by the rearranged copies the kernels stage."""
+    t = torch.empty(count_table_bytes(N, K) // 4, dtype=torch.int32, device=device)
     _check(lib().pvq_build_count_table(N, K, _ptr(t), t.numel() * 4, _stream()), "pvq_build_count_table")
     return t
+
+
+def count_table_view(table, N, K):
+    """The first section of the blob: uint32 words [N][K+1][W] of N(n,k)."""
+    W = code_words(N, K)
+    return table[:N * (K + 1) * W].view(N, K + 1, W)
 
 
 def build_scale_codebook(N, G, scale_bits, device="cuda"):
@@ -168,7 +174,7 @@ def encode(x, N, K, scale_bits, table, edges, out=None):
     rows, cols = x.shape
     G = cols // N
     if out is None:
-        out = alloc_encoded(rows, G, table.shape[2], scale_bits, x.device)
+        out = alloc_encoded(rows, G, code_words(N, K), scale_bits, x.device)
     codes, sidx, rnorm = out
     _check(lib().pvq_encode(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), N, K, scale_bits,
                             _ptr(table, torch.int32), _ptr(edges, torch.float32), _ptr(codes, torch.int32),
