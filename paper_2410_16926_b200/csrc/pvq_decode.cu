@@ -1,162 +1,33 @@
 // Decode kernel: direction code -> pyramid point (Algorithm 3) -> unit sphere
 // times dequantised amplitude -> bf16 (Sec. 2.4, Sec. 3.4).
 //
-// One thread decodes one group; a warp takes 32 consecutive groups.  Algorithm 3
-// is run as a walk over the cells (i, col) of the count table, i the position
-// and col the pulses still to place, from (0, K) to (N, 0).  With r the part of
-// the code not yet explained and t = N(N-1-i, col), one step does
-//
-//   first test at a position:   r >= t   -> r -= t, one pulse here, go left (col-1)
-//                               else     -> y_i = 0, go down (i+1)
-//   after a pulse at i:         r >= 2t  -> r -= 2t, one more pulse, go left
-//                               else     -> y_i = -m if r >= t (then r -= t) else +m, go down
-//
-// which is Algorithm 3's loop with the test that fails for magnitude m and the
-// sign test read from the same table entry.  Every step goes left or down, so
-// every group takes exactly N + K steps and at step s sits on the anti-diagonal
-// i - col = s - K: the 32 threads of a warp run the same instructions with no
-// data-dependent branch, and their table reads fall on neighbouring diagonal
-// cells, which the table layout puts in different banks.
-//
-// r only shrinks.  Once every thread of the warp has r below 2^63 (2^31) the warp
-// continues in a copy of the loop that works on two-word (one-word) integers
-// and reads a table of that width, whose larger entries are saturated.
+// One thread decodes one group; a warp takes 32 consecutive groups, walks their
+// codes in lockstep (pvq_walk.cuh) and writes the 32 groups with coalesced
+// 16-byte stores from shared memory.
 #include <algorithm>
 
-#include "mp_uint.cuh"
-#include "pvq_internal.cuh"
+#include "pvq_walk.cuh"
 
 namespace pvq {
 
 namespace {
 
 constexpr int kDecThreads = 512;
-constexpr unsigned kFull = 0xffffffffu;
-
-// Shared-memory accesses of the walk by 32-bit shared-window address.
-__device__ __forceinline__ uint32_t shared_addr(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-template <int PW>
-__device__ __forceinline__ mp<PW> load_entry(uint32_t addr) {
-    mp<PW> t;
-    if constexpr (PW == 1) {
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t.w[0]) : "r"(addr));
-    } else if constexpr (PW == 2) {
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(t.w[0]), "=r"(t.w[1]) : "r"(addr));
-    } else if constexpr (PW <= 4) {  // 16-byte entries
-        uint32_t v[4];
-        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
-                     : "r"(addr));
-#pragma unroll
-        for (int w = 0; w < PW; ++w) t.w[w] = v[w];
-    } else {  // 24-byte entries, 8-byte aligned
-        uint32_t v[6];
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v[0]), "=r"(v[1]) : "r"(addr));
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+8];" : "=r"(v[2]), "=r"(v[3]) : "r"(addr));
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+16];" : "=r"(v[4]), "=r"(v[5]) : "r"(addr));
-#pragma unroll
-        for (int w = 0; w < PW; ++w) t.w[w] = v[w];
-    }
-    return t;
-}
-
-template <typename YT>
-__device__ __forceinline__ void store_y(uint32_t addr, int val) {
-    if constexpr (sizeof(YT) == 1)
-        asm volatile("st.shared.u8 [%0], %1;" ::"r"(addr), "r"(val) : "memory");
-    else
-        asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "r"(val) : "memory");
-}
-
-// State of one thread's walk.
-struct Walk {
-    int v;        // pulses placed at the current position so far
-    uint32_t y;   // shared address of this thread's slot for the current position
-    uint32_t y0;  // ... for position 0
-};
-
-// Runs steps s .. S-1 on PW-word integers with the table `tab` (entries of EB bytes),
-// leaving early, at a multiple of 8 steps, once every thread's r fits `next_words` words
-// with a bit to spare.  Returns the step reached.
-template <int PW, int EB, int CW, typename YT>
-__device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab, int rowlen, int K, int s,
-                                          const int S, const int next_words) {
-    mp<PW> r;
-#pragma unroll
-    for (int w = 0; w < PW; ++w) r.w[w] = rfull.w[w];
-    const int D = (rowlen + 1) * EB;                   // one step down and one right
-    const int i0 = static_cast<int>(st.y - st.y0) / static_cast<int>(sizeof(YT));  // position reached
-    uint32_t p = tab + i0 * D + (K - s) * EB;          // entry (i, col) of this step
-    int v = st.v;
-    uint32_t y = st.y;
-
-    auto step = [&]() {
-        const mp<PW> t = load_entry<PW>(p);
-        mp<PW> d2, d1;
-        const bool lt1 = mp_sub_borrow<PW>(d2, r, t);   // d2 = r - t
-        const bool lt2 = mp_sub_borrow<PW>(d1, d2, t);  // d1 = r - 2t
-        const bool placed = v > 0;
-        const bool ge1 = !lt1;
-        const bool ge2 = ge1 && !lt2 && placed;
-        const bool more = placed ? ge2 : ge1;  // another pulse at this position
-#pragma unroll
-        for (int w = 0; w < PW; ++w) r.w[w] = ge2 ? d1.w[w] : (ge1 ? d2.w[w] : r.w[w]);
-        if (!more) {
-            store_y<YT>(y, (ge1 && placed) ? -v : v);
-            y += sizeof(YT);
-            p += D;
-        }
-        v = more ? v + 1 : 0;
-        p -= EB;
-    };
-
-    while (s + 8 <= S) {
-        if (next_words > 0) {
-            // does r fit next_words words with the top bit clear?
-            uint32_t hi = 0;
-#pragma unroll
-            for (int w = 2; w < PW; ++w) hi |= r.w[w];
-            if constexpr (PW > 1) hi |= next_words == 2 ? (r.w[1] >> 31) : r.w[1];
-            if (next_words == 1) hi |= r.w[0] >> 31;
-            if (__all_sync(kFull, hi == 0u)) break;
-        }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) step();
-        s += 8;
-    }
-    if (next_words == 0 || s + 8 > S) {
-        for (; s < S; ++s) step();
-    }
-#pragma unroll
-    for (int w = 0; w < PW; ++w) rfull.w[w] = r.w[w];
-    st.v = v;
-    st.y = y;
-    return s;
-}
 
 template <int N, int W, typename YT>
 __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_constant__ BatchArgs a) {
     extern __shared__ __align__(16) uint8_t smem[];
-    constexpr int TW = W <= 2 ? W : (W <= 4 ? 4 : 6);  // words per entry of the widest table
     constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;  // bytes between two threads' slots
     const int K = a.K;
     const TableLayout L = table_layout(N, K, W);
-    const int phases = a.walk_phases;
-    const uint32_t tab_bytes = L.walk_off[phases - 1] + L.walk_bytes[phases - 1] - L.walk_off[0];
+    const uint32_t tab_bytes = walk_tables_bytes(L, a.walk_phases);
 
     {   // stage the walk tables: one flat copy
         const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(a.table) + L.walk_off[0]);
         uint4* dst = reinterpret_cast<uint4*>(smem);
         for (uint32_t q = threadIdx.x; q < tab_bytes / 16; q += blockDim.x) dst[q] = src[q];
     }
-    const uint32_t tab0 = shared_addr(smem);
-    const uint32_t tab2 = tab0 + (L.walk_off[1] - L.walk_off[0]);
-    const uint32_t tab1 = tab0 + (L.walk_off[2] - L.walk_off[0]);
-    const bool has2 = phases >= 2 && L.walk_bytes[1] != 0;
-    const bool has1 = phases >= 3;
+    const WalkTables wt = walk_tables(L, shared_addr(smem), a.walk_phases);
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -173,7 +44,6 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
     __syncthreads();
 
     const int b = a.scale_bits;
-    const int S = N + K;
     const unsigned warps_total = gridDim.x * (blockDim.x >> 5);
     bool bad = false;
 
@@ -207,71 +77,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
                 amp = __fmul_rn(m.row_norm[row], m.levels[q]);
             }
         }
-
-        // ---- the walk
-        Walk st;
-        st.v = 0;
-        st.y = st.y0 = shared_addr(yslots);
-        int s = 0;
-        s = walk_phase<W, TW * 4, W, YT>(c, st, tab0, L.rowlen, K, s, S, has2 ? 2 : (has1 ? 1 : 0));
-        if constexpr (W > 2) {
-            if (s < S && has2) s = walk_phase<2, 8, W, YT>(c, st, tab2, L.rowlen, K, s, S, has1 ? 1 : 0);
-        }
-        if constexpr (W > 1) {
-            if (s < S && has1) s = walk_phase<1, 4, W, YT>(c, st, tab1, L.rowlen, K, s, S, 0);
-        }
-
-        // ---- scale: point on the unit sphere times the amplitude
-        int ssy = 0;
-        if constexpr (sizeof(YT) == 1) {
-            const int* y4 = reinterpret_cast<const int*>(yslots);
-#pragma unroll
-            for (int v = 0; v < N / 4; ++v) ssy = __dp4a(y4[v], y4[v], ssy);
-        } else {
-#pragma unroll 8
-            for (int v = 0; v < N; ++v) ssy += static_cast<int>(yslots[v]) * static_cast<int>(yslots[v]);
-        }
-        wscale[lane] = __fdiv_rn(amp, __fsqrt_rn(static_cast<float>(ssy)));
-        __syncwarp();
-
-        // ---- coalesced stores: N/8 threads per group, 16 bytes each
-        constexpr int TPG = N / 8;       // threads per group
-        constexpr int GPI = 32 / TPG;    // groups per iteration
-        const int part = lane % TPG;
-#pragma unroll 1
-        for (int it = 0; it < TPG; ++it) {
-            const int gl = it * GPI + lane / TPG;  // group within the tile
-            const long long gj = g0 + gl;
-            if (gj < ngroups) {
-                const YT* ys = reinterpret_cast<const YT*>(wbuf + gl * YS) + part * 8;
-                const float sc = wscale[gl];
-                float f[8];
-                if constexpr (sizeof(YT) == 1) {
-                    const uint32_t lo = reinterpret_cast<const uint32_t*>(ys)[0];
-                    const uint32_t hi = reinterpret_cast<const uint32_t*>(ys)[1];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        f[e] = static_cast<float>(static_cast<int>(static_cast<int8_t>(lo >> (8 * e))));
-                        f[4 + e] = static_cast<float>(static_cast<int>(static_cast<int8_t>(hi >> (8 * e))));
-                    }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) f[e] = static_cast<float>(static_cast<int>(ys[e]));
-                }
-                const unsigned row = static_cast<unsigned>(gj) / static_cast<unsigned>(m.G);
-                const unsigned g = static_cast<unsigned>(gj) - row * static_cast<unsigned>(m.G);
-                uint4 o;
-                o.x = pack_bf16x2(__fmul_rn(f[0], sc), __fmul_rn(f[1], sc));
-                o.y = pack_bf16x2(__fmul_rn(f[2], sc), __fmul_rn(f[3], sc));
-                o.z = pack_bf16x2(__fmul_rn(f[4], sc), __fmul_rn(f[5], sc));
-                o.w = pack_bf16x2(__fmul_rn(f[6], sc), __fmul_rn(f[7], sc));
-                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.out) +
-                                                      static_cast<size_t>(row) * m.ld_out +
-                                                      static_cast<size_t>(g) * N + part * 8);
-                *dst = o;
-            }
-        }
-        __syncwarp();  // the slots are rewritten by the next tile
+        walk_code<N, W, YT>(c, wt, K, yslots);
+        emit_tile<N, YT>(m, wbuf, wscale, lane, amp, g0, ngroups);
     }
     if (bad && a.status) atomicOr(a.status, PVQ_STATUS_INVALID_CODE);
 }
@@ -299,19 +106,13 @@ int launch_decode_t(BatchArgs& a, cudaStream_t stream) {
     int threads = kDecThreads;
     int phases = 0;
     size_t smem = 0;
-    for (; threads >= 128 && phases == 0; threads /= 2) {
+    for (; threads >= 128; threads /= 2) {
         const size_t wbufs = static_cast<size_t>(threads / 32) * (32 * YS + 128);
-        for (int p = 3; p >= 1; --p) {
-            if (p > 1 && L.walk_bytes[p - 1] == 0) continue;
-            const size_t tab = L.walk_off[p - 1] + L.walk_bytes[p - 1] - L.walk_off[0];
-            const size_t need = ((tab + 15) & ~size_t(15)) + wbufs;
-            if (need <= static_cast<size_t>(smem_max)) {
-                phases = p;
-                smem = need;
-                break;
-            }
+        phases = walk_phases_that_fit(L, static_cast<size_t>(smem_max) - std::min<size_t>(smem_max, wbufs));
+        if (phases) {
+            smem = ((walk_tables_bytes(L, phases) + 15u) & ~size_t(15)) + wbufs;
+            break;
         }
-        if (phases) break;
     }
     if (phases == 0) return PVQ_ERR_UNSUPPORTED;
     a.walk_phases = phases;

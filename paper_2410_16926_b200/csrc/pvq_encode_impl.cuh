@@ -3,13 +3,12 @@
 //
 // One thread encodes one group; a thread block covers whole rows (the row norm
 // is the only quantity shared between groups).  Steps per group, in the order
-// of Sec. 3.3: group norms, row norm, amplitude index (Step 5), direction
-// (Step 3: l1 scale, floor, greedy fix-up), Fischer index (Step 7, Algorithm 2).
+// of Sec. 3.3: group norms, row norm, direction (Step 3: l1 scale, floor,
+// greedy fix-up), Fischer index (Step 7, Algorithm 2), amplitude index (Step 5).
 #pragma once
 #include <algorithm>
 
-#include "mp_uint.cuh"
-#include "pvq_internal.cuh"
+#include "pvq_walk.cuh"
 
 namespace pvq {
 
@@ -36,110 +35,195 @@ __device__ __forceinline__ void sort_desc(float (&v)[N]) {
     }
 }
 
-// Direction of one group (Sec. 2.5 / Algorithm 1 in the floor + greedy reading).
-//   a_i = |x_i| * (K / l1), m_i = floor(a_i), e_i = a_i - m_i, d = K - sum m_i.
-// The greedy loop "give one pulse to the largest residual, lowest index first
-// among equals, d times" touches every element at most once when 0 <= d <= N
-// (after its pulse an element's residual is negative, below every untouched
-// one), so its result is: the d elements with the largest (e_i, -i) get +1.
-// They are found with a sorting network on the residuals: v = d-th largest
-// value; everything above v gets a pulse, and the elements equal to v share
-// what is left, lowest index first.
+// v[idx] for a run-time idx in [0, N): a binary tree of selects on the bits of idx.
 template <int N>
-__device__ __forceinline__ void quantize_direction(const float (&x)[N], float l1, int K, int (&m)[N]) {
-    const float gsc = __fdiv_rn(static_cast<float>(K), l1);
-    if (!(l1 > 0.0f) || isinf(gsc)) {  // no direction: (K, 0, ..., 0)
+__device__ __forceinline__ float pick(const float (&v)[N], int idx) {
+    float t[N];
 #pragma unroll
-        for (int i = 0; i < N; ++i) m[i] = 0;
-        m[0] = K;
-        return;
+    for (int i = 0; i < N; ++i) t[i] = v[i];
+#pragma unroll
+    for (int s = 1, bit = 0; s < N; s <<= 1, ++bit) {
+        const bool hi = (idx >> bit) & 1;
+#pragma unroll
+        for (int i = 0; i < N; i += 2 * s) t[i] = hi ? t[i + s] : t[i];
     }
-    float e[N], srt[N];
-    int sum = 0;
+    return t[0];
+}
+
+constexpr float kMagic = 8388608.0f;  // 2^23: a + 2^23 rounded down is 2^23 + floor(a) for 0 <= a < 2^23
+constexpr int kMagicBits = 0x4B000000;
+
+// Direction of one group (Sec. 2.5 / Algorithm 1 in the floor + greedy reading).
+//   a_i = |x_i| * (K / l1), f_i = floor(a_i), e_i = a_i - f_i, d = K - sum f_i.
+// The greedy loop "give one pulse to the largest residual, lowest index first among
+// equals, d times" touches every element at most once when 0 <= d <= N (after its pulse
+// an element's residual is negative, below every untouched one), so its result is: the d
+// elements with the largest (e_i, -i) get +1.  v = the d-th largest residual comes from a
+// sorting network; every e_i >= v gets a pulse, and when that hands out more than d (equal
+// residuals straddle the cut) the elements equal to v share what is left, lowest index
+// first.
+//
+// Out: mag[i] = 2^23 + |y_i| as a float (the integer sits in the low mantissa bits).
+// Returns false for a group without direction (l1 zero or not finite, or a scale that
+// overflows): the point is then (K, 0, ..., 0).
+template <int N>
+__device__ __forceinline__ bool quantize_direction(const float (&x)[N], float l1, int K, float (&mag)[N]) {
+    const float gsc = __fdiv_rn(static_cast<float>(K), l1);
+    if (!(l1 > 0.0f) || !(l1 <= 3.4028234e38f) || !(gsc <= 3.4028234e38f)) return false;
+    float srt[N];
+    float sumf = 0.0f;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
         const float av = __fmul_rn(fabsf(x[i]), gsc);
-        const float f = floorf(av);
-        m[i] = static_cast<int>(f);
-        e[i] = __fsub_rn(av, f);
-        srt[i] = e[i];
-        sum += m[i];
+        const float t = __fadd_rd(av, kMagic);
+        const float f = __fsub_rn(t, kMagic);  // floor(av), exact
+        srt[i] = __fsub_rn(av, f);
+        sumf = __fadd_rn(sumf, f);             // small integers: exact
     }
-    int d = K - sum;
-    d = max(0, min(d, N));  // finite input keeps d in [0, N]; the clamp is for NaN / Inf only
+    const int d = K - static_cast<int>(sumf);
+    if (d < 0 || d > N) return false;  // cannot happen for finite input; keeps the table walk in range
     sort_desc<N>(srt);
-    float v = 2.0f;  // above every residual: d == 0 adds nothing
-#pragma unroll
-    for (int i = 0; i < N; ++i)
-        if (i == d - 1) v = srt[i];
-    int above = 0;
-#pragma unroll
-    for (int i = 0; i < N; ++i) above += (e[i] > v) ? 1 : 0;
-    int ties = d - above;  // pulses for the elements equal to v
+    const float v = d > 0 ? pick<N>(srt, d - 1) : 2.0f;  // 2 is above every residual
+    float cnt = 0.0f;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        const bool eq = (e[i] == v) && (ties > 0);
-        ties -= eq ? 1 : 0;
-        m[i] += ((e[i] > v) || eq) ? 1 : 0;
+        const float av = __fmul_rn(fabsf(x[i]), gsc);
+        const float t = __fadd_rd(av, kMagic);
+        const float e = __fsub_rn(av, __fsub_rn(t, kMagic));
+        const float one = e >= v ? 1.0f : 0.0f;
+        mag[i] = __fadd_rn(t, one);
+        cnt = __fadd_rn(cnt, one);
     }
+    if (static_cast<int>(cnt) != d) {
+        // more residuals equal to v than pulses left for them: redo with the tie rule
+        int above = 0;
 #pragma unroll
-    for (int i = 0; i < N; ++i)
-        if (signbit(x[i])) m[i] = -m[i];
+        for (int i = 0; i < N; ++i) {
+            const float av = __fmul_rn(fabsf(x[i]), gsc);
+            const float t = __fadd_rd(av, kMagic);
+            above += __fsub_rn(av, __fsub_rn(t, kMagic)) > v ? 1 : 0;
+        }
+        int ties = d - above;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const float av = __fmul_rn(fabsf(x[i]), gsc);
+            const float t = __fadd_rd(av, kMagic);
+            const float e = __fsub_rn(av, __fsub_rn(t, kMagic));
+            const bool eq = (e == v) && (ties > 0);
+            ties -= eq ? 1 : 0;
+            mag[i] = __fadd_rn(t, ((e > v) || eq) ? 1.0f : 0.0f);
+        }
+    }
+    return true;
 }
 
-// Algorithm 2: c = sum over non-zero positions of
-//   N(n,k) + 2 sum_{j=1}^{|y_i|-1} N(n,k-j) + [y_i < 0] N(n,k-|y_i|),  n = N-1-i.
-template <int N, int W>
-__device__ __forceinline__ mp<W> enumerate(const int (&y)[N], int K, const uint32_t* __restrict__ tab) {
+// Algorithm 2 with the cumulative table of App. C.2.  With V(n,k) = sum_{j<=k} N(n,j) the
+// contribution of y_i (n = N-1-i dimensions after it, k pulses before it, k' = k - |y_i|
+// after it) is
+//     U(n,k) - 2 V(n,k')      for y_i > 0        U(n,k) = V(n,k) + V(n,k-1)
+//     U(n,k) - U(n,k')        for y_i <= 0       (zero when y_i = 0, as k' = k)
+// so every position costs two table reads, one add and one subtract, whatever |y_i| is.
+// All arithmetic is modulo 2^(32 W); the total is the code, which is below 2^(32 W).
+//   tabU, tab2V   shared addresses of the two tables, rows of `rowbytes` bytes, entry
+//                 (i, col + 1) at i * rowbytes + (col + 1) * EB
+//   mag[i]        2^23 + |y_i| as float bits; x[i] gives the sign
+template <int N, int W, int EB>
+__device__ __forceinline__ mp<W> enumerate_uv(const float (&mag)[N], const float (&x)[N], int K, uint32_t tabU,
+                                              uint32_t tab2V, int rowbytes) {
     mp<W> c;
     mp_zero(c);
-    int k = K;
-    const int rowstride = (K + 1) * W;
+    // kb = byte offset of column k in a row: (k + 1) * EB.  |y_i| * EB is taken from the float
+    // bits of mag[i], whose constant part is folded into `fold`.
+    uint32_t kb = (K + 1) * EB;
+    const uint32_t fold = static_cast<uint32_t>(kMagicBits) * EB;  // wraps; only differences are used
+    uint32_t rowU = tabU;
+    const uint32_t delta = tab2V - tabU;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        const int mag = abs(y[i]);
-        if (mag > 0) {
-            const uint32_t* row = tab + (N - 1 - i) * rowstride;
-            mp_add<W>(c, mp_load<W>(row + k * W));
-            for (int j = 1; j < mag; ++j) {
-                mp<W> t = mp_load<W>(row + (k - j) * W);
-                mp_dbl<W>(t);
-                mp_add<W>(c, t);
-            }
-            if (y[i] < 0) mp_add<W>(c, mp_load<W>(row + (k - mag) * W));
-            k -= mag;
-        }
+        const int mbits = __float_as_int(mag[i]);
+        const uint32_t kb2 = kb - (static_cast<uint32_t>(mbits) * EB - fold);
+        const bool nonpos = (mbits == kMagicBits) || (__float_as_int(x[i]) < 0);  // y_i <= 0
+        const mp<W> u = load_entry<W>(rowU + kb);
+        const mp<W> s = load_entry<W>(rowU + kb2 + (nonpos ? 0u : delta));
+        mp_add<W>(c, u);
+        mp<W> d;
+        mp_sub_borrow<W>(d, c, s);
+        c = d;
+        kb = kb2;
+        rowU += rowbytes;
     }
     return c;
 }
 
-template <int N, int W>
-__device__ __forceinline__ bool deenumerate_rt(mp<W> r, int K, const uint32_t* __restrict__ tab, int (&y)[N]) {
-    int k = K;
-    const int rowstride = (K + 1) * W;
+// The same sum from the single table V (for tables too large to stage twice):
+//     V(n,k) + V(n,k-1) - V(n,k') - V(n,k' - [y_i <= 0]).
+template <int N, int W, int EB>
+__device__ __forceinline__ mp<W> enumerate_v(const float (&mag)[N], const float (&x)[N], int K, uint32_t tabV,
+                                             int rowbytes) {
+    mp<W> c;
+    mp_zero(c);
+    uint32_t kb = (K + 1) * EB;
+    const uint32_t fold = static_cast<uint32_t>(kMagicBits) * EB;
+    uint32_t row = tabV;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        y[i] = 0;
-        if (k > 0) {
-            const uint32_t* row = tab + (N - 1 - i) * rowstride;
-            mp<W> t = mp_load<W>(row + k * W);
-            if (mp_sub_if_ge<W>(r, t)) {
-                int j = 1;
-                t = mp_load<W>(row + (k - 1) * W);
-                while (j < k) {
-                    mp<W> d = t;
-                    mp_dbl<W>(d);
-                    if (!mp_sub_if_ge<W>(r, d)) break;
-                    ++j;
-                    t = mp_load<W>(row + (k - j) * W);
-                }
-                const bool neg = mp_sub_if_ge<W>(r, t);
-                y[i] = neg ? -j : j;
-                k -= j;
-            }
-        }
+        const int mbits = __float_as_int(mag[i]);
+        const uint32_t kb2 = kb - (static_cast<uint32_t>(mbits) * EB - fold);
+        const bool nonpos = (mbits == kMagicBits) || (__float_as_int(x[i]) < 0);
+        mp_add<W>(c, load_entry<W>(row + kb));
+        mp_add<W>(c, load_entry<W>(row + kb - EB));
+        mp<W> d;
+        mp_sub_borrow<W>(d, c, load_entry<W>(row + kb2));
+        mp_sub_borrow<W>(c, d, load_entry<W>(row + kb2 - (nonpos ? static_cast<uint32_t>(EB) : 0u)));
+        kb = kb2;
+        row += rowbytes;
     }
-    return k == 0 && mp_is_zero<W>(r);
+    return c;
+}
+
+// Algorithm 2 as the walk of pvq_walk.cuh run forwards, on the decoder's table: from
+// (0, K), a pulse at the current position adds t (its first) or 2t (a further one) and
+// goes left, the end of a position adds t when y_i < 0 and goes down; t = N(N-1-i, col).
+// N + K steps of the same instructions for every thread.  Used by the fused kernel when
+// the cumulative tables do not fit in shared memory beside the decoder's.  y: the thread's
+// slots holding the signed point (one spare slot is read past the end).
+template <int N, int W, int EB, typename YT>
+__device__ __forceinline__ mp<W> enumerate_walk(const YT* y, uint32_t tab0, int rowlen, int K) {
+    mp<W> c;
+    mp_zero(c);
+    const int D = (rowlen + 1) * EB;
+    uint32_t p = tab0 + K * EB;
+    int yi = y[0];
+    int rem = abs(yi);
+    int v = 0;
+    const int S = N + K;
+#pragma unroll 2
+    for (int s = 0; s < S; ++s) {
+        const mp<W> t = load_entry<W>(p);
+        const bool more = rem > 0;
+        const bool add1 = more || (yi < 0);
+        const bool add2 = more && v > 0;
+        mp<W> a1, a2;
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+            a1.w[w] = add1 ? t.w[w] : 0u;
+            a2.w[w] = add2 ? t.w[w] : 0u;
+        }
+        mp_add<W>(c, a1);
+        mp_add<W>(c, a2);
+        if (more) {
+            rem -= 1;
+            v += 1;
+        } else {
+            ++y;
+            yi = *y;
+            rem = abs(yi);
+            v = 0;
+            p += D;
+        }
+        p -= EB;
+    }
+    return c;
 }
 
 template <int N>
@@ -169,22 +253,61 @@ __device__ __forceinline__ void load_group(const void* base, size_t elem_off, bo
     }
 }
 
-// Shared memory: [count table][ss per thread slot, padded rows][edges][scale-index words]
-template <int N, int W, bool FUSED>
-__global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ BatchArgs a, int ss_floats,
-                                                      int bf16) {
-    extern __shared__ __align__(16) uint32_t smem[];
+// Launch-time geometry of the encode kernels' shared memory (bytes from the start).
+struct EncodeSmem {
+    uint32_t enc_bytes;   // staged encoder table(s)
+    uint32_t walk_bytes;  // fused: staged walk tables
+    uint32_t ss_off, edges_off, levels_off, idx_off, wbuf_off;
+    int ss_floats;
+    int enum_mode;        // 2: U and 2V staged, 1: V only, 0: none (fused: the walk table serves)
+    int walk_phases;
+};
+
+// Shared memory: [encoder tables][walk tables (fused)][ss per thread slot, padded rows]
+//                [edges][levels (fused)][scale-index words][per-warp slots (fused)]
+template <int N, int W, bool FUSED, typename YT>
+__global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ BatchArgs a,
+                                                      const __grid_constant__ EncodeSmem sm, int bf16) {
+    extern __shared__ __align__(16) uint8_t smem[];
+    constexpr int TW = W <= 2 ? W : (W <= 4 ? 4 : 6);
+    constexpr int EB = TW * 4;
+    constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
     const int K = a.K;
     const int b = a.scale_bits;
     const int nedges = (1 << b) - 1;
-    const int tab_words = N * (K + 1) * W;
-    uint32_t* s_tab = smem;
-    float* s_ss = reinterpret_cast<float*>(smem + tab_words);                   // ss_floats
-    float* s_edges = s_ss + ss_floats;                                   // 256
-    float* s_levels = s_edges + 256;                                            // 256 (fused only)
-    uint32_t* s_idx = reinterpret_cast<uint32_t*>(s_levels + (FUSED ? 256 : 0));  // max_rpt * words per row
+    const TableLayout L = table_layout(N, K, W);
+    float* s_ss = reinterpret_cast<float*>(smem + sm.ss_off);
+    float* s_edges = reinterpret_cast<float*>(smem + sm.edges_off);
+    float* s_levels = reinterpret_cast<float*>(smem + sm.levels_off);
+    uint32_t* s_idx = reinterpret_cast<uint32_t*>(smem + sm.idx_off);
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int nwarps = blockDim.x >> 5;
 
-    for (int i = threadIdx.x; i < tab_words; i += blockDim.x) s_tab[i] = a.table[i];
+    {   // stage the tables
+        const uint8_t* blob = reinterpret_cast<const uint8_t*>(a.table);
+        const uint4* src = reinterpret_cast<const uint4*>(blob + (sm.enum_mode == 2 ? L.enc_off[0] : L.enc_off[2]));
+        uint4* dst = reinterpret_cast<uint4*>(smem);
+        for (uint32_t q = threadIdx.x; q < sm.enc_bytes / 16; q += blockDim.x) dst[q] = src[q];
+        if constexpr (FUSED) {
+            const uint4* wsrc = reinterpret_cast<const uint4*>(blob + L.walk_off[0]);
+            uint4* wdst = reinterpret_cast<uint4*>(smem + sm.enc_bytes);
+            for (uint32_t q = threadIdx.x; q < sm.walk_bytes / 16; q += blockDim.x) wdst[q] = wsrc[q];
+        }
+    }
+    const uint32_t tabA = shared_addr(smem);
+    const uint32_t tabB = tabA + ((L.enc_bytes + 127u) & ~127u);  // 2V, when two tables are staged
+    const int rowbytes = (K + 2) * EB;
+    WalkTables wt;
+    uint8_t* wbuf = nullptr;
+    float* wscale = nullptr;
+    YT* yslots = nullptr;
+    if constexpr (FUSED) {
+        wt = walk_tables(L, tabA + sm.enc_bytes, sm.walk_phases);
+        wbuf = smem + sm.wbuf_off + warp * (32 * YS + 128);
+        yslots = reinterpret_cast<YT*>(wbuf + lane * YS);
+        wscale = reinterpret_cast<float*>(wbuf + 32 * YS);
+    }
     const float* cur_edges = nullptr;
 
     for (unsigned tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
@@ -208,9 +331,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             for (int i = threadIdx.x; i < rpt * idx_words; i += blockDim.x) s_idx[i] = 0u;
         __syncthreads();
 
-        const int rl = threadIdx.x / G;       // row within the tile
-        const int g = threadIdx.x - rl * G;   // group within the row
-        const long long row = static_cast<long long>(tile - m.tile_begin) * rpt + rl;
+        const int rl = threadIdx.x / G;      // row within the tile
+        const int g = threadIdx.x - rl * G;  // group within the row
+        const long long row0 = static_cast<long long>(tile - m.tile_begin) * rpt;
+        const long long row = row0 + rl;
         const bool active = rl < rpt && row < m.rows;
 
         float x[N];
@@ -225,30 +349,63 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             for (int i = 0; i < N; ++i) t[i] = __fmul_rn(x[i], x[i]);
             ss = tree_sum<N>(t);
             s_ss[rl * gp + g] = ss;
+        } else {
+#pragma unroll
+            for (int i = 0; i < N; ++i) x[i] = 0.0f;
         }
         __syncthreads();
-        // row energy: balanced tree over the (zero padded) groups of each row
-        for (int s = 1; s < gp; s <<= 1) {
-            for (int i = threadIdx.x; i < rpt * gp; i += blockDim.x) {
-                const int gg = i & (gp - 1);
-                if ((gg & (2 * s - 1)) == 0) s_ss[i] = __fadd_rn(s_ss[i], s_ss[i + s]);
+        // row energy: balanced tree over the (zero padded) groups of each row, one warp per row
+        for (int r = warp; r < rpt; r += nwarps) {
+            float* rs = s_ss + r * gp;
+            for (int s = 1; s < gp; s <<= 1) {
+                for (int j = lane * 2 * s; j < gp; j += 64 * s) rs[j] = __fadd_rn(rs[j], rs[j + s]);
+                __syncwarp();
             }
-            __syncthreads();
         }
+
+        // direction and its index; nothing here needs the row norm
+        float mag[N];
+        const bool has_dir = quantize_direction<N>(x, l1, K, mag);
+        if (!has_dir) {  // (K, 0, ..., 0)
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+                mag[i] = kMagic;
+                x[i] = 0.0f;
+            }
+            mag[0] = __int_as_float(kMagicBits + K);
+        }
+        mp<W> c;
+        if (sm.enum_mode == 2) {
+            c = enumerate_uv<N, W, EB>(mag, x, K, tabA, tabB, rowbytes);
+        } else if (sm.enum_mode == 1) {
+            c = enumerate_v<N, W, EB>(mag, x, K, tabA, rowbytes);
+        } else {
+            if constexpr (FUSED) {
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+                    const int mi2 = __float_as_int(mag[i]) - kMagicBits;
+                    yslots[i] = static_cast<YT>(__float_as_int(x[i]) < 0 ? -mi2 : mi2);
+                }
+                c = enumerate_walk<N, W, EB, YT>(yslots, wt.tab0, wt.rowlen, K);
+            } else {
+                mp_zero(c);
+            }
+        }
+
+        __syncthreads();  // row energies are in s_ss[r * gp]
+        float rnorm = 0.0f;
+        int q = 0;
         if (active) {
             const float ss_row = s_ss[rl * gp];
-            const float rnorm = __fsqrt_rn(ss_row);
+            rnorm = __fsqrt_rn(ss_row);
             // Step 5: q = floor(CDF(u) 2^b) as the number of bin edges <= u
             const float u = ss_row > 0.0f ? __fdiv_rn(ss, ss_row) : 0.0f;
-            int q = 0;
             for (int step = 1 << (b - 1); step >= 1; step >>= 1)
                 if (s_edges[q + step - 1] <= u) q += step;
+        }
 
-            int y[N];
-            quantize_direction<N>(x, l1, K, y);
-            const mp<W> c = enumerate<N, W>(y, K, s_tab);
-
-            if constexpr (!FUSED) {
+        if constexpr (!FUSED) {
+            if (active) {
                 if (g == 0) m.row_norm[row] = rnorm;
                 uint32_t* cp = m.codes + (static_cast<size_t>(row) * G + g) * W;
 #pragma unroll
@@ -256,47 +413,33 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
                 const unsigned bit = static_cast<unsigned>(g) * b;
                 const unsigned sh = bit & 31u;
                 atomicOr(&s_idx[rl * idx_words + (bit >> 5)], static_cast<uint32_t>(q) << sh);
-                if (sh + b > 32u) atomicOr(&s_idx[rl * idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));
-            } else {
-                int yd[N];
-                const bool ok = deenumerate_rt<N, W>(c, K, s_tab, yd);
-                int ssy = 0;
-#pragma unroll
-                for (int i = 0; i < N; ++i) ssy += yd[i] * yd[i];
-                const float amp = __fmul_rn(rnorm, s_levels[q]);
-                float sc = __fdiv_rn(amp, __fsqrt_rn(static_cast<float>(ssy)));
-                if (!ok) sc = 0.0f;
-                uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.out) +
-                                                      static_cast<size_t>(row) * m.ld_out +
-                                                      static_cast<size_t>(g) * N);
-#pragma unroll
-                for (int v = 0; v < N / 8; ++v) {
-                    uint32_t p[4];
-#pragma unroll
-                    for (int e2 = 0; e2 < 4; ++e2) {
-                        const float lo = __fmul_rn(static_cast<float>(yd[v * 8 + 2 * e2]), sc);
-                        const float hi = __fmul_rn(static_cast<float>(yd[v * 8 + 2 * e2 + 1]), sc);
-                        p[e2] = pack_bf16x2(lo, hi);
-                    }
-                    dst[v] = make_uint4(p[0], p[1], p[2], p[3]);
-                }
+                if (sh + b > 32u)
+                    atomicOr(&s_idx[rl * idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));
             }
-        }
-        if constexpr (!FUSED) {
             __syncthreads();
             for (int i = threadIdx.x; i < rpt * idx_words; i += blockDim.x) {
                 const int r2 = i / idx_words;
-                const long long row2 = static_cast<long long>(tile - m.tile_begin) * rpt + r2;
+                const long long row2 = row0 + r2;
                 if (row2 < m.rows)
                     reinterpret_cast<uint32_t*>(m.scale_idx + static_cast<size_t>(row2) * m.sstride)[i - r2 * idx_words] =
                         s_idx[i];
             }
+        } else {
+            // decode the code just made: walk, then scale and store the warp's 32 groups.
+            // Threads t .. t+31 of a warp hold consecutive groups of the tile's rows.
+            const float amp = active ? __fmul_rn(rnorm, s_levels[q]) : 0.0f;
+            if (!active) mp_zero(c);
+            walk_code<N, W, YT>(c, wt, K, yslots);
+            const long long g0 = row0 * G + (threadIdx.x & ~31);
+            const long long gend = (m.rows < row0 + rpt ? m.rows : row0 + rpt) * G;
+            emit_tile<N, YT>(m, wbuf, wscale, lane, amp, g0, gend);
         }
     }
 }
 
-template <int N, int W, bool FUSED>
+template <int N, int W, bool FUSED, typename YT>
 static int launch_encode_t(BatchArgs& a, int dtype, cudaStream_t stream) {
+    constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
     // Block size: a multiple of 32 that wastes the fewest thread slots over the batch.
     int best_threads = 0;
     long long best_cost = -1;
@@ -337,31 +480,70 @@ static int launch_encode_t(BatchArgs& a, int dtype, cudaStream_t stream) {
         ss_floats = std::max(ss_floats, a.m[i].rows_per_tile * gp);
     }
     a.total_tiles = tiles;
-    const size_t smem = (static_cast<size_t>(N) * (a.K + 1) * W + ss_floats + 256 + (FUSED ? 256 : 0) +
-                         max_idx_words) * 4u;
-    if (smem > 200 * 1024) return PVQ_ERR_UNSUPPORTED;
-    auto kern = encode_kernel<N, W, FUSED>;
+
+    int dev = 0, sms = 0, smem_max = 0;
     cudaError_t e;
-    if (smem > 48 * 1024) {
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        if (e != cudaSuccess) return set_cuda_error(e);
-    }
-    int dev = 0, sms = 0, per_sm = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return set_cuda_error(e);
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
         return set_cuda_error(e);
+    if ((e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+        return set_cuda_error(e);
+
+    const TableLayout L = table_layout(N, a.K, W);
+    const size_t small = (static_cast<size_t>(ss_floats) + 256 + (FUSED ? 256 : 0) + max_idx_words) * 4u + 64u;
+    const size_t wbufs = FUSED ? static_cast<size_t>(threads / 32) * (32 * YS + 128) : 0;
+    const size_t enc_one = (L.enc_bytes + 127u) & ~size_t(127);
+    EncodeSmem sm;
+    sm.walk_bytes = 0;
+    sm.walk_phases = 0;
+    size_t walk = 0;
+    const size_t cap = static_cast<size_t>(smem_max);
+    if (FUSED) {  // the widest walk table has to fit; then as many encoder tables as still do
+        sm.enum_mode = -1;
+        for (int mode = 2; mode >= 0 && sm.enum_mode < 0; --mode) {
+            const size_t fixed = mode * enc_one + small + wbufs;
+            if (fixed >= cap) continue;
+            const int ph = walk_phases_that_fit(L, cap - fixed);
+            if (ph == 0) continue;
+            sm.enum_mode = mode;
+            sm.walk_phases = ph;
+        }
+        if (sm.enum_mode < 0) return PVQ_ERR_UNSUPPORTED;
+        walk = (walk_tables_bytes(L, sm.walk_phases) + 15u) & ~size_t(15);
+        sm.walk_bytes = static_cast<uint32_t>(walk);
+    } else {
+        sm.enum_mode = 2 * enc_one + small <= cap ? 2 : 1;
+        if (sm.enum_mode == 1 && enc_one + small > cap) return PVQ_ERR_UNSUPPORTED;
+    }
+    sm.enc_bytes = static_cast<uint32_t>(sm.enum_mode * enc_one);
+    sm.ss_floats = ss_floats;
+    sm.ss_off = static_cast<uint32_t>(sm.enc_bytes + walk);
+    sm.edges_off = sm.ss_off + ss_floats * 4u;
+    sm.levels_off = sm.edges_off + 256u * 4u;
+    sm.idx_off = sm.levels_off + (FUSED ? 256u * 4u : 0u);
+    sm.wbuf_off = (sm.idx_off + max_idx_words * 4u + 15u) & ~15u;
+    const size_t smem = sm.wbuf_off + wbufs;
+    if (smem > static_cast<size_t>(smem_max)) return PVQ_ERR_UNSUPPORTED;
+
+    auto kern = encode_kernel<N, W, FUSED, YT>;
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))) !=
+        cudaSuccess)
+        return set_cuda_error(e);
+    int per_sm = 0;
     if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem)) != cudaSuccess)
         return set_cuda_error(e);
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
     const unsigned grid = std::min<unsigned>(tiles, static_cast<unsigned>(sms * per_sm));
-    kern<<<grid, threads, smem, stream>>>(a, ss_floats, dtype == PVQ_DTYPE_BF16 ? 1 : 0);
+    kern<<<grid, threads, smem, stream>>>(a, sm, dtype == PVQ_DTYPE_BF16 ? 1 : 0);
     e = cudaGetLastError();
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 
 template <int N, int W>
 static int launch_encode_nw(BatchArgs& a, int dtype, bool fused, cudaStream_t s) {
-    return fused ? launch_encode_t<N, W, true>(a, dtype, s) : launch_encode_t<N, W, false>(a, dtype, s);
+    if (!fused) return launch_encode_t<N, W, false, int8_t>(a, dtype, s);
+    if (a.K <= 127) return launch_encode_t<N, W, true, int8_t>(a, dtype, s);
+    return launch_encode_t<N, W, true, int16_t>(a, dtype, s);
 }
 
 }  // namespace pvq

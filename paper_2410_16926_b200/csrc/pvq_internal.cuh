@@ -56,12 +56,21 @@ struct BatchArgs {
 // rowlen is K+1 rounded up to an even number: consecutive positions on a diagonal of the
 // table, (i, col) and (i+1, col+1), are then an odd number of entries apart, so threads that
 // sit on neighbouring diagonals' cells read different shared-memory banks.
+//
+//   enc[0..2]   for the encoder, rows by position i, K+2 entries of `top_words` words each,
+//               entry (i, col+1) for col = -1..K, with V(n,k) = sum_{j<=k} N(n,j), V(n,-1) = 0
+//               (App. C.2) and n = N-1-i, all modulo 2^(32 W):
+//                 enc[0]  U(n,col) = V(n,col) + V(n,col-1)
+//                 enc[1]  2 V(n,col)
+//                 enc[2]  V(n,col)
 struct TableLayout {
     int rowlen;
     int top_words;
     uint32_t bound_off;
     uint32_t walk_off[3];
     uint32_t walk_bytes[3];
+    uint32_t enc_off[3];
+    uint32_t enc_bytes;  // of each of the three
     uint32_t total;
 };
 
@@ -71,7 +80,8 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
         L.rowlen = 0;
         L.top_words = 0;
         L.bound_off = 0;
-        for (int p = 0; p < 3; ++p) L.walk_off[p] = L.walk_bytes[p] = 0;
+        for (int p = 0; p < 3; ++p) L.walk_off[p] = L.walk_bytes[p] = L.enc_off[p] = 0;
+        L.enc_bytes = 0;
         L.total = static_cast<uint32_t>(N) * (K + 1) * W * 4u;
         return L;
     }
@@ -87,6 +97,11 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
         L.walk_off[p] = off;
         L.walk_bytes[p] = entries * words[p] * 4u;
         off += (L.walk_bytes[p] + 127u) & ~127u;
+    }
+    L.enc_bytes = static_cast<uint32_t>(N) * (K + 2) * L.top_words * 4u;
+    for (int p = 0; p < 3; ++p) {
+        L.enc_off[p] = off;
+        off += (L.enc_bytes + 127u) & ~127u;
     }
     L.total = off;
     return L;

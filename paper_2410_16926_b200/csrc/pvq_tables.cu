@@ -102,6 +102,42 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
             blob[L.walk_off[2] / 4 + e] = hi ? 0xffffffffu : v[0];
         }
     }
+    // encoder tables: one thread per position runs the prefix sum V(n,k) = V(n,k-1) + N(n,k)
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) {
+        const uint32_t* row = blob + static_cast<size_t>(N - 1 - i) * KP * W;
+        const int TW = L.top_words;
+        uint32_t* eu = blob + L.enc_off[0] / 4 + static_cast<size_t>(i) * (K + 2) * TW;
+        uint32_t* e2 = blob + L.enc_off[1] / 4 + static_cast<size_t>(i) * (K + 2) * TW;
+        uint32_t* ev = blob + L.enc_off[2] / 4 + static_cast<size_t>(i) * (K + 2) * TW;
+        uint32_t v[W], vprev[W];
+#pragma unroll
+        for (int w = 0; w < W; ++w) v[w] = vprev[w] = 0u;
+        for (int c = -1; c <= K; ++c) {
+            if (c >= 0) {
+#pragma unroll
+                for (int w = 0; w < W; ++w) vprev[w] = v[w];
+                unsigned long long carry = 0;
+#pragma unroll
+                for (int w = 0; w < W; ++w) {
+                    const unsigned long long sum = static_cast<unsigned long long>(v[w]) + row[c * W + w] + carry;
+                    v[w] = static_cast<uint32_t>(sum);
+                    carry = sum >> 32;
+                }
+            }
+            unsigned long long cu = 0, c2 = 0;
+            for (int w = 0; w < TW; ++w) {
+                const uint32_t a = w < W ? v[w < W ? w : 0] : 0u, bprev = w < W ? vprev[w < W ? w : 0] : 0u;
+                const unsigned long long su = static_cast<unsigned long long>(a) + bprev + cu;
+                const unsigned long long s2 = static_cast<unsigned long long>(a) + a + c2;
+                cu = su >> 32;
+                c2 = s2 >> 32;
+                const bool in = w < W;  // words beyond W stay zero: the sums are kept modulo 2^(32 W)
+                eu[(c + 1) * TW + w] = in ? static_cast<uint32_t>(su) : 0u;
+                e2[(c + 1) * TW + w] = in ? static_cast<uint32_t>(s2) : 0u;
+                ev[(c + 1) * TW + w] = a;
+            }
+        }
+    }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         // N(N,K) = N(N-1,K) + 2 sum_{j=1..K} N(N-1,K-j)   (every point of P(N,K) by its first
         // coordinate: 0, or +-j with K-j pulses left for the other N-1)
