@@ -12,27 +12,51 @@
 
 namespace pvq {
 
-// ---- descending sorting network (Batcher odd-even merge sort), in registers ----
+// ---- descending sorting network (Batcher's odd-even merge sort), in registers ----
+// Written as template recursion so that every index is a compile-time constant: a loop
+// nest that the compiler leaves partly rolled would put the array in local memory.
+template <int N, int I, int J>
+__device__ __forceinline__ void cmp_exchange(float (&v)[N]) {
+    const float hi = fmaxf(v[I], v[J]);
+    const float lo = fminf(v[I], v[J]);
+    v[I] = hi;
+    v[J] = lo;
+}
+
+// compare-exchange (I, I+R), (I+M, I+M+R), ... while I+R < END
+template <int N, int I, int R, int M, int END>
+__device__ __forceinline__ void cmp_exchange_row(float (&v)[N]) {
+    if constexpr (I + R < END) {
+        cmp_exchange<N, I, I + R>(v);
+        cmp_exchange_row<N, I + M, R, M, END>(v);
+    }
+}
+
+// merges the two sorted halves of the LEN elements LO, LO+R, LO+2R, ...
+template <int N, int LO, int LEN, int R>
+__device__ __forceinline__ void oddeven_merge(float (&v)[N]) {
+    constexpr int M = R * 2;
+    if constexpr (M < LEN) {
+        oddeven_merge<N, LO, LEN, M>(v);
+        oddeven_merge<N, LO + R, LEN, M>(v);
+        cmp_exchange_row<N, LO + R, R, M, LO + LEN>(v);
+    } else {
+        cmp_exchange<N, LO, LO + R>(v);
+    }
+}
+
+template <int N, int LO, int LEN>
+__device__ __forceinline__ void oddeven_sort(float (&v)[N]) {
+    if constexpr (LEN > 1) {
+        oddeven_sort<N, LO, LEN / 2>(v);
+        oddeven_sort<N, LO + LEN / 2, LEN / 2>(v);
+        oddeven_merge<N, LO, LEN, 1>(v);
+    }
+}
+
 template <int N>
 __device__ __forceinline__ void sort_desc(float (&v)[N]) {
-#pragma unroll
-    for (int p = 1; p < N; p <<= 1) {
-#pragma unroll
-        for (int k = p; k >= 1; k >>= 1) {
-#pragma unroll
-            for (int j = k % p; j + k < N; j += 2 * k) {
-#pragma unroll
-                for (int i = 0; i < k; ++i) {
-                    if (i + j + k < N && (i + j) / (2 * p) == (i + j + k) / (2 * p)) {
-                        const float hi = fmaxf(v[i + j], v[i + j + k]);
-                        const float lo = fminf(v[i + j], v[i + j + k]);
-                        v[i + j] = hi;
-                        v[i + j + k] = lo;
-                    }
-                }
-            }
-        }
-    }
+    oddeven_sort<N, 0, N>(v);
 }
 
 // v[idx] for a run-time idx in [0, N): a binary tree of selects on the bits of idx.
@@ -42,12 +66,29 @@ __device__ __forceinline__ float pick(const float (&v)[N], int idx) {
 #pragma unroll
     for (int i = 0; i < N; ++i) t[i] = v[i];
 #pragma unroll
-    for (int s = 1, bit = 0; s < N; s <<= 1, ++bit) {
+    for (int bit = 0; (1 << bit) < N; ++bit) {
+        const int s = 1 << bit;
         const bool hi = (idx >> bit) & 1;
 #pragma unroll
         for (int i = 0; i < N; i += 2 * s) t[i] = hi ? t[i + s] : t[i];
     }
     return t[0];
+}
+
+// |a| with the sign bit of s
+__device__ __forceinline__ float with_sign_of(float a, float s) {
+    return __int_as_float(__float_as_int(a) | (__float_as_int(s) & static_cast<int>(0x80000000u)));
+}
+
+// Element i of a group held as it sits in memory: N/2 words of two bf16 each, or N fp32 words.
+// Widening bf16 is exact.  A group stays in this form for the whole kernel (half the
+// registers of N floats for bf16) and its elements are widened where they are used.
+template <int N, bool BF16>
+__device__ __forceinline__ float raw_value(const uint32_t (&raw)[BF16 ? N / 2 : N], int i) {
+    if constexpr (BF16)
+        return __uint_as_float((i & 1) ? (raw[i / 2] & 0xffff0000u) : (raw[i / 2] << 16));
+    else
+        return __uint_as_float(raw[i]);
 }
 
 constexpr float kMagic = 8388608.0f;  // 2^23: a + 2^23 rounded down is 2^23 + floor(a) for 0 <= a < 2^23
@@ -60,58 +101,61 @@ constexpr int kMagicBits = 0x4B000000;
 // an element's residual is negative, below every untouched one), so its result is: the d
 // elements with the largest (e_i, -i) get +1.  v = the d-th largest residual comes from a
 // sorting network; every e_i >= v gets a pulse, and when that hands out more than d (equal
-// residuals straddle the cut) the elements equal to v share what is left, lowest index
-// first.
+// residuals straddle the cut) the elements equal to v with the highest indices give theirs
+// back.
 //
-// Out: mag[i] = 2^23 + |y_i| as a float (the integer sits in the low mantissa bits).
-// Returns false for a group without direction (l1 zero or not finite, or a scale that
-// overflows): the point is then (K, 0, ..., 0).
-template <int N>
-__device__ __forceinline__ bool quantize_direction(const float (&x)[N], float l1, int K, float (&mag)[N]) {
+// Out: mag[i] = 2^23 + |y_i| as a float (the integer sits in the low mantissa bits) with the
+// sign bit of x_i.  Returns false for a group without direction (l1 zero or not finite, or
+// a scale that overflows): the point is then (K, 0, ..., 0).
+template <int N, bool BF16>
+__device__ __forceinline__ bool quantize_direction(const uint32_t (&raw)[BF16 ? N / 2 : N], float l1, int K,
+                                                   float (&mag)[N]) {
     const float gsc = __fdiv_rn(static_cast<float>(K), l1);
     if (!(l1 > 0.0f) || !(l1 <= 3.4028234e38f) || !(gsc <= 3.4028234e38f)) return false;
     float srt[N];
     float sumf = 0.0f;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        const float av = __fmul_rn(fabsf(x[i]), gsc);
+        const float av = __fmul_rn(fabsf(raw_value<N, BF16>(raw, i)), gsc);
         const float t = __fadd_rd(av, kMagic);
         const float f = __fsub_rn(t, kMagic);  // floor(av), exact
         srt[i] = __fsub_rn(av, f);
         sumf = __fadd_rn(sumf, f);             // small integers: exact
     }
     const int d = K - static_cast<int>(sumf);
-    if (d < 0 || d > N) return false;  // cannot happen for finite input; keeps the table walk in range
+    if (d < 0 || d > N) return false;  // cannot happen for finite input; keeps the table reads in range
     sort_desc<N>(srt);
     const float v = d > 0 ? pick<N>(srt, d - 1) : 2.0f;  // 2 is above every residual
+    // The residuals are computed again rather than kept: N more registers through the sort
+    // cost more than the arithmetic.  (The empty asm hides from the compiler that gsc2 == gsc
+    // and, by naming v, keeps this second pass from being scheduled into the sort.)
+    float gsc2 = gsc;
+    asm volatile("" : "+f"(gsc2) : "f"(v));
     float cnt = 0.0f;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-        const float av = __fmul_rn(fabsf(x[i]), gsc);
+        const float xi = raw_value<N, BF16>(raw, i);
+        const float av = __fmul_rn(fabsf(xi), gsc2);
         const float t = __fadd_rd(av, kMagic);
         const float e = __fsub_rn(av, __fsub_rn(t, kMagic));
         const float one = e >= v ? 1.0f : 0.0f;
-        mag[i] = __fadd_rn(t, one);
+        mag[i] = with_sign_of(__fadd_rn(t, one), xi);
         cnt = __fadd_rn(cnt, one);
     }
-    if (static_cast<int>(cnt) != d) {
-        // more residuals equal to v than pulses left for them: redo with the tie rule
-        int above = 0;
+    int excess = static_cast<int>(cnt) - d;
+    if (excess > 0) {
+        // Residuals equal to v straddle the cut: of the elements equal to v the ones with the
+        // highest indices give their pulse back (lowest index first among equals).
+        float gsc3 = gsc;
+        asm volatile("" : "+f"(gsc3) : "r"(excess));
 #pragma unroll
-        for (int i = 0; i < N; ++i) {
-            const float av = __fmul_rn(fabsf(x[i]), gsc);
-            const float t = __fadd_rd(av, kMagic);
-            above += __fsub_rn(av, __fsub_rn(t, kMagic)) > v ? 1 : 0;
-        }
-        int ties = d - above;
-#pragma unroll
-        for (int i = 0; i < N; ++i) {
-            const float av = __fmul_rn(fabsf(x[i]), gsc);
+        for (int i = N - 1; i >= 0; --i) {
+            const float av = __fmul_rn(fabsf(raw_value<N, BF16>(raw, i)), gsc3);
             const float t = __fadd_rd(av, kMagic);
             const float e = __fsub_rn(av, __fsub_rn(t, kMagic));
-            const bool eq = (e == v) && (ties > 0);
-            ties -= eq ? 1 : 0;
-            mag[i] = __fadd_rn(t, ((e > v) || eq) ? 1.0f : 0.0f);
+            const bool drop = (e == v) && (excess > 0);
+            excess -= drop ? 1 : 0;
+            mag[i] = __int_as_float(__float_as_int(mag[i]) - (drop ? 1 : 0));  // |y_i| sits in the low bits
         }
     }
     return true;
@@ -126,10 +170,12 @@ __device__ __forceinline__ bool quantize_direction(const float (&x)[N], float l1
 // All arithmetic is modulo 2^(32 W); the total is the code, which is below 2^(32 W).
 //   tabU, tab2V   shared addresses of the two tables, rows of `rowbytes` bytes, entry
 //                 (i, col + 1) at i * rowbytes + (col + 1) * EB
-//   mag[i]        2^23 + |y_i| as float bits; x[i] gives the sign
+//   mag[i]        2^23 + |y_i| as float bits, sign bit = sign of y_i (also set for "-0").
+//                 As a signed integer it is <= the bits of 2^23 exactly when y_i <= 0, and
+//                 times EB (a multiple of 4) the sign bit drops out of the 32-bit product.
 template <int N, int W, int EB>
-__device__ __forceinline__ mp<W> enumerate_uv(const float (&mag)[N], const float (&x)[N], int K, uint32_t tabU,
-                                              uint32_t tab2V, int rowbytes) {
+__device__ __forceinline__ mp<W> enumerate_uv(const float (&mag)[N], int K, uint32_t tabU, uint32_t tab2V,
+                                              int rowbytes) {
     mp<W> c;
     mp_zero(c);
     // kb = byte offset of column k in a row: (k + 1) * EB.  |y_i| * EB is taken from the float
@@ -142,7 +188,7 @@ __device__ __forceinline__ mp<W> enumerate_uv(const float (&mag)[N], const float
     for (int i = 0; i < N; ++i) {
         const int mbits = __float_as_int(mag[i]);
         const uint32_t kb2 = kb - (static_cast<uint32_t>(mbits) * EB - fold);
-        const bool nonpos = (mbits == kMagicBits) || (__float_as_int(x[i]) < 0);  // y_i <= 0
+        const bool nonpos = mbits <= kMagicBits;  // y_i <= 0
         const mp<W> u = load_entry<W>(rowU + kb);
         const mp<W> s = load_entry<W>(rowU + kb2 + (nonpos ? 0u : delta));
         mp_add<W>(c, u);
@@ -158,8 +204,7 @@ __device__ __forceinline__ mp<W> enumerate_uv(const float (&mag)[N], const float
 // The same sum from the single table V (for tables too large to stage twice):
 //     V(n,k) + V(n,k-1) - V(n,k') - V(n,k' - [y_i <= 0]).
 template <int N, int W, int EB>
-__device__ __forceinline__ mp<W> enumerate_v(const float (&mag)[N], const float (&x)[N], int K, uint32_t tabV,
-                                             int rowbytes) {
+__device__ __forceinline__ mp<W> enumerate_v(const float (&mag)[N], int K, uint32_t tabV, int rowbytes) {
     mp<W> c;
     mp_zero(c);
     uint32_t kb = (K + 1) * EB;
@@ -169,7 +214,7 @@ __device__ __forceinline__ mp<W> enumerate_v(const float (&mag)[N], const float 
     for (int i = 0; i < N; ++i) {
         const int mbits = __float_as_int(mag[i]);
         const uint32_t kb2 = kb - (static_cast<uint32_t>(mbits) * EB - fold);
-        const bool nonpos = (mbits == kMagicBits) || (__float_as_int(x[i]) < 0);
+        const bool nonpos = mbits <= kMagicBits;
         mp_add<W>(c, load_entry<W>(row + kb));
         mp_add<W>(c, load_entry<W>(row + kb - EB));
         mp<W> d;
@@ -226,30 +271,18 @@ __device__ __forceinline__ mp<W> enumerate_walk(const YT* y, uint32_t tab0, int 
     return c;
 }
 
-template <int N>
-__device__ __forceinline__ void load_group(const void* base, size_t elem_off, bool bf16, float (&x)[N]) {
-    if (bf16) {
-        const uint4* p = reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(base) + elem_off);
+// The N values of one group as they sit in memory, fetched with 16-byte loads.
+template <int N, bool BF16>
+__device__ __forceinline__ void load_raw(const void* base, size_t elem_off, uint32_t (&r)[BF16 ? N / 2 : N]) {
+    constexpr int RW = BF16 ? N / 2 : N;
+    const uint4* p = reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(base) + elem_off * (BF16 ? 2 : 4));
 #pragma unroll
-        for (int v = 0; v < N / 8; ++v) {
-            const uint4 q = p[v];
-            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                x[v * 8 + 2 * e] = __uint_as_float(w[e] << 16);
-                x[v * 8 + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
-            }
-        }
-    } else {
-        const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(base) + elem_off);
-#pragma unroll
-        for (int v = 0; v < N / 4; ++v) {
-            const float4 q = p[v];
-            x[v * 4] = q.x;
-            x[v * 4 + 1] = q.y;
-            x[v * 4 + 2] = q.z;
-            x[v * 4 + 3] = q.w;
-        }
+    for (int v = 0; v < RW / 4; ++v) {
+        const uint4 q = p[v];
+        r[4 * v] = q.x;
+        r[4 * v + 1] = q.y;
+        r[4 * v + 2] = q.z;
+        r[4 * v + 3] = q.w;
     }
 }
 
@@ -258,28 +291,57 @@ struct EncodeSmem {
     uint32_t enc_bytes;   // staged encoder table(s)
     uint32_t walk_bytes;  // fused: staged walk tables
     uint32_t ss_off, edges_off, levels_off, idx_off, wbuf_off;
-    int ss_floats;
+    int ss_floats;        // per buffer (there are two)
+    int idx_words;        // per buffer (there are two)
     int enum_mode;        // 2: U and 2V staged, 1: V only, 0: none (fused: the walk table serves)
     int walk_phases;
 };
 
-// Shared memory: [encoder tables][walk tables (fused)][ss per thread slot, padded rows]
-//                [edges][levels (fused)][scale-index words][per-warp slots (fused)]
-template <int N, int W, bool FUSED, typename YT>
+// Where a thread works in a tile.
+struct TileLoc {
+    int mi;          // matrix
+    int G, rpt, gp;  // groups per row, rows per tile, G rounded up to a power of two
+    int rl, g;       // row within the tile, group within the row
+    long long row0;  // first row of the tile
+    bool active;     // this thread has a group
+};
+
+__device__ __forceinline__ TileLoc locate(const BatchArgs& a, unsigned tile) {
+    TileLoc t;
+    t.mi = find_matrix(a, tile);
+    const MatrixArgs& m = a.m[t.mi];
+    t.G = m.G;
+    t.rpt = m.rows_per_tile;
+    t.gp = 1;
+    while (t.gp < t.G) t.gp <<= 1;
+    t.rl = threadIdx.x / t.G;
+    t.g = threadIdx.x - t.rl * t.G;
+    t.row0 = static_cast<long long>(tile - m.tile_begin) * t.rpt;
+    t.active = t.rl < t.rpt && t.row0 + t.rl < m.rows;
+    return t;
+}
+
+// Shared memory: [encoder tables][walk tables (fused)][2 x ss per thread slot, padded rows]
+//                [edges][levels (fused)][2 x scale-index words][per-warp slots (fused)]
+// The two ss / scale-index buffers alternate between consecutive tiles, which leaves three
+// block-wide barriers per tile (two in the fused kernel); the input of the next tile is
+// requested as soon as the registers that held this tile's input are free.
+template <int N, int W, bool FUSED, typename YT, bool BF16>
 __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ BatchArgs a,
-                                                      const __grid_constant__ EncodeSmem sm, int bf16) {
+                                                      const __grid_constant__ EncodeSmem sm) {
     extern __shared__ __align__(16) uint8_t smem[];
     constexpr int TW = W <= 2 ? W : (W <= 4 ? 4 : 6);
     constexpr int EB = TW * 4;
     constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
+    constexpr int RW = BF16 ? N / 2 : N;
     const int K = a.K;
     const int b = a.scale_bits;
     const int nedges = (1 << b) - 1;
     const TableLayout L = table_layout(N, K, W);
-    float* s_ss = reinterpret_cast<float*>(smem + sm.ss_off);
+    float* s_ss2 = reinterpret_cast<float*>(smem + sm.ss_off);
     float* s_edges = reinterpret_cast<float*>(smem + sm.edges_off);
     float* s_levels = reinterpret_cast<float*>(smem + sm.levels_off);
-    uint32_t* s_idx = reinterpret_cast<uint32_t*>(smem + sm.idx_off);
+    uint32_t* s_idx2 = reinterpret_cast<uint32_t*>(smem + sm.idx_off);
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
@@ -294,6 +356,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             uint4* wdst = reinterpret_cast<uint4*>(smem + sm.enc_bytes);
             for (uint32_t q = threadIdx.x; q < sm.walk_bytes / 16; q += blockDim.x) wdst[q] = wsrc[q];
         }
+        for (int i = threadIdx.x; i < 2 * sm.idx_words; i += blockDim.x) s_idx2[i] = 0u;
     }
     const uint32_t tabA = shared_addr(smem);
     const uint32_t tabB = tabA + ((L.enc_bytes + 127u) & ~127u);  // 2V, when two tables are staged
@@ -310,50 +373,58 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     }
     const float* cur_edges = nullptr;
 
-    for (unsigned tile = blockIdx.x; tile < a.total_tiles; tile += gridDim.x) {
-        const int mi = find_matrix(a, tile);
-        const MatrixArgs& m = a.m[mi];
-        const int G = m.G;
-        const int rpt = m.rows_per_tile;
-        int gp = 1;
-        while (gp < G) gp <<= 1;
-        const int idx_words = m.sstride >> 2;
+    unsigned tile = blockIdx.x;
+    if (tile >= a.total_tiles) return;
+    TileLoc loc = locate(a, tile);
+    uint32_t raw[RW];
+#pragma unroll
+    for (int i = 0; i < RW; ++i) raw[i] = 0u;
+    if (loc.active) {
+        const MatrixArgs& m0 = a.m[loc.mi];
+        load_raw<N, BF16>(m0.x, static_cast<size_t>(loc.row0 + loc.rl) * m0.ld + static_cast<size_t>(loc.g) * N, raw);
+    }
+    __syncthreads();  // tables staged, index words cleared
 
-        __syncthreads();  // previous tile is done with shared memory
+    for (int buf = 0;; buf ^= 1) {
+        const MatrixArgs& m = a.m[loc.mi];
+        const int G = loc.G, rpt = loc.rpt, gp = loc.gp, rl = loc.rl, g = loc.g;
+        const long long row0 = loc.row0;
+        const long long row = row0 + rl;
+        const bool active = loc.active;
+        const int idx_words = m.sstride >> 2;
+        float* s_ss = s_ss2 + buf * sm.ss_floats;
+        uint32_t* s_idx = s_idx2 + buf * sm.idx_words;
+
+        // group norms; an inactive thread holds zeros
+        float l1, ss;
+        {
+            float t[N];
+#pragma unroll
+            for (int i = 0; i < N; ++i) t[i] = fabsf(raw_value<N, BF16>(raw, i));
+            l1 = tree_sum<N>(t);
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+                const float xi = raw_value<N, BF16>(raw, i);
+                t[i] = __fmul_rn(xi, xi);
+            }
+            ss = tree_sum<N>(t);
+        }
+        if (active) {
+            s_ss[rl * gp + g] = ss;
+            if (g < gp - G) s_ss[rl * gp + G + g] = 0.0f;  // zero padding of the row's tree
+        }
+        __syncthreads();  // (1) group energies of this tile are in s_ss; nobody is in the previous tile
+
         if (cur_edges != m.edges) {  // uniform across the block
             for (int i = threadIdx.x; i < nedges; i += blockDim.x) s_edges[i] = m.edges[i];
             if constexpr (FUSED)
                 for (int i = threadIdx.x; i <= nedges; i += blockDim.x) s_levels[i] = m.levels[i];
             cur_edges = m.edges;
         }
-        for (int i = threadIdx.x; i < rpt * gp; i += blockDim.x) s_ss[i] = 0.0f;  // zero padding of the tree
-        if constexpr (!FUSED)
-            for (int i = threadIdx.x; i < rpt * idx_words; i += blockDim.x) s_idx[i] = 0u;
-        __syncthreads();
-
-        const int rl = threadIdx.x / G;      // row within the tile
-        const int g = threadIdx.x - rl * G;  // group within the row
-        const long long row0 = static_cast<long long>(tile - m.tile_begin) * rpt;
-        const long long row = row0 + rl;
-        const bool active = rl < rpt && row < m.rows;
-
-        float x[N];
-        float l1 = 0.0f, ss = 0.0f;
-        if (active) {
-            load_group<N>(m.x, static_cast<size_t>(row) * m.ld + static_cast<size_t>(g) * N, bf16 != 0, x);
-            float t[N];
-#pragma unroll
-            for (int i = 0; i < N; ++i) t[i] = fabsf(x[i]);
-            l1 = tree_sum<N>(t);
-#pragma unroll
-            for (int i = 0; i < N; ++i) t[i] = __fmul_rn(x[i], x[i]);
-            ss = tree_sum<N>(t);
-            s_ss[rl * gp + g] = ss;
-        } else {
-#pragma unroll
-            for (int i = 0; i < N; ++i) x[i] = 0.0f;
+        if constexpr (!FUSED) {  // the other buffer's index words, for the next tile
+            uint32_t* other = s_idx2 + (buf ^ 1) * sm.idx_words;
+            for (int i = threadIdx.x; i < sm.idx_words; i += blockDim.x) other[i] = 0u;
         }
-        __syncthreads();
         // row energy: balanced tree over the (zero padded) groups of each row, one warp per row
         for (int r = warp; r < rpt; r += nwarps) {
             float* rs = s_ss + r * gp;
@@ -363,28 +434,43 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             }
         }
 
-        // direction and its index; nothing here needs the row norm
+        // direction; nothing here needs the row norm.  mag[i] carries the sign of x_i.
         float mag[N];
-        const bool has_dir = quantize_direction<N>(x, l1, K, mag);
+        const bool has_dir = quantize_direction<N, BF16>(raw, l1, K, mag);
         if (!has_dir) {  // (K, 0, ..., 0)
 #pragma unroll
-            for (int i = 0; i < N; ++i) {
-                mag[i] = kMagic;
-                x[i] = 0.0f;
-            }
+            for (int i = 0; i < N; ++i) mag[i] = kMagic;
             mag[0] = __int_as_float(kMagicBits + K);
         }
+
+        // raw is dead: ask for the next tile's input now, it arrives while the index is computed
+        const unsigned next_tile = tile + gridDim.x;
+        const bool have_next = next_tile < a.total_tiles;
+        TileLoc nloc = loc;
+        if (have_next) {
+            nloc = locate(a, next_tile);
+            if (nloc.active) {
+                const MatrixArgs& mn = a.m[nloc.mi];
+                load_raw<N, BF16>(mn.x, static_cast<size_t>(nloc.row0 + nloc.rl) * mn.ld + static_cast<size_t>(nloc.g) * N,
+                                  raw);
+            } else {
+#pragma unroll
+                for (int i = 0; i < RW; ++i) raw[i] = 0u;
+            }
+        }
+
         mp<W> c;
         if (sm.enum_mode == 2) {
-            c = enumerate_uv<N, W, EB>(mag, x, K, tabA, tabB, rowbytes);
+            c = enumerate_uv<N, W, EB>(mag, K, tabA, tabB, rowbytes);
         } else if (sm.enum_mode == 1) {
-            c = enumerate_v<N, W, EB>(mag, x, K, tabA, rowbytes);
+            c = enumerate_v<N, W, EB>(mag, K, tabA, rowbytes);
         } else {
             if constexpr (FUSED) {
 #pragma unroll
                 for (int i = 0; i < N; ++i) {
-                    const int mi2 = __float_as_int(mag[i]) - kMagicBits;
-                    yslots[i] = static_cast<YT>(__float_as_int(x[i]) < 0 ? -mi2 : mi2);
+                    const int mb = __float_as_int(mag[i]);
+                    const int mi2 = (mb & 0x7fffffff) - kMagicBits;
+                    yslots[i] = static_cast<YT>(mb < 0 ? -mi2 : mi2);
                 }
                 c = enumerate_walk<N, W, EB, YT>(yslots, wt.tab0, wt.rowlen, K);
             } else {
@@ -392,7 +478,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             }
         }
 
-        __syncthreads();  // row energies are in s_ss[r * gp]
+        __syncthreads();  // (2) row energies are in s_ss[r * gp]
         float rnorm = 0.0f;
         int q = 0;
         if (active) {
@@ -416,7 +502,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
                 if (sh + b > 32u)
                     atomicOr(&s_idx[rl * idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));
             }
-            __syncthreads();
+            __syncthreads();  // (3) the tile's index words are complete
             for (int i = threadIdx.x; i < rpt * idx_words; i += blockDim.x) {
                 const int r2 = i / idx_words;
                 const long long row2 = row0 + r2;
@@ -434,11 +520,15 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             const long long gend = (m.rows < row0 + rpt ? m.rows : row0 + rpt) * G;
             emit_tile<N, YT>(m, wbuf, wscale, lane, amp, g0, gend);
         }
+
+        if (!have_next) break;
+        tile = next_tile;
+        loc = nloc;
     }
 }
 
-template <int N, int W, bool FUSED, typename YT>
-static int launch_encode_t(BatchArgs& a, int dtype, cudaStream_t stream) {
+template <int N, int W, bool FUSED, typename YT, bool BF16>
+static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
     // Block size: a multiple of 32 that wastes the fewest thread slots over the batch.
     int best_threads = 0;
@@ -490,7 +580,7 @@ static int launch_encode_t(BatchArgs& a, int dtype, cudaStream_t stream) {
         return set_cuda_error(e);
 
     const TableLayout L = table_layout(N, a.K, W);
-    const size_t small = (static_cast<size_t>(ss_floats) + 256 + (FUSED ? 256 : 0) + max_idx_words) * 4u + 64u;
+    const size_t small = (2 * static_cast<size_t>(ss_floats) + 256 + (FUSED ? 256 : 0) + 2 * max_idx_words) * 4u + 64u;
     const size_t wbufs = FUSED ? static_cast<size_t>(threads / 32) * (32 * YS + 128) : 0;
     const size_t enc_one = (L.enc_bytes + 127u) & ~size_t(127);
     EncodeSmem sm;
@@ -517,15 +607,16 @@ static int launch_encode_t(BatchArgs& a, int dtype, cudaStream_t stream) {
     }
     sm.enc_bytes = static_cast<uint32_t>(sm.enum_mode * enc_one);
     sm.ss_floats = ss_floats;
+    sm.idx_words = max_idx_words;
     sm.ss_off = static_cast<uint32_t>(sm.enc_bytes + walk);
-    sm.edges_off = sm.ss_off + ss_floats * 4u;
+    sm.edges_off = sm.ss_off + 2u * ss_floats * 4u;
     sm.levels_off = sm.edges_off + 256u * 4u;
     sm.idx_off = sm.levels_off + (FUSED ? 256u * 4u : 0u);
-    sm.wbuf_off = (sm.idx_off + max_idx_words * 4u + 15u) & ~15u;
+    sm.wbuf_off = (sm.idx_off + 2u * max_idx_words * 4u + 15u) & ~15u;
     const size_t smem = sm.wbuf_off + wbufs;
     if (smem > static_cast<size_t>(smem_max)) return PVQ_ERR_UNSUPPORTED;
 
-    auto kern = encode_kernel<N, W, FUSED, YT>;
+    auto kern = encode_kernel<N, W, FUSED, YT, BF16>;
     if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))) !=
         cudaSuccess)
         return set_cuda_error(e);
@@ -534,16 +625,22 @@ static int launch_encode_t(BatchArgs& a, int dtype, cudaStream_t stream) {
         return set_cuda_error(e);
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
     const unsigned grid = std::min<unsigned>(tiles, static_cast<unsigned>(sms * per_sm));
-    kern<<<grid, threads, smem, stream>>>(a, sm, dtype == PVQ_DTYPE_BF16 ? 1 : 0);
+    kern<<<grid, threads, smem, stream>>>(a, sm);
     e = cudaGetLastError();
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 
+template <int N, int W, bool BF16>
+static int launch_encode_nwb(BatchArgs& a, bool fused, cudaStream_t s) {
+    if (!fused) return launch_encode_t<N, W, false, int8_t, BF16>(a, s);
+    if (a.K <= 127) return launch_encode_t<N, W, true, int8_t, BF16>(a, s);
+    return launch_encode_t<N, W, true, int16_t, BF16>(a, s);
+}
+
 template <int N, int W>
 static int launch_encode_nw(BatchArgs& a, int dtype, bool fused, cudaStream_t s) {
-    if (!fused) return launch_encode_t<N, W, false, int8_t>(a, dtype, s);
-    if (a.K <= 127) return launch_encode_t<N, W, true, int8_t>(a, dtype, s);
-    return launch_encode_t<N, W, true, int16_t>(a, dtype, s);
+    return dtype == PVQ_DTYPE_BF16 ? launch_encode_nwb<N, W, true>(a, fused, s)
+                                   : launch_encode_nwb<N, W, false>(a, fused, s);
 }
 
 }  // namespace pvq
