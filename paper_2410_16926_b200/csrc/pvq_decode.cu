@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
         uint4* dst = reinterpret_cast<uint4*>(smem);
         for (uint32_t q = threadIdx.x; q < tab_bytes / 16; q += blockDim.x) dst[q] = src[q];
     }
-    const WalkTables wt = walk_tables(L, shared_addr(smem), a.walk_phases);
+    const WalkTables wt = walk_tables(L, shared_addr(smem), a.walk_phases, a);
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;

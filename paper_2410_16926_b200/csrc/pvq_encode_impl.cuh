@@ -366,7 +366,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     float* wscale = nullptr;
     YT* yslots = nullptr;
     if constexpr (FUSED) {
-        wt = walk_tables(L, tabA + sm.enc_bytes, sm.walk_phases);
+        wt = walk_tables(L, tabA + sm.enc_bytes, sm.walk_phases, a);
         wbuf = smem + sm.wbuf_off + warp * (32 * YS + 128);
         yslots = reinterpret_cast<YT*>(wbuf + lane * YS);
         wscale = reinterpret_cast<float*>(wbuf + 32 * YS);

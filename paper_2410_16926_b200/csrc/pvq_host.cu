@@ -248,6 +248,8 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
     a.scale_bits = scale_bits;
     a.table = d_table;
     a.status = d_status;
+    a.c_one = 1u;
+    a.c_minus_one = 0xffffffffu;
     for (int i = 0; i < count; ++i) {
         st = fill_matrix(descs[i], need, dtype, c, &a.m[i]);
         if (st != PVQ_OK) return st;

@@ -40,6 +40,10 @@ struct BatchArgs {
     const uint32_t* table;  // the blob written by pvq_build_count_table (see TableLayout)
     uint32_t* status;
     int walk_phases;        // decode: how many of the walk tables are staged in shared memory (1..3)
+    // The integers 1 and -1 as kernel arguments.  Multiply-adds by a factor the assembler cannot
+    // see through stay multiply-adds, which run on the FMA pipe; the walk uses them for plain
+    // moves, adds and subtracts to take load off the integer ALU pipe, its bottleneck.
+    uint32_t c_one, c_minus_one;
 };
 
 // Layout of the table blob.  Section 0 is the count table as the paper defines it,
@@ -49,9 +53,10 @@ struct BatchArgs {
 //   bound       N(N,K) as 8 words (codes are valid below it)
 //   walk[0]     rows by position i (row i holds N(N-1-i, .)), `rowlen` entries of
 //               `top_words` words each, entry (i, col) = N(N-1-i, col), zero padded
-//   walk[1]     same with 2-word entries, values that need more than 2 words replaced by
-//               2^64-1 (present when top_words > 2)
-//   walk[2]     same with 1-word entries saturated at 2^32-1 (present when top_words > 1)
+//   walk[1]     same with 2-word entries, values from 2^62 up replaced by 2^62 (present when
+//               top_words > 2)
+//   walk[2]     same with 1-word entries, values from 2^30 up replaced by 2^30 (present when
+//               top_words > 1)
 //
 // rowlen is K+1 rounded up to an even number: consecutive positions on a diagonal of the
 // table, (i, col) and (i+1, col+1), are then an odd number of entries apart, so threads that

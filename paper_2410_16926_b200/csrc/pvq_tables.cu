@@ -87,19 +87,22 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
             v[w] = pad ? 0xffffffffu : blob[(static_cast<size_t>(N - 1 - i) * KP + col) * W + w];
         uint32_t* top = blob + L.walk_off[0] / 4 + static_cast<size_t>(e) * L.top_words;
         for (int w = 0; w < L.top_words; ++w) top[w] = w < W ? v[w] : 0u;
-        if (L.walk_bytes[1]) {
+        if (L.walk_bytes[1]) {  // two-word copy: values from 2^62 up become 2^62
             uint32_t hi = 0;
 #pragma unroll
             for (int w = 2; w < W; ++w) hi |= v[w];
+            const uint32_t v1 = W > 1 ? v[W > 1 ? 1 : 0] : 0u;
+            const bool big = pad || hi != 0u || (v1 >> 30) != 0u;
             uint32_t* t2 = blob + L.walk_off[1] / 4 + static_cast<size_t>(e) * 2;
-            t2[0] = hi ? 0xffffffffu : v[0];
-            t2[1] = hi ? 0xffffffffu : (W > 1 ? v[W > 1 ? 1 : 0] : 0u);
+            t2[0] = big ? 0u : v[0];
+            t2[1] = big ? 0x40000000u : v1;
         }
-        if (L.walk_bytes[2]) {
+        if (L.walk_bytes[2]) {  // one-word copy: values from 2^30 up become 2^30
             uint32_t hi = 0;
 #pragma unroll
             for (int w = 1; w < W; ++w) hi |= v[w];
-            blob[L.walk_off[2] / 4 + e] = hi ? 0xffffffffu : v[0];
+            const bool big = pad || hi != 0u || (v[0] >> 30) != 0u;
+            blob[L.walk_off[2] / 4 + e] = big ? 0x40000000u : v[0];
         }
     }
     // encoder tables: one thread per position runs the prefix sum V(n,k) = V(n,k-1) + N(n,k)

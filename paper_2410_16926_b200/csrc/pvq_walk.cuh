@@ -17,9 +17,11 @@
 // data-dependent branch, and their table reads fall on neighbouring diagonal
 // cells, which the table layout puts in different banks.
 //
-// r only shrinks.  Once every thread of the warp has r below 2^63 (2^31) the warp
+// r only shrinks.  Once every thread of the warp has r below 2^62 (2^30) the warp
 // continues in a copy of the loop that works on two-word (one-word) integers
-// and reads a table of that width, whose larger entries are saturated.
+// and reads a table of that width, whose larger entries are replaced by 2^62 (2^30):
+// no r of that phase reaches them, and with two spare bits the sign of a difference
+// tells the comparison.
 #pragma once
 #include "mp_uint.cuh"
 #include "pvq_internal.cuh"
@@ -33,25 +35,26 @@ __device__ __forceinline__ uint32_t shared_addr(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-template <int PW>
+// Entry of PW words at shared address addr + OFF (OFF a compile-time byte offset).
+template <int PW, int OFF = 0>
 __device__ __forceinline__ mp<PW> load_entry(uint32_t addr) {
     mp<PW> t;
     if constexpr (PW == 1) {
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t.w[0]) : "r"(addr));
+        asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(t.w[0]) : "r"(addr), "n"(OFF));
     } else if constexpr (PW == 2) {
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(t.w[0]), "=r"(t.w[1]) : "r"(addr));
+        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(t.w[0]), "=r"(t.w[1]) : "r"(addr), "n"(OFF));
     } else if constexpr (PW <= 4) {  // 16-byte entries
         uint32_t v[4];
-        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+        asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4+%5];"
                      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
-                     : "r"(addr));
+                     : "r"(addr), "n"(OFF));
 #pragma unroll
         for (int w = 0; w < PW; ++w) t.w[w] = v[w];
     } else {  // 24-byte entries, 8-byte aligned
         uint32_t v[6];
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v[0]), "=r"(v[1]) : "r"(addr));
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+8];" : "=r"(v[2]), "=r"(v[3]) : "r"(addr));
-        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+16];" : "=r"(v[4]), "=r"(v[5]) : "r"(addr));
+        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v[0]), "=r"(v[1]) : "r"(addr), "n"(OFF));
+        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v[2]), "=r"(v[3]) : "r"(addr), "n"(OFF + 8));
+        asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v[4]), "=r"(v[5]) : "r"(addr), "n"(OFF + 16));
 #pragma unroll
         for (int w = 0; w < PW; ++w) t.w[w] = v[w];
     }
@@ -66,6 +69,22 @@ __device__ __forceinline__ void store_y(uint32_t addr, int val) {
         asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "r"(val) : "memory");
 }
 
+// d = a - b for the narrow phases (1 or 2 words), where the operands leave the two top bits
+// free: the sign bit of the top word of d then says whether a < b.
+template <int PW>
+__device__ __forceinline__ bool sub_negative(mp<PW>& d, const mp<PW>& a, const mp<PW>& b) {
+    static_assert(PW == 1 || PW == 2, "narrow phases only");
+    if constexpr (PW == 1) {
+        d.w[0] = a.w[0] - b.w[0];
+    } else {
+        asm("sub.cc.u32 %0, %2, %4;\n\t"
+            "subc.u32 %1, %3, %5;"
+            : "=&r"(d.w[0]), "=&r"(d.w[1])
+            : "r"(a.w[0]), "r"(a.w[1]), "r"(b.w[0]), "r"(b.w[1]));
+    }
+    return static_cast<int>(d.w[PW - 1]) < 0;
+}
+
 // State of one thread's walk.
 struct Walk {
     int v;        // pulses placed at the current position so far
@@ -73,12 +92,122 @@ struct Walk {
     uint32_t y0;  // ... for position 0
 };
 
+// The two factors of BatchArgs (1 and -1) the walk multiplies by.
+struct Factors {
+    uint32_t one, minus_one;
+};
+
+// One step at the entry U entries to the left of p (the caller moves p left after a block of
+// steps; p moves down here when a position ends).  The slot of the current position is
+// written at every step; the write of the step that ends the position is the last one.
+//
+// Generic form (any width, borrow flags), used by the widest phase.
+template <int PW, int EB, typename YT, int U>
+__device__ __forceinline__ void walk_step_wide(mp<PW>& r, uint32_t& p, int& v, uint32_t& y, const int D) {
+    const mp<PW> t = load_entry<PW, -U * EB>(p);
+    mp<PW> d2, d1;
+    const bool lt1 = mp_sub_borrow<PW>(d2, r, t);   // d2 = r - t
+    const bool lt2 = mp_sub_borrow<PW>(d1, d2, t);  // d1 = r - 2t
+    const bool placed = v > 0;
+    const bool ge1 = !lt1;
+    const bool ge2 = ge1 && !lt2 && placed;
+    const bool more = ge2 || (ge1 && !placed);  // another pulse at this position
+#pragma unroll
+    for (int w = 0; w < PW; ++w) r.w[w] = ge2 ? d1.w[w] : (ge1 ? d2.w[w] : r.w[w]);
+    store_y<YT>(y, (ge1 && placed) ? -v : v);
+    y += more ? 0u : static_cast<uint32_t>(sizeof(YT));
+    p += more ? 0u : static_cast<uint32_t>(D);
+    v = more ? v + 1 : 0;
+}
+
+// Narrow forms (1 and 2 words, operands below 2^(32 PW - 2) so that the sign of a difference
+// is the comparison), written out instruction by instruction.  Moves, the running counters
+// and (for one word) the subtractions are multiply-adds by 1 / -1 on the FMA pipe; compares,
+// carry chains and predicate logic stay on the integer pipe.
+template <int EB, typename YT, int U>
+__device__ __forceinline__ void walk_step_1(uint32_t& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                            const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, ng;\n\t"
+        ".reg .u32 t, d2, d1, x, val;\n\t"
+        "ld.shared.u32 t, [%3+%7];\n\t"
+        "mad.lo.u32 d2, t, %5, %0;\n\t"      // r - t
+        "mad.lo.u32 d1, t, %5, d2;\n\t"      // r - 2t
+        "setp.gt.s32 pl, %1, 0;\n\t"         // a pulse already placed here
+        "setp.ge.s32 g1, d2, 0;\n\t"
+        "selp.u32 x, d1, d2, pl;\n\t"        // the difference that decides "one more pulse"
+        "setp.ge.s32 mo, x, 0;\n\t"
+        "and.pred ng, g1, pl;\n\t"           // if the position ends here: negative
+        "@g1 mad.lo.u32 %0, d2, %4, 0;\n\t"  // r = d2
+        "@mo mad.lo.u32 %0, x, %4, 0;\n\t"   // r = x
+        "mad.lo.u32 val, %1, %4, 0;\n\t"     // +v
+        "@ng mad.lo.u32 val, %1, %5, 0;\n\t" // -v
+        "st.shared.u%9 [%2], val;\n\t"
+        "@!mo add.u32 %2, %2, %8;\n\t"       // next slot
+        "@!mo add.u32 %3, %3, %6;\n\t"       // next row
+        "mad.lo.u32 %1, %1, %4, %4;\n\t"     // v + 1
+        "@!mo mov.u32 %1, 0;\n\t"
+        "}"
+        : "+r"(r), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * EB), "n"(SZ), "n"(SZ * 8)
+        : "memory");
+}
+
+template <int EB, typename YT, int U>
+__device__ __forceinline__ void walk_step_2(mp<2>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                            const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, a0, a1, b0, b1, xh, val;\n\t"
+        "ld.shared.v2.u32 {t0, t1}, [%4+%8];\n\t"
+        "sub.cc.u32 a0, %0, t0;\n\t"          // d2 = r - t
+        "subc.u32 a1, %1, t1;\n\t"
+        "sub.cc.u32 b0, a0, t0;\n\t"          // d1 = r - 2t
+        "subc.u32 b1, a1, t1;\n\t"
+        "setp.gt.s32 pl, %2, 0;\n\t"
+        "setp.ge.s32 g1, a1, 0;\n\t"
+        "selp.u32 xh, b1, a1, pl;\n\t"
+        "setp.ge.s32 mo, xh, 0;\n\t"
+        "and.pred ng, g1, pl;\n\t"
+        "and.pred m2, mo, pl;\n\t"
+        "@g1 mad.lo.u32 %0, a0, %5, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %5, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %5, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %5, 0;\n\t"
+        "mad.lo.u32 val, %2, %5, 0;\n\t"
+        "@ng mad.lo.u32 val, %2, %6, 0;\n\t"
+        "st.shared.u%10 [%3], val;\n\t"
+        "@!mo add.u32 %3, %3, %9;\n\t"
+        "@!mo add.u32 %4, %4, %7;\n\t"
+        "mad.lo.u32 %2, %2, %5, %5;\n\t"
+        "@!mo mov.u32 %2, 0;\n\t"
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * EB), "n"(SZ), "n"(SZ * 8)
+        : "memory");
+}
+
+template <int PW, int EB, bool HEADROOM, typename YT, int U>
+__device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                          const Factors f) {
+    if constexpr (HEADROOM && PW == 1)
+        walk_step_1<EB, YT, U>(r.w[0], p, v, y, D, f);
+    else if constexpr (HEADROOM && PW == 2)
+        walk_step_2<EB, YT, U>(r, p, v, y, D, f);
+    else
+        walk_step_wide<PW, EB, YT, U>(r, p, v, y, D);
+}
+
 // Runs steps s .. S-1 on PW-word integers with the table `tab` (entries of EB bytes),
 // leaving early, at a multiple of 8 steps, once every thread's r fits `next_words` words
-// with a bit to spare.  Returns the step reached.
-template <int PW, int EB, int CW, typename YT>
+// with two bits to spare.  Returns the step reached.
+template <int PW, int EB, bool HEADROOM, int CW, typename YT>
 __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab, int rowlen, int K, int s,
-                                          const int S, const int next_words) {
+                                          const int S, const int next_words, const Factors f) {
     mp<PW> r;
 #pragma unroll
     for (int w = 0; w < PW; ++w) r.w[w] = rfull.w[w];
@@ -88,42 +217,32 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
     int v = st.v;
     uint32_t y = st.y;
 
-    auto step = [&]() {
-        const mp<PW> t = load_entry<PW>(p);
-        mp<PW> d2, d1;
-        const bool lt1 = mp_sub_borrow<PW>(d2, r, t);   // d2 = r - t
-        const bool lt2 = mp_sub_borrow<PW>(d1, d2, t);  // d1 = r - 2t
-        const bool placed = v > 0;
-        const bool ge1 = !lt1;
-        const bool ge2 = ge1 && !lt2 && placed;
-        const bool more = placed ? ge2 : ge1;  // another pulse at this position
-#pragma unroll
-        for (int w = 0; w < PW; ++w) r.w[w] = ge2 ? d1.w[w] : (ge1 ? d2.w[w] : r.w[w]);
-        if (!more) {
-            store_y<YT>(y, (ge1 && placed) ? -v : v);
-            y += sizeof(YT);
-            p += D;
-        }
-        v = more ? v + 1 : 0;
-        p -= EB;
-    };
-
     while (s + 8 <= S) {
         if (next_words > 0) {
-            // does r fit next_words words with the top bit clear?
+            // does r fit next_words words with the two top bits clear?
             uint32_t hi = 0;
 #pragma unroll
             for (int w = 2; w < PW; ++w) hi |= r.w[w];
-            if constexpr (PW > 1) hi |= next_words == 2 ? (r.w[1] >> 31) : r.w[1];
-            if (next_words == 1) hi |= r.w[0] >> 31;
+            if constexpr (PW > 1) hi |= next_words == 2 ? (r.w[1] >> 30) : r.w[1];
+            if (next_words == 1) hi |= r.w[0] >> 30;
             if (__all_sync(kFull, hi == 0u)) break;
         }
-#pragma unroll
-        for (int u = 0; u < 8; ++u) step();
+        walk_step<PW, EB, HEADROOM, YT, 0>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 1>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 2>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 3>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 4>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 5>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 6>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 7>(r, p, v, y, D, f);
+        p -= 8 * EB;
         s += 8;
     }
     if (next_words == 0 || s + 8 > S) {
-        for (; s < S; ++s) step();
+        for (; s < S; ++s) {
+            walk_step<PW, EB, HEADROOM, YT, 0>(r, p, v, y, D, f);
+            p -= EB;
+        }
     }
 #pragma unroll
     for (int w = 0; w < PW; ++w) rfull.w[w] = r.w[w];
@@ -132,15 +251,16 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
     return s;
 }
 
-
 // The three staged walk tables as shared addresses, and which of them exist.
 struct WalkTables {
     uint32_t tab0, tab2, tab1;
     bool has2, has1;
     int rowlen;
+    Factors f;
 };
 
-__device__ __forceinline__ WalkTables walk_tables(const TableLayout& L, uint32_t smem_base, int phases) {
+__device__ __forceinline__ WalkTables walk_tables(const TableLayout& L, uint32_t smem_base, int phases,
+                                                  const BatchArgs& a) {
     WalkTables t;
     t.tab0 = smem_base;
     t.tab2 = smem_base + (L.walk_off[1] - L.walk_off[0]);
@@ -148,6 +268,8 @@ __device__ __forceinline__ WalkTables walk_tables(const TableLayout& L, uint32_t
     t.has2 = phases >= 2 && L.walk_bytes[1] != 0;
     t.has1 = phases >= 3;
     t.rowlen = L.rowlen;
+    t.f.one = a.c_one;
+    t.f.minus_one = a.c_minus_one;
     return t;
 }
 
@@ -174,12 +296,12 @@ __device__ __forceinline__ void walk_code(mp<W>& c, const WalkTables& t, int K, 
     st.v = 0;
     st.y = st.y0 = shared_addr(yslots);
     int s = 0;
-    s = walk_phase<W, TW * 4, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, t.has2 ? 2 : (t.has1 ? 1 : 0));
+    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, t.has2 ? 2 : (t.has1 ? 1 : 0), t.f);
     if constexpr (W > 2) {
-        if (s < S && t.has2) s = walk_phase<2, 8, W, YT>(c, st, t.tab2, t.rowlen, K, s, S, t.has1 ? 1 : 0);
+        if (s < S && t.has2) s = walk_phase<2, 8, true, W, YT>(c, st, t.tab2, t.rowlen, K, s, S, t.has1 ? 1 : 0, t.f);
     }
     if constexpr (W > 1) {
-        if (s < S && t.has1) s = walk_phase<1, 4, W, YT>(c, st, t.tab1, t.rowlen, K, s, S, 0);
+        if (s < S && t.has1) s = walk_phase<1, 4, true, W, YT>(c, st, t.tab1, t.rowlen, K, s, S, 0, t.f);
     }
 }
 
