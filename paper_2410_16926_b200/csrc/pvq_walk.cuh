@@ -92,6 +92,11 @@ struct Walk {
     uint32_t y0;  // ... for position 0
 };
 
+// What a slot holds for y_i: y_i + 128 in a byte (the store's float conversion then needs no
+// sign handling), or y_i itself in 16 bits when K does not fit a byte.
+template <typename YT>
+constexpr int kSlotBias = sizeof(YT) == 1 ? 128 : 0;
+
 // The two factors of BatchArgs (1 and -1) the walk multiplies by.
 struct Factors {
     uint32_t one, minus_one;
@@ -114,7 +119,7 @@ __device__ __forceinline__ void walk_step_wide(mp<PW>& r, uint32_t& p, int& v, u
     const bool more = ge2 || (ge1 && !placed);  // another pulse at this position
 #pragma unroll
     for (int w = 0; w < PW; ++w) r.w[w] = ge2 ? d1.w[w] : (ge1 ? d2.w[w] : r.w[w]);
-    store_y<YT>(y, (ge1 && placed) ? -v : v);
+    store_y<YT>(y, ((ge1 && placed) ? -v : v) + kSlotBias<YT>);
     y += more ? 0u : static_cast<uint32_t>(sizeof(YT));
     p += more ? 0u : static_cast<uint32_t>(D);
     v = more ? v + 1 : 0;
@@ -142,8 +147,8 @@ __device__ __forceinline__ void walk_step_1(uint32_t& r, uint32_t& p, int& v, ui
         "and.pred ng, g1, pl;\n\t"           // if the position ends here: negative
         "@g1 mad.lo.u32 %0, d2, %4, 0;\n\t"  // r = d2
         "@mo mad.lo.u32 %0, x, %4, 0;\n\t"   // r = x
-        "mad.lo.u32 val, %1, %4, 0;\n\t"     // +v
-        "@ng mad.lo.u32 val, %1, %5, 0;\n\t" // -v
+        "mad.lo.u32 val, %1, %4, %10;\n\t"     // bias + v
+        "@ng mad.lo.u32 val, %1, %5, %10;\n\t" // bias - v
         "st.shared.u%9 [%2], val;\n\t"
         "@!mo add.u32 %2, %2, %8;\n\t"       // next slot
         "@!mo add.u32 %3, %3, %6;\n\t"       // next row
@@ -151,7 +156,7 @@ __device__ __forceinline__ void walk_step_1(uint32_t& r, uint32_t& p, int& v, ui
         "@!mo mov.u32 %1, 0;\n\t"
         "}"
         : "+r"(r), "+r"(v), "+r"(y), "+r"(p)
-        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * EB), "n"(SZ), "n"(SZ * 8)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * EB), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
 
@@ -178,8 +183,8 @@ __device__ __forceinline__ void walk_step_2(mp<2>& r, uint32_t& p, int& v, uint3
         "@g1 mad.lo.u32 %1, a1, %5, 0;\n\t"
         "@m2 mad.lo.u32 %0, b0, %5, 0;\n\t"
         "@m2 mad.lo.u32 %1, b1, %5, 0;\n\t"
-        "mad.lo.u32 val, %2, %5, 0;\n\t"
-        "@ng mad.lo.u32 val, %2, %6, 0;\n\t"
+        "mad.lo.u32 val, %2, %5, %11;\n\t"
+        "@ng mad.lo.u32 val, %2, %6, %11;\n\t"
         "st.shared.u%10 [%3], val;\n\t"
         "@!mo add.u32 %3, %3, %9;\n\t"
         "@!mo add.u32 %4, %4, %7;\n\t"
@@ -187,9 +192,98 @@ __device__ __forceinline__ void walk_step_2(mp<2>& r, uint32_t& p, int& v, uint3
         "@!mo mov.u32 %2, 0;\n\t"
         "}"
         : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(v), "+r"(y), "+r"(p)
-        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * EB), "n"(SZ), "n"(SZ * 8)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * EB), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
+
+// Widest phase for 3- and 4-word codes (16-byte entries), borrow flags instead of sign bits.
+#define PVQ_WIDE_TAIL(R0, NXT)                                                         \
+        "setp.gt.s32 pl, %" #R0 ", 0;\n\t"                                            \
+        "setp.eq.u32 g1, ab, 0;\n\t"                                                   \
+        "or.b32 ob, ab, bb;\n\t"                                                       \
+        "selp.u32 ob, ob, ab, pl;\n\t"                                                 \
+        "setp.eq.u32 mo, ob, 0;\n\t"                                                   \
+        "and.pred ng, g1, pl;\n\t"                                                     \
+        "and.pred m2, mo, pl;\n\t"
+
+template <typename YT, int U>
+__device__ __forceinline__ void walk_step_w3(mp<3>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                             const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, t2, t3, a0, a1, a2, ab, b0, b1, b2, bb, ob, val;\n\t"
+        "ld.shared.v4.u32 {t0, t1, t2, t3}, [%5+%9];\n\t"
+        "sub.cc.u32 a0, %0, t0;\n\t"
+        "subc.cc.u32 a1, %1, t1;\n\t"
+        "subc.cc.u32 a2, %2, t2;\n\t"
+        "subc.u32 ab, 0, 0;\n\t"               // 0 or -1: r < t
+        "sub.cc.u32 b0, a0, t0;\n\t"
+        "subc.cc.u32 b1, a1, t1;\n\t"
+        "subc.cc.u32 b2, a2, t2;\n\t"
+        "subc.u32 bb, 0, 0;\n\t"               // r - t < t
+        PVQ_WIDE_TAIL(3, 0)
+        "@g1 mad.lo.u32 %0, a0, %6, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %6, 0;\n\t"
+        "@g1 mad.lo.u32 %2, a2, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %2, b2, %6, 0;\n\t"
+        "mad.lo.u32 val, %3, %6, %12;\n\t"
+        "@ng mad.lo.u32 val, %3, %7, %12;\n\t"
+        "st.shared.u%11 [%4], val;\n\t"
+        "@!mo add.u32 %4, %4, %10;\n\t"
+        "@!mo add.u32 %5, %5, %8;\n\t"
+        "mad.lo.u32 %3, %3, %6, %6;\n\t"
+        "@!mo mov.u32 %3, 0;\n\t"
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 16), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+
+template <typename YT, int U>
+__device__ __forceinline__ void walk_step_w4(mp<4>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                             const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, t2, t3, a0, a1, a2, a3, ab, b0, b1, b2, b3, bb, ob, val;\n\t"
+        "ld.shared.v4.u32 {t0, t1, t2, t3}, [%6+%10];\n\t"
+        "sub.cc.u32 a0, %0, t0;\n\t"
+        "subc.cc.u32 a1, %1, t1;\n\t"
+        "subc.cc.u32 a2, %2, t2;\n\t"
+        "subc.cc.u32 a3, %3, t3;\n\t"
+        "subc.u32 ab, 0, 0;\n\t"
+        "sub.cc.u32 b0, a0, t0;\n\t"
+        "subc.cc.u32 b1, a1, t1;\n\t"
+        "subc.cc.u32 b2, a2, t2;\n\t"
+        "subc.cc.u32 b3, a3, t3;\n\t"
+        "subc.u32 bb, 0, 0;\n\t"
+        PVQ_WIDE_TAIL(4, 0)
+        "@g1 mad.lo.u32 %0, a0, %7, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %7, 0;\n\t"
+        "@g1 mad.lo.u32 %2, a2, %7, 0;\n\t"
+        "@g1 mad.lo.u32 %3, a3, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %2, b2, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %3, b3, %7, 0;\n\t"
+        "mad.lo.u32 val, %4, %7, %13;\n\t"
+        "@ng mad.lo.u32 val, %4, %8, %13;\n\t"
+        "st.shared.u%12 [%5], val;\n\t"
+        "@!mo add.u32 %5, %5, %11;\n\t"
+        "@!mo add.u32 %6, %6, %9;\n\t"
+        "mad.lo.u32 %4, %4, %7, %7;\n\t"
+        "@!mo mov.u32 %4, 0;\n\t"
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(r.w[3]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 16), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+#undef PVQ_WIDE_TAIL
 
 template <int PW, int EB, bool HEADROOM, typename YT, int U>
 __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32_t& y, const int D,
@@ -198,6 +292,10 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
         walk_step_1<EB, YT, U>(r.w[0], p, v, y, D, f);
     else if constexpr (HEADROOM && PW == 2)
         walk_step_2<EB, YT, U>(r, p, v, y, D, f);
+    else if constexpr (!HEADROOM && PW == 3)
+        walk_step_w3<YT, U>(r, p, v, y, D, f);
+    else if constexpr (!HEADROOM && PW == 4)
+        walk_step_w4<YT, U>(r, p, v, y, D, f);
     else
         walk_step_wide<PW, EB, YT, U>(r, p, v, y, D);
 }
@@ -313,13 +411,19 @@ template <int N, typename YT>
 __device__ __forceinline__ void emit_tile(const MatrixArgs& m, uint8_t* wbuf, float* wscale, int lane, float amp,
                                           long long g0, long long ngroups) {
     constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
-    const YT* yslots = reinterpret_cast<const YT*>(wbuf + lane * YS);
     int ssy = 0;
     if constexpr (sizeof(YT) == 1) {
-        const int* y4 = reinterpret_cast<const int*>(yslots);
+        // slots hold b = y + 128:  sum y^2 = sum b^2 - 256 sum b + 128^2 N
+        const unsigned* y4 = reinterpret_cast<const unsigned*>(wbuf + lane * YS);
+        unsigned sq = 0, su = 0;
 #pragma unroll
-        for (int v = 0; v < N / 4; ++v) ssy = __dp4a(y4[v], y4[v], ssy);
+        for (int v = 0; v < N / 4; ++v) {
+            sq = __dp4a(y4[v], y4[v], sq);
+            su = __dp4a(y4[v], 0x01010101u, su);
+        }
+        ssy = static_cast<int>(sq) - 256 * static_cast<int>(su) + 16384 * N;
     } else {
+        const YT* yslots = reinterpret_cast<const YT*>(wbuf + lane * YS);
 #pragma unroll 8
         for (int v = 0; v < N; ++v) ssy += static_cast<int>(yslots[v]) * static_cast<int>(yslots[v]);
     }
@@ -329,28 +433,44 @@ __device__ __forceinline__ void emit_tile(const MatrixArgs& m, uint8_t* wbuf, fl
     constexpr int TPG = N / 8;     // threads per group, 16 bytes each
     constexpr int GPI = 32 / TPG;  // groups per iteration
     const int part = lane % TPG;
+    // row and group-in-row of the tile's first group; the tile's other groups follow from it
+    // without a division as long as they sit in that row or the next
+    const unsigned G = static_cast<unsigned>(m.G);
+    const unsigned row0 = static_cast<unsigned>(g0) / G;
+    const unsigned off0 = static_cast<unsigned>(g0) - row0 * G;
 #pragma unroll 1
     for (int it = 0; it < TPG; ++it) {
         const int gl = it * GPI + lane / TPG;  // group within the tile
         const long long gj = g0 + gl;
         if (gj < ngroups) {
-            const YT* ys = reinterpret_cast<const YT*>(wbuf + gl * YS) + part * 8;
+            const uint8_t* ys = wbuf + gl * YS + part * 8 * sizeof(YT);
             const float sc = wscale[gl];
             float f[8];
             if constexpr (sizeof(YT) == 1) {
+                // byte b into the low mantissa bits of 2^23: the float 2^23 + b, then minus 2^23 + 128
                 const uint32_t lo = reinterpret_cast<const uint32_t*>(ys)[0];
                 const uint32_t hi = reinterpret_cast<const uint32_t*>(ys)[1];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    f[e] = static_cast<float>(static_cast<int>(static_cast<int8_t>(lo >> (8 * e))));
-                    f[4 + e] = static_cast<float>(static_cast<int>(static_cast<int8_t>(hi >> (8 * e))));
+                    f[e] = __fsub_rn(__uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7540u + e)), 8388736.0f);
+                    f[4 + e] = __fsub_rn(__uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7540u + e)), 8388736.0f);
                 }
             } else {
+                const YT* yv = reinterpret_cast<const YT*>(ys);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = static_cast<float>(static_cast<int>(ys[e]));
+                for (int e = 0; e < 8; ++e) f[e] = static_cast<float>(static_cast<int>(yv[e]));
             }
-            const unsigned row = static_cast<unsigned>(gj) / static_cast<unsigned>(m.G);
-            const unsigned g = static_cast<unsigned>(gj) - row * static_cast<unsigned>(m.G);
+            unsigned g = off0 + static_cast<unsigned>(gl);
+            unsigned row = row0;
+            if (g >= G) {
+                g -= G;
+                row += 1;
+                if (g >= G) {  // rows shorter than a tile
+                    const unsigned q = g / G;
+                    row += q;
+                    g -= q * G;
+                }
+            }
             uint4 o;
             o.x = pack_bf16x2(__fmul_rn(f[0], sc), __fmul_rn(f[1], sc));
             o.y = pack_bf16x2(__fmul_rn(f[2], sc), __fmul_rn(f[3], sc));
