@@ -31,10 +31,24 @@
  *                      [g*b, (g+1)*b) of the row, b = scale_bits; the row stride
  *                      is pvq_scale_row_stride(G, b) = ceil(G*b/8) rounded up to 4.
  *   row_norm   float   row_norm[r].
- *   count table uint32 table[(n*(K+1) + k)*W + w] = word w of N(n,k) for
- *                      n = 0..N-1 (dimensions left after a position) and
- *                      k = 0..K; pvq_count_table_bytes(N,K) bytes, 16-byte
- *                      aligned.
+ *   count table uint32 pvq_count_table_bytes(N,K) bytes, 16-byte aligned, written by
+ *                      pvq_build_count_table.  It opens with the table of the paper,
+ *                      table[(n*(K+1) + k)*W + w] = word w of N(n,k) for n = 0..N-1
+ *                      (dimensions left after a position) and k = 0..K.  For N <= 64
+ *                      and W <= 6 the same numbers follow, rearranged for the kernels
+ *                      (each section starts on a 128-byte boundary, in this order):
+ *                        N(N,K) as 8 words;
+ *                        the decoder's tables, rows by position i (row i = N(N-1-i, .)),
+ *                        K+1 rounded up to even entries per row: one with entries of
+ *                        1, 2, 4 or 6 words (the first that holds W), then, when W > 2,
+ *                        one with 2-word entries where values from 2^62 up are
+ *                        replaced by 2^62, and, when W > 1, one with 1-word entries
+ *                        where values from 2^30 up are replaced by 2^30;
+ *                        the encoder's tables, rows by position, K+2 entries per row for
+ *                        k = -1..K, of the cumulative counts V(n,k) = sum_{j<=k} N(n,j)
+ *                        (App. C.2) modulo 2^(32 W): V(n,k) + V(n,k-1), then 2 V(n,k),
+ *                        then V(n,k).
+ *                      Callers treat everything after the first section as opaque.
  *   edges      float   2^b - 1 ascending bin edges of u.
  *   levels     float   2^b values sqrt(PPF((q + 1/2) / 2^b)): the factor that
  *                      multiplies row_norm to give the dequantised amplitude.
@@ -85,7 +99,8 @@ int pvq_max_pulses(int N, int index_bits, int* K_out);
 /* W = ceil(pvq_index_bits / 32), at least 1. */
 int pvq_code_words(int N, int K, int* W_out);
 
-/* Bytes of the device count table for (N,K): N * (K+1) * W * 4.  0 on bad arguments. */
+/* Bytes of the device count table for (N,K), all sections: at least N * (K+1) * W * 4.
+ * 0 on bad arguments. */
 size_t pvq_count_table_bytes(int N, int K);
 
 /* Row stride in bytes of the packed amplitude indices. */

@@ -77,6 +77,62 @@ def test_count_table_word_for_word(N, K):
     assert np.array_equal(as_u32(pvq.count_table_view(t, N, K)), ref)
 
 
+def _blob_layout(N, K, W):
+    """Byte offsets of the sections that follow the count table (see include/pvq.h)."""
+    up = lambda v: (v + 127) & ~127
+    rowlen = (K + 2) & ~1
+    top = W if W <= 2 else (4 if W <= 4 else 6)
+    off = up(N * (K + 1) * W * 4)
+    lay = {"bound": off, "rowlen": rowlen, "top": top}
+    off += 128
+    for name, words in (("walk_top", top), ("walk2", 2 if top > 2 else 0), ("walk1", 1 if top > 1 else 0)):
+        lay[name] = (off, words)
+        off += up(N * rowlen * words * 4)
+    for name in ("enc_u", "enc_2v", "enc_v"):
+        lay[name] = off
+        off += up(N * (K + 2) * top * 4)
+    lay["total"] = off
+    return lay
+
+
+@pytest.mark.parametrize("N,K", [(8, 16), (16, 18), (32, 22), (32, 50), (32, 105), (64, 96), (64, 26)])
+def test_table_blob_sections(N, K):
+    """Every rearranged section of the table blob holds the numbers of the count table."""
+    W = pvq.code_words(N, K)
+    blob = as_u32(pvq.build_count_table(N, K))
+    torch.cuda.synchronize()
+    lay = _blob_layout(N, K, W)
+    assert blob.size * 4 == lay["total"] == pvq.count_table_bytes(N, K)
+    full = po.count_table(N, K, W)                      # rows n = 0..N
+    val = [[po.code_to_int(full[n, k]) for k in range(K + 1)] for n in range(N + 1)]
+    mask = (1 << (32 * W)) - 1
+    words = lambda v, nw: [(v >> (32 * w)) & 0xFFFFFFFF for w in range(nw)]
+    assert list(blob[lay["bound"] // 4: lay["bound"] // 4 + 8]) == words(val[N][K], 8)
+    rowlen, top = lay["rowlen"], lay["top"]
+    for name, sat_bits in (("walk_top", None), ("walk2", 62), ("walk1", 30)):
+        off, nw = lay[name]
+        if nw == 0:
+            continue
+        sec = blob[off // 4: off // 4 + N * rowlen * nw].reshape(N, rowlen, nw)
+        for i in range(N):
+            for col in range(K + 1):
+                v = val[N - 1 - i][col]
+                if sat_bits is not None and v >= (1 << sat_bits):
+                    v = 1 << sat_bits
+                assert list(sec[i, col]) == words(v, nw), (name, i, col)
+    for name in ("enc_u", "enc_2v", "enc_v"):
+        off = lay[name]
+        sec = blob[off // 4: off // 4 + N * (K + 2) * top].reshape(N, K + 2, top)
+        for i in range(N):
+            V = [0]
+            for col in range(K + 1):
+                V.append(V[-1] + val[N - 1 - i][col])          # V[col + 1] = V(n, col), V[0] = V(n, -1)
+            for c1 in range(K + 2):
+                prev = V[c1 - 1] if c1 > 0 else 0
+                want = {"enc_u": V[c1] + prev, "enc_2v": 2 * V[c1], "enc_v": V[c1]}[name] & mask
+                assert list(sec[i, c1]) == words(want, top), (name, i, c1)
+
+
 @pytest.mark.parametrize("N,G,b", [(32, 16, 8), (32, 128, 4), (32, 448, 8), (64, 448, 6), (32, 128, 8),
                                    (8, 2, 3), (16, 5, 1)])
 def test_scale_codebook_against_scipy(N, G, b):
