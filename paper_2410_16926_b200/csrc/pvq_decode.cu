@@ -1,9 +1,9 @@
 // Decode kernel: direction code -> pyramid point (Algorithm 3) -> unit sphere
 // times dequantised amplitude -> bf16 (Sec. 2.4, Sec. 3.4).
 //
-// One thread decodes one group; a warp takes 32 consecutive groups, walks their
-// codes in lockstep (pvq_walk.cuh) and writes the 32 groups with coalesced
-// 16-byte stores from shared memory.
+// One thread decodes one group; a warp takes 32 consecutive groups and walks their
+// codes in lockstep (pvq_walk.cuh), each thread collecting its point in shared
+// memory, from where it scales it and writes its N bf16 values with 16-byte stores.
 #include <algorithm>
 
 #include "pvq_walk.cuh"
@@ -31,9 +31,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    uint8_t* wbuf = smem + ((tab_bytes + 15u) & ~15u) + warp * (32 * YS + 128);
-    YT* yslots = reinterpret_cast<YT*>(wbuf + lane * YS);
-    float* wscale = reinterpret_cast<float*>(wbuf + 32 * YS);
+    YT* yslots = reinterpret_cast<YT*>(smem + ((tab_bytes + 15u) & ~15u) + threadIdx.x * YS);
 
     // N(N,K): codes at or above it are invalid
     mp<W> bound;
@@ -43,31 +41,42 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
     const bool bound_wide = bw[W] != 0u;  // N(N,K) = 2^(32W) exactly: every W-word code is valid
     __syncthreads();
 
-    const int b = a.scale_bits;
+    const unsigned b = a.scale_bits;
     const unsigned warps_total = gridDim.x * (blockDim.x >> 5);
     bool bad = false;
 
     for (unsigned tile = blockIdx.x * (blockDim.x >> 5) + warp; tile < a.total_tiles; tile += warps_total) {
         const int mi = find_matrix(a, tile);
         const MatrixArgs& m = a.m[mi];
-        const long long g0 = static_cast<long long>(tile - m.tile_begin) * 32;  // first group of the tile
-        const long long ngroups = m.rows * m.G;
-        const long long gi = g0 + lane;
+        const unsigned G = static_cast<unsigned>(m.G);
+        const unsigned ngroups = static_cast<unsigned>(m.rows) * G;  // below 2^31 (checked by the host)
+        const unsigned g0 = (tile - m.tile_begin) * 32u;             // first group of the tile
+        const unsigned gi = g0 + lane;
         const bool active = gi < ngroups;
+        // row and group-in-row: one division per tile, the threads follow from the first group
+        unsigned row = g0 / G;
+        unsigned g = g0 - row * G + lane;
+        if (g >= G) {
+            g -= G;
+            row += 1;
+            if (g >= G) {  // rows shorter than a tile
+                const unsigned q = g / G;
+                row += q;
+                g -= q * G;
+            }
+        }
 
         mp<W> c;
         mp_zero(c);
         float amp = 0.0f;
         if (active) {
-            c = mp_load<W>(m.codes + gi * W);
+            c = mp_load<W>(m.codes + static_cast<size_t>(gi) * W);
             mp<W> tmp;
             const bool valid = bound_wide || mp_sub_borrow<W>(tmp, c, bound);
             if (!valid) {  // decodes to zeros: walk code 0, whose point has no negative entry
                 bad = true;
                 mp_zero(c);
             } else {
-                const unsigned row = static_cast<unsigned>(gi) / static_cast<unsigned>(m.G);
-                const unsigned g = static_cast<unsigned>(gi) - row * static_cast<unsigned>(m.G);
                 // amplitude index: bits [g*b, g*b + b) of the row's LSB-first stream
                 const uint8_t* srow = m.scale_idx + static_cast<size_t>(row) * m.sstride;
                 const unsigned bit = g * b;
@@ -78,7 +87,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
             }
         }
         walk_code<N, W, YT>(c, wt, K, yslots);
-        emit_tile<N, YT>(m, wbuf, wscale, lane, amp, g0, ngroups);
+        if (active) emit_group<N, YT>(m, yslots, amp, row, g);
     }
     if (bad && a.status) atomicOr(a.status, PVQ_STATUS_INVALID_CODE);
 }
@@ -94,20 +103,17 @@ int launch_decode_t(BatchArgs& a, cudaStream_t stream) {
     }
     a.total_tiles = tiles;
     const TableLayout L = table_layout(N, a.K, W);
-    int dev = 0, sms = 0, smem_max = 0;
-    cudaError_t e;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return set_cuda_error(e);
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
-        return set_cuda_error(e);
-    if ((e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
-        return set_cuda_error(e);
+    DeviceInfo di;
+    int st = device_info(&di);
+    if (st != PVQ_OK) return st;
+    const int sms = di.sms, smem_max = di.smem_max;
     // As many of the narrower walk tables as fit beside the widest one; fewer threads if even
     // that leaves no room for their output slots.
     int threads = kDecThreads;
     int phases = 0;
     size_t smem = 0;
     for (; threads >= 128; threads /= 2) {
-        const size_t wbufs = static_cast<size_t>(threads / 32) * (32 * YS + 128);
+        const size_t wbufs = static_cast<size_t>(threads) * YS;
         phases = walk_phases_that_fit(L, static_cast<size_t>(smem_max) - std::min<size_t>(smem_max, wbufs));
         if (phases) {
             smem = ((walk_tables_bytes(L, phases) + 15u) & ~size_t(15)) + wbufs;
@@ -117,18 +123,14 @@ int launch_decode_t(BatchArgs& a, cudaStream_t stream) {
     if (phases == 0) return PVQ_ERR_UNSUPPORTED;
     a.walk_phases = phases;
     auto kern = decode_kernel<N, W, YT>;
-    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))) !=
-        cudaSuccess)
-        return set_cuda_error(e);
     int per_sm = 0;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem)) != cudaSuccess)
-        return set_cuda_error(e);
+    if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
     const unsigned warps_per_block = threads / 32;
     const unsigned blocks_needed = (tiles + warps_per_block - 1) / warps_per_block;
     const unsigned grid = std::max(1u, std::min<unsigned>(blocks_needed, static_cast<unsigned>(sms * per_sm)));
     kern<<<grid, threads, smem, stream>>>(a);
-    e = cudaGetLastError();
+    const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 

@@ -362,14 +362,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     const uint32_t tabB = tabA + ((L.enc_bytes + 127u) & ~127u);  // 2V, when two tables are staged
     const int rowbytes = (K + 2) * EB;
     WalkTables wt;
-    uint8_t* wbuf = nullptr;
-    float* wscale = nullptr;
     YT* yslots = nullptr;
     if constexpr (FUSED) {
         wt = walk_tables(L, tabA + sm.enc_bytes, sm.walk_phases, a);
-        wbuf = smem + sm.wbuf_off + warp * (32 * YS + 128);
-        yslots = reinterpret_cast<YT*>(wbuf + lane * YS);
-        wscale = reinterpret_cast<float*>(wbuf + 32 * YS);
+        yslots = reinterpret_cast<YT*>(smem + sm.wbuf_off + threadIdx.x * YS);
     }
     const float* cur_edges = nullptr;
 
@@ -511,14 +507,11 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
                         s_idx[i];
             }
         } else {
-            // decode the code just made: walk, then scale and store the warp's 32 groups.
-            // Threads t .. t+31 of a warp hold consecutive groups of the tile's rows.
+            // decode the code just made (every thread of the warp walks, in lockstep)
             const float amp = active ? __fmul_rn(rnorm, s_levels[q]) : 0.0f;
             if (!active) mp_zero(c);
             walk_code<N, W, YT>(c, wt, K, yslots);
-            const long long g0 = row0 * G + (threadIdx.x & ~31);
-            const long long gend = (m.rows < row0 + rpt ? m.rows : row0 + rpt) * G;
-            emit_tile<N, YT>(m, wbuf, wscale, lane, amp, g0, gend);
+            if (active) emit_group<N, YT>(m, yslots, amp, static_cast<unsigned>(row), static_cast<unsigned>(g));
         }
 
         if (!have_next) break;
@@ -571,17 +564,14 @@ static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     }
     a.total_tiles = tiles;
 
-    int dev = 0, sms = 0, smem_max = 0;
-    cudaError_t e;
-    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return set_cuda_error(e);
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
-        return set_cuda_error(e);
-    if ((e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
-        return set_cuda_error(e);
+    DeviceInfo di;
+    int st = device_info(&di);
+    if (st != PVQ_OK) return st;
+    const int sms = di.sms, smem_max = di.smem_max;
 
     const TableLayout L = table_layout(N, a.K, W);
     const size_t small = (2 * static_cast<size_t>(ss_floats) + 256 + (FUSED ? 256 : 0) + 2 * max_idx_words) * 4u + 64u;
-    const size_t wbufs = FUSED ? static_cast<size_t>(threads / 32) * (32 * YS + 128) : 0;
+    const size_t wbufs = FUSED ? static_cast<size_t>(threads) * YS : 0;
     const size_t enc_one = (L.enc_bytes + 127u) & ~size_t(127);
     EncodeSmem sm;
     sm.walk_bytes = 0;
@@ -617,16 +607,12 @@ static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     if (smem > static_cast<size_t>(smem_max)) return PVQ_ERR_UNSUPPORTED;
 
     auto kern = encode_kernel<N, W, FUSED, YT, BF16>;
-    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem))) !=
-        cudaSuccess)
-        return set_cuda_error(e);
     int per_sm = 0;
-    if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem)) != cudaSuccess)
-        return set_cuda_error(e);
+    if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
     const unsigned grid = std::min<unsigned>(tiles, static_cast<unsigned>(sms * per_sm));
     kern<<<grid, threads, smem, stream>>>(a, sm);
-    e = cudaGetLastError();
+    const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 

@@ -4,6 +4,7 @@
 #include <cstring>
 #include <map>
 #include <mutex>
+#include <tuple>
 #include <utility>
 #include <vector>
 
@@ -84,6 +85,60 @@ static int index_bits_exact(int N, int K) {
     for (int k = 0; k < K; ++k)
         if (!c.advance()) return -1;
     return c.col[static_cast<size_t>(N)].ceil_log2();
+}
+
+int device_info(DeviceInfo* out) {
+    static std::mutex mu;
+    static std::map<int, DeviceInfo> memo;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find(dev);
+    if (it == memo.end()) {
+        DeviceInfo d;
+        if ((e = cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+            return set_cuda_error(e);
+        if ((e = cudaDeviceGetAttribute(&d.smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+            return set_cuda_error(e);
+        it = memo.emplace(dev, d).first;
+    }
+    *out = it->second;
+    return PVQ_OK;
+}
+
+int prepare_kernel(const void* kern, int threads, size_t smem, int* blocks_per_sm) {
+    struct Key {
+        const void* kern;
+        int dev, threads;
+        size_t smem;
+        bool operator<(const Key& o) const {
+            return std::tie(kern, dev, threads, smem) < std::tie(o.kern, o.dev, o.threads, o.smem);
+        }
+    };
+    static std::mutex mu;
+    static std::map<Key, int> memo;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_cuda_error(e);
+    std::lock_guard<std::mutex> lock(mu);
+    const Key key{kern, dev, threads, smem};
+    auto it = memo.find(key);
+    if (it == memo.end()) {
+        // the attribute is per kernel and device: keep it at the largest size asked for so far
+        size_t largest = smem;
+        for (const auto& kv : memo)
+            if (kv.first.kern == kern && kv.first.dev == dev) largest = std::max(largest, kv.first.smem);
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(largest))) !=
+            cudaSuccess)
+            return set_cuda_error(e);
+        int per_sm = 0;
+        if ((e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem)) != cudaSuccess)
+            return set_cuda_error(e);
+        it = memo.emplace(key, per_sm).first;
+    }
+    *blocks_per_sm = it->second;
+    return PVQ_OK;
 }
 
 // W for (N,K); memoised, since every hot call asks for it.

@@ -117,6 +117,16 @@ int set_cuda_error(cudaError_t e);  // records e, returns PVQ_ERR_CUDA
 int code_words_for(int N, int K);   // W, or 0 when it cannot be computed
 bool is_aligned(const void* p, size_t a);
 
+// What a launcher needs to know about the current device and a kernel at a given block size
+// and dynamic shared memory: looked up once, then served from a cache (the queries cost more
+// than a small launch).  prepare_kernel also raises the kernel's shared-memory limit.
+struct DeviceInfo {
+    int sms;
+    int smem_max;  // opt-in shared memory per block
+};
+int device_info(DeviceInfo* out);                                                  // pvq_status
+int prepare_kernel(const void* kern, int threads, size_t smem, int* blocks_per_sm);  // pvq_status
+
 // launchers (one per kernel family); all return a pvq_status
 int launch_decode(const BatchArgs& args, int N, int W, cudaStream_t stream);
 int launch_encode(const BatchArgs& args, int dtype, int N, int W, bool fused, cudaStream_t stream);

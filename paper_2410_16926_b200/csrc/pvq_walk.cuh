@@ -403,18 +403,17 @@ __device__ __forceinline__ void walk_code(mp<W>& c, const WalkTables& t, int K, 
     }
 }
 
-// After walk_code by all threads of a warp: scale each group's point to the unit sphere
-// times `amp` (this thread's group) and write the warp's 32 groups as bf16 with 16-byte
-// stores.  wbuf: the warp's slot area (thread l at wbuf + l*YS), wscale: 32 floats.
-// Group l of the tile is global group g0 + l of matrix m; groups >= ngroups are skipped.
+// After walk_code: scale this thread's point to the unit sphere times `amp` and write its N
+// values as bf16 with 16-byte stores (row `row`, group `g` of matrix m).  Each thread writes
+// its own N*2 contiguous bytes; the threads of a warp hold consecutive groups, so a warp
+// fills a contiguous stretch of the row.
 template <int N, typename YT>
-__device__ __forceinline__ void emit_tile(const MatrixArgs& m, uint8_t* wbuf, float* wscale, int lane, float amp,
-                                          long long g0, long long ngroups) {
-    constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
+__device__ __forceinline__ void emit_group(const MatrixArgs& m, const YT* yslots, float amp, unsigned row,
+                                           unsigned g) {
+    const uint32_t* y4 = reinterpret_cast<const uint32_t*>(yslots);
     int ssy = 0;
     if constexpr (sizeof(YT) == 1) {
         // slots hold b = y + 128:  sum y^2 = sum b^2 - 256 sum b + 128^2 N
-        const unsigned* y4 = reinterpret_cast<const unsigned*>(wbuf + lane * YS);
         unsigned sq = 0, su = 0;
 #pragma unroll
         for (int v = 0; v < N / 4; ++v) {
@@ -423,66 +422,34 @@ __device__ __forceinline__ void emit_tile(const MatrixArgs& m, uint8_t* wbuf, fl
         }
         ssy = static_cast<int>(sq) - 256 * static_cast<int>(su) + 16384 * N;
     } else {
-        const YT* yslots = reinterpret_cast<const YT*>(wbuf + lane * YS);
 #pragma unroll 8
         for (int v = 0; v < N; ++v) ssy += static_cast<int>(yslots[v]) * static_cast<int>(yslots[v]);
     }
-    wscale[lane] = __fdiv_rn(amp, __fsqrt_rn(static_cast<float>(ssy)));
-    __syncwarp();
-
-    constexpr int TPG = N / 8;     // threads per group, 16 bytes each
-    constexpr int GPI = 32 / TPG;  // groups per iteration
-    const int part = lane % TPG;
-    // row and group-in-row of the tile's first group; the tile's other groups follow from it
-    // without a division as long as they sit in that row or the next
-    const unsigned G = static_cast<unsigned>(m.G);
-    const unsigned row0 = static_cast<unsigned>(g0) / G;
-    const unsigned off0 = static_cast<unsigned>(g0) - row0 * G;
-#pragma unroll 1
-    for (int it = 0; it < TPG; ++it) {
-        const int gl = it * GPI + lane / TPG;  // group within the tile
-        const long long gj = g0 + gl;
-        if (gj < ngroups) {
-            const uint8_t* ys = wbuf + gl * YS + part * 8 * sizeof(YT);
-            const float sc = wscale[gl];
-            float f[8];
-            if constexpr (sizeof(YT) == 1) {
-                // byte b into the low mantissa bits of 2^23: the float 2^23 + b, then minus 2^23 + 128
-                const uint32_t lo = reinterpret_cast<const uint32_t*>(ys)[0];
-                const uint32_t hi = reinterpret_cast<const uint32_t*>(ys)[1];
+    const float sc = __fdiv_rn(amp, __fsqrt_rn(static_cast<float>(ssy)));
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.out) + static_cast<size_t>(row) * m.ld_out +
+                                          static_cast<size_t>(g) * N);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    f[e] = __fsub_rn(__uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7540u + e)), 8388736.0f);
-                    f[4 + e] = __fsub_rn(__uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7540u + e)), 8388736.0f);
-                }
-            } else {
-                const YT* yv = reinterpret_cast<const YT*>(ys);
+    for (int q = 0; q < N / 8; ++q) {
+        float f[8];
+        if constexpr (sizeof(YT) == 1) {
+            // byte b into the low mantissa bits of 2^23: the float 2^23 + b, then minus 2^23 + 128
+            const uint32_t lo = y4[2 * q], hi = y4[2 * q + 1];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = static_cast<float>(static_cast<int>(yv[e]));
+            for (int e = 0; e < 4; ++e) {
+                f[e] = __fsub_rn(__uint_as_float(__byte_perm(lo, 0x4B000000u, 0x7540u + e)), 8388736.0f);
+                f[4 + e] = __fsub_rn(__uint_as_float(__byte_perm(hi, 0x4B000000u, 0x7540u + e)), 8388736.0f);
             }
-            unsigned g = off0 + static_cast<unsigned>(gl);
-            unsigned row = row0;
-            if (g >= G) {
-                g -= G;
-                row += 1;
-                if (g >= G) {  // rows shorter than a tile
-                    const unsigned q = g / G;
-                    row += q;
-                    g -= q * G;
-                }
-            }
-            uint4 o;
-            o.x = pack_bf16x2(__fmul_rn(f[0], sc), __fmul_rn(f[1], sc));
-            o.y = pack_bf16x2(__fmul_rn(f[2], sc), __fmul_rn(f[3], sc));
-            o.z = pack_bf16x2(__fmul_rn(f[4], sc), __fmul_rn(f[5], sc));
-            o.w = pack_bf16x2(__fmul_rn(f[6], sc), __fmul_rn(f[7], sc));
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.out) +
-                                                  static_cast<size_t>(row) * m.ld_out +
-                                                  static_cast<size_t>(g) * N + part * 8);
-            *dst = o;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = static_cast<float>(static_cast<int>(yslots[8 * q + e]));
         }
+        uint4 o;
+        o.x = pack_bf16x2(__fmul_rn(f[0], sc), __fmul_rn(f[1], sc));
+        o.y = pack_bf16x2(__fmul_rn(f[2], sc), __fmul_rn(f[3], sc));
+        o.z = pack_bf16x2(__fmul_rn(f[4], sc), __fmul_rn(f[5], sc));
+        o.w = pack_bf16x2(__fmul_rn(f[6], sc), __fmul_rn(f[7], sc));
+        dst[q] = o;
     }
-    __syncwarp();  // the slots are rewritten by the next tile
 }
 
 }  // namespace pvq
