@@ -34,6 +34,15 @@ if ROOT not in sys.path:
 L2_BYTES = 126 * 1024 * 1024
 FALLBACK_HBM_GBS = 6650.0
 
+# Per-launch counters of the kernels from the ncu captures summarised under profiles/ (same
+# workload and launch configuration as this bench): DRAM bytes read + written, and warp
+# instructions executed.  Set an entry to None when its kernel changes until it is re-captured.
+NCU_COUNTERS = {
+    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_668_352 + 774_144, "warp_inst": 32_381_488},
+    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_651_648 + 1_280, "warp_inst": 40_036_062},
+}
+SMS, SCHEDULERS_PER_SM = 148, 4      # issue slots per cycle on the part = SMS * SCHEDULERS_PER_SM
+
 
 def log(*a):
     print(*a, file=sys.stderr, flush=True)
@@ -406,9 +415,23 @@ def main():
                          "frac_of_%s_hbm" % peak_kind: nbytes / (avg * 1e-3) / 1e9 / peak,
                          "frac_of_nominal_8TBps": nbytes / (avg * 1e-3) / 1e9 / 8000.0}
     dom = max(kernels, key=lambda k: kernels[k]["avg_ms"])
+    ncu = NCU_COUNTERS.get((wl.name, dom))
     roofline = {"kernel": "pvq %s_kernel" % dom, "bound": "hbm", "achieved": kernels[dom]["GBps"], "peak": peak,
                 "peak_source": "%s (MEASURED_PEAKS.json hbm_gbs)" % peak_kind if peak_kind == "measured"
-                else "fallback", "unit": "GB/s", "frac": kernels[dom]["GBps"] / peak, "traffic": None}
+                else "fallback", "unit": "GB/s", "frac": kernels[dom]["GBps"] / peak,
+                "traffic": ncu["dram_bytes"] if ncu else None}
+    # The limit that binds in practice: instruction issue (every kernel here is integer work
+    # on a table walk).  achieved = ncu's warp instructions per launch / measured time,
+    # peak = issue slots per second at the SM clock sampled during the run.
+    issue = {}
+    for name in kernels:
+        c = NCU_COUNTERS.get((wl.name, name))
+        mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz")
+        if c and mhz:
+            ach = c["warp_inst"] / (kernels[name]["avg_ms"] * 1e-3)
+            pk = SMS * SCHEDULERS_PER_SM * mhz * 1e6
+            issue[name] = {"bound": "alu", "achieved": ach / 1e9, "peak": pk / 1e9, "unit": "Gwarp-inst/s",
+                           "frac": ach / pk, "warp_inst_per_weight": c["warp_inst"] / wl.weights}
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -419,7 +442,7 @@ def main():
             "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u32+f32", "data": "synthetic",
             "config": config, "Gweights_per_s": wl.weights * args.steps * world / (total_ms * 1e-3) / 1e9,
-            "kernels": kernels, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
+            "kernels": kernels, "roofline": roofline, "issue": issue, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
             "gpu_launches": len(per) * args.steps}
     print(json.dumps(line))
     if world > 1:

@@ -186,7 +186,7 @@ int pvq_decode_batched(const pvq_matrix_desc* descs, int count, int N, int K, in
 /* ---- for callers that cannot allocate device memory ---------------------------------- */
 
 /* Size of the count table that is built into the library image (see below). */
-#define PVQ_STATIC_TABLE_BYTES (384u * 1024u)
+#define PVQ_STATIC_TABLE_BYTES (1024u * 1024u)
 
 /* pvq_decode without a caller-provided count table.  (The paper has no counterpart: this
  * is a packaging variant of pvq_decode, with identical results.)
