@@ -38,8 +38,9 @@ FALLBACK_HBM_GBS = 6650.0
 # workload and launch configuration as this bench): DRAM bytes read + written, and warp
 # instructions executed.  Set an entry to None when its kernel changes until it is re-captured.
 NCU_COUNTERS = {
-    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_668_352 + 774_144, "warp_inst": 32_381_488},
-    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_651_648 + 1_280, "warp_inst": 40_036_062},
+    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_967_104 + 5_376, "warp_inst": 32_381_488},
+    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_651_136 + 5_120, "warp_inst": 40_036_062},
+    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_499_584 + 89_775_872, "warp_inst": 218_715_576},
 }
 SMS, SCHEDULERS_PER_SM = 148, 4      # issue slots per cycle on the part = SMS * SCHEDULERS_PER_SM
 
@@ -323,7 +324,7 @@ def oracle_sample(wl, target_seconds=12.0):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

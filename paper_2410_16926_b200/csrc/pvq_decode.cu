@@ -112,7 +112,7 @@ int launch_decode_t(BatchArgs& a, cudaStream_t stream) {
     int threads = kDecThreads;
     int phases = 0;
     size_t smem = 0;
-    for (; threads >= 128; threads /= 2) {
+    for (; threads >= 128; threads -= 32) {
         const size_t wbufs = static_cast<size_t>(threads) * YS;
         phases = walk_phases_that_fit(L, static_cast<size_t>(smem_max) - std::min<size_t>(smem_max, wbufs));
         if (phases) {

@@ -283,6 +283,59 @@ __device__ __forceinline__ void walk_step_w4(mp<4>& r, uint32_t& p, int& v, uint
         : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 16), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
+// Widest phase for 5- and 6-word codes (24-byte entries; a 5-word code walks with a zero
+// sixth word).
+template <typename YT, int U>
+__device__ __forceinline__ void walk_step_w6(uint32_t (&r)[6], uint32_t& p, int& v, uint32_t& y, const int D,
+                                             const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, t2, t3, t4, t5, a0, a1, a2, a3, a4, a5, ab, b0, b1, b2, b3, b4, b5, bb, ob, val;\n\t"
+        "ld.shared.v2.u32 {t0, t1}, [%8+%12];\n\t"
+        "ld.shared.v2.u32 {t2, t3}, [%8+%13];\n\t"
+        "ld.shared.v2.u32 {t4, t5}, [%8+%14];\n\t"
+        "sub.cc.u32 a0, %0, t0;\n\t"
+        "subc.cc.u32 a1, %1, t1;\n\t"
+        "subc.cc.u32 a2, %2, t2;\n\t"
+        "subc.cc.u32 a3, %3, t3;\n\t"
+        "subc.cc.u32 a4, %4, t4;\n\t"
+        "subc.cc.u32 a5, %5, t5;\n\t"
+        "subc.u32 ab, 0, 0;\n\t"
+        "sub.cc.u32 b0, a0, t0;\n\t"
+        "subc.cc.u32 b1, a1, t1;\n\t"
+        "subc.cc.u32 b2, a2, t2;\n\t"
+        "subc.cc.u32 b3, a3, t3;\n\t"
+        "subc.cc.u32 b4, a4, t4;\n\t"
+        "subc.cc.u32 b5, a5, t5;\n\t"
+        "subc.u32 bb, 0, 0;\n\t"
+        PVQ_WIDE_TAIL(6, 0)
+        "@g1 mad.lo.u32 %0, a0, %9, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %9, 0;\n\t"
+        "@g1 mad.lo.u32 %2, a2, %9, 0;\n\t"
+        "@g1 mad.lo.u32 %3, a3, %9, 0;\n\t"
+        "@g1 mad.lo.u32 %4, a4, %9, 0;\n\t"
+        "@g1 mad.lo.u32 %5, a5, %9, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %9, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %9, 0;\n\t"
+        "@m2 mad.lo.u32 %2, b2, %9, 0;\n\t"
+        "@m2 mad.lo.u32 %3, b3, %9, 0;\n\t"
+        "@m2 mad.lo.u32 %4, b4, %9, 0;\n\t"
+        "@m2 mad.lo.u32 %5, b5, %9, 0;\n\t"
+        "mad.lo.u32 val, %6, %9, %17;\n\t"
+        "@ng mad.lo.u32 val, %6, %10, %17;\n\t"
+        "st.shared.u%16 [%7], val;\n\t"
+        "@!mo add.u32 %7, %7, %15;\n\t"
+        "@!mo add.u32 %8, %8, %11;\n\t"
+        "mad.lo.u32 %6, %6, %9, %9;\n\t"
+        "@!mo mov.u32 %6, 0;\n\t"
+        "}"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 24), "n"(-U * 24 + 8), "n"(-U * 24 + 16), "n"(SZ),
+          "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
 #undef PVQ_WIDE_TAIL
 
 template <int PW, int EB, bool HEADROOM, typename YT, int U>
@@ -296,7 +349,14 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
         walk_step_w3<YT, U>(r, p, v, y, D, f);
     else if constexpr (!HEADROOM && PW == 4)
         walk_step_w4<YT, U>(r, p, v, y, D, f);
-    else
+    else if constexpr (!HEADROOM && PW == 6)
+        walk_step_w6<YT, U>(r.w, p, v, y, D, f);
+    else if constexpr (!HEADROOM && PW == 5) {
+        uint32_t r6[6] = {r.w[0], r.w[1], r.w[2], r.w[3], r.w[4], 0u};
+        walk_step_w6<YT, U>(r6, p, v, y, D, f);
+#pragma unroll
+        for (int w = 0; w < 5; ++w) r.w[w] = r6[w];
+    } else
         walk_step_wide<PW, EB, YT, U>(r, p, v, y, D);
 }
 
