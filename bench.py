@@ -319,6 +319,25 @@ def oracle_sample(wl, target_seconds=12.0):
     return nb / t / 1e9, po.threads(), "first %s rows of each matrix, %.1f s" % (rows, t), nb, t
 
 
+# ----------------------------------------------------------------- over the ranks
+
+def max_over_ranks(value, world, device=None):
+    """The slowest rank's time: what every multi-GPU number is divided by."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(step_bytes, steps, world, total_ms):
+    """GB/s of the whole job: every rank runs its own replica of the workload (rows shard with no
+    exchange), so the bytes add up over the ranks and the time is the slowest rank's."""
+    return step_bytes * steps * world / (total_ms * 1e-3) / 1e9
+
+
 # --------------------------------------------------------------------------- main
 
 def main():
@@ -384,21 +403,15 @@ def main():
     total_ms, per = run.run(args.steps, warmup)
     barrier()
     clocks = sampler.stop()
-    if world > 1:
-        t = torch.tensor([total_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    value = step_bytes * args.steps * world / (total_ms * 1e-3) / 1e9
+    total_ms = max_over_ranks(total_ms, world, device)
+    value = whole_job_value(step_bytes, args.steps, world, total_ms)
 
     e2e = None
     if not args.no_e2e:
         e_steps = max(3, min(args.steps, 20))
         ms, h2d, d2h = run.run_e2e(e_steps, 3)
-        if world > 1:
-            t = torch.tensor([ms], device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": step_bytes * world / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms,
+        ms = max_over_ranks(ms, world, device)
+        e2e = {"value": whole_job_value(step_bytes, 1, world, ms), "unit": "GB/s", "ms_per_step": ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank != 0:
