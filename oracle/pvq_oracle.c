@@ -16,6 +16,8 @@
  *   amplitude          Sec. 2.3 (amplitude = ||w||_2), Sec. 3.3 Step 5 and
  *                      Sec. 3.4 (quantile quantiser on s_g^2 / ||s||^2)
  *   reconstruction     Sec. 2.4 (projection of the pyramid point on the sphere)
+ *   rotation           Sec. 2.3 "Hadamard coherence processing" / Sec. 3.3 Step 1, along
+ *                      the input dimension: x <- (x * s) H_n / sqrt(n) per block of n
  *
  * Integers are multi-word unsigned numbers kept as little-endian arrays of
  * 32-bit limbs and handled one limb at a time with a 64-bit carry.
@@ -550,6 +552,49 @@ int pvqo_decode(const uint32_t *codes, const uint8_t *scale_idx, const float *ro
     }
     free(t);
     if (status) *status |= bad;
+    return 0;
+}
+
+/* ------------------------------------------------ rotation (Sec. 2.3, Step 1) */
+
+/*
+ * Random-sign Hadamard rotation along the columns, independently on every
+ * contiguous block of `block` columns of every row (block a power of two
+ * dividing cols): with s the +-1 sign vector of length `block` (shared by all
+ * blocks and rows) and H the Sylvester-Walsh-Hadamard matrix,
+ *     out = (x * s) H / sqrt(block).
+ * H is applied as log2(block) stages of butterflies with strides 1, 2, 4, ...:
+ * (a, b) -> (a + b, a - b) on elements j and j + stride, each sum rounded to
+ * binary32; the scale is the binary32 nearest to 1/sqrt(block), applied last
+ * with one multiplication.  That order is a convention of this build (parity
+ * unpinned by the paper); the result is pinned to H by exact cases.
+ * dtype 0 = fp32 in, 1 = bf16 in; out is fp32 [rows][cols].
+ */
+int pvqo_rotate(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld, int block,
+                const float *signs, float *out) {
+    if (block < 1 || (block & (block - 1)) || cols % block) return -1;
+    float scale = (float)(1.0 / sqrt((double)block));
+    for (int64_t r = 0; r < rows; ++r) {
+        float *o = out + r * cols;
+        for (int64_t c = 0; c < cols; ++c) {
+            float v = dtype == 0 ? ((const float *)x)[r * ld + c]
+                                 : bf16_to_f32(((const uint16_t *)x)[r * ld + c]);
+            o[c] = v * signs[c % block];
+        }
+        for (int64_t b0 = 0; b0 < cols; b0 += block) {
+            float *v = o + b0;
+            for (int h = 1; h < block; h <<= 1) {
+                for (int j0 = 0; j0 < block; j0 += 2 * h) {
+                    for (int j = j0; j < j0 + h; ++j) {
+                        float a = v[j], b = v[j + h];
+                        v[j] = a + b;
+                        v[j + h] = a - b;
+                    }
+                }
+            }
+            for (int j = 0; j < block; ++j) v[j] = v[j] * scale;
+        }
+    }
     return 0;
 }
 

@@ -33,6 +33,7 @@ def lib():
         L.pvqo_scale_row_stride.restype = C.c_size_t
         L.pvqo_encode.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, vp, i32]
         L.pvqo_decode.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, i32, vp, vp, i64, vp, i32]
+        L.pvqo_rotate.argtypes = [vp, i32, i64, i64, i64, i32, vp, vp]
         L.pvqo_threads.argtypes = []
         _lib = L
     return _lib
@@ -155,6 +156,19 @@ def decode(codes: np.ndarray, sidx: np.ndarray, rnorm: np.ndarray, N: int, K: in
     if rc != 0:
         raise ValueError("oracle decode rejected its arguments")
     return out, int(status[0])
+
+
+def rotate(x: np.ndarray, block: int, signs: np.ndarray) -> np.ndarray:
+    """Random-sign Hadamard rotation along the columns (Sec. 2.3 / Step 1): float32 [rows][cols]."""
+    assert x.ndim == 2 and x.flags.c_contiguous
+    dtype = 0 if x.dtype == np.float32 else 1
+    assert x.dtype in (np.float32, np.uint16)
+    signs = np.ascontiguousarray(signs, dtype=np.float32)
+    assert signs.size == block
+    out = np.zeros(x.shape, dtype=np.float32)
+    if lib().pvqo_rotate(_p(x), dtype, x.shape[0], x.shape[1], x.shape[1], block, _p(signs), _p(out)) != 0:
+        raise ValueError("oracle rotate rejected its arguments")
+    return out
 
 
 def unpack_scale_idx(sidx: np.ndarray, G: int, scale_bits: int) -> np.ndarray:

@@ -508,3 +508,53 @@ def test_zero_row_and_invalid_code():
     codes[2, 1, 0] = pr.count(N, K)       # first invalid value
     out_bits, status = po.decode(codes, sidx, rnorm, N, K, b, amp)
     assert status == 1 and np.all(out_bits[2, 8:16] == 0) and np.any(out_bits[2, :8] != 0)
+
+
+# ------------------------------------------------------------ rotation (Sec. 2.3, Step 1)
+
+def _hadamard(n):
+    h = np.array([[1.0]])
+    while h.shape[0] < n:
+        h = np.block([[h, h], [h, -h]])
+    return h
+
+
+@pytest.mark.parametrize("block,cols", [(4, 12), (16, 16), (64, 128), (256, 512)])
+def test_rotation_is_the_hadamard_matrix_exactly_on_small_integers(block, cols):
+    # power-of-four blocks scale by a power of two and small integers add without rounding:
+    # the butterflies must then equal the matrix product bit for bit
+    rng = np.random.default_rng(block)
+    x = rng.integers(-8, 9, size=(5, cols)).astype(np.float32)
+    s = (rng.integers(0, 2, size=block) * 2 - 1).astype(np.float32)
+    got = po.rotate(x, block, s)
+    xs = (x.reshape(5, cols // block, block) * s).astype(np.float64)
+    want = (xs @ _hadamard(block)) / np.sqrt(block)
+    assert np.array_equal(got.astype(np.float64), want.reshape(5, cols))
+
+
+@pytest.mark.parametrize("block", [8, 32, 512])
+def test_rotation_against_the_matrix_for_irrational_scales(block):
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((3, 2 * block)).astype(np.float32)
+    s = (rng.integers(0, 2, size=block) * 2 - 1).astype(np.float32)
+    got = po.rotate(x, block, s).astype(np.float64)
+    want = ((x.reshape(3, 2, block) * s).astype(np.float64) @ _hadamard(block) / np.sqrt(block)).reshape(3, -1)
+    assert np.max(np.abs(got - want)) < 1e-5 * np.sqrt(block)
+    # orthogonal: norms are kept
+    assert np.allclose(np.linalg.norm(got, axis=1), np.linalg.norm(x.astype(np.float64), axis=1), rtol=1e-5)
+
+
+def test_rotation_twice_without_signs_is_the_identity():
+    rng = np.random.default_rng(3)
+    x = rng.integers(-20, 21, size=(4, 64)).astype(np.float32)
+    ones = np.ones(16, dtype=np.float32)
+    assert np.array_equal(po.rotate(po.rotate(x, 16, ones), 16, ones), x)      # H H = n I, exact here
+
+
+def test_rotation_of_bf16_input_widens_exactly():
+    from paper_2410_16926_b200 import inputs
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((2, 64)).astype(np.float32)
+    xb = inputs.f32_to_bf16_bits(x)
+    s = np.ones(64, dtype=np.float32)
+    assert np.array_equal(po.rotate(xb, 64, s), po.rotate(inputs.bf16_bits_to_f32(xb), 64, s))
