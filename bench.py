@@ -88,7 +88,7 @@ def algorithmic_bytes(wl, direction):
 def make_workload(name):
     from paper_2410_16926_b200 import inputs
     return {"c1": inputs.config1, "c2": inputs.config2, "c3": inputs.config3, "c4": inputs.config4,
-            "c5": inputs.config5}[name]()
+            "c5": inputs.config5, "c5r": inputs.config5_unrotated}[name]()
 
 
 # ------------------------------------------------------------------------ clocks
@@ -155,6 +155,7 @@ class GpuRun:
         self.K = pvq.max_pulses(N, wl.index_bits)
         self.W = pvq.code_words(N, self.K)
         self.table = pvq.build_count_table(N, self.K, device)
+        self.signs = torch.from_numpy(wl.signs).to(device) if wl.signs is not None else None
         self.books = {}
         for m in wl.matrices:
             G = m.cols // N
@@ -197,10 +198,16 @@ class GpuRun:
         self.pvq.roundtrip(it["x"], self.wl.N, self.K, self.wl.scale_bits, self.table, it["edges"],
                            it["levels"], out=it["out"])
 
+    def fused_rotate(self, items):
+        it = items[0]
+        self.pvq.rotate_roundtrip(it["x"], self.wl.rot_block, self.signs, self.wl.N, self.K, self.wl.scale_bits,
+                                  self.table, it["edges"], it["levels"], out=it["out"])
+
     def phases(self):
         return {"encode+decode": [("encode", self.encode), ("decode", self.decode)],
                 "decode": [("decode", self.decode)],
-                "roundtrip": [("roundtrip", self.fused)]}[self.wl.mode]
+                "roundtrip": [("roundtrip", self.fused)],
+                "rotate_roundtrip": [("rotate_roundtrip", self.fused_rotate)]}[self.wl.mode]
 
     def run(self, steps, warmup):
         """Returns (total_ms, {phase: [ms per launch]}) timed with CUDA events on the launch stream."""
@@ -237,7 +244,7 @@ class GpuRun:
         def step():
             nonlocal h2d, d2h
             h2d = d2h = 0
-            if wl.mode in ("encode+decode", "roundtrip"):
+            if wl.mode in ("encode+decode", "roundtrip", "rotate_roundtrip"):
                 for it, h in zip(items, self.host):
                     it["x"].copy_(h, non_blocking=True)
                     h2d += h.numel() * h.element_size()
@@ -301,13 +308,15 @@ def oracle_sample(wl, target_seconds=12.0):
             e_np, l_np = books[m.cols // N]
             comp = compressed_bytes(rows, m.cols, N, wl.index_bits, b)
             t0 = time.perf_counter()
+            if wl.mode == "rotate_roundtrip":
+                x = po.rotate(x, wl.rot_block, wl.signs)
             enc = po.encode(x, N, K, b, e_np, W=W)
             if wl.mode != "decode":
-                nbytes += x.nbytes + (comp if wl.mode == "encode+decode" else 0)
+                nbytes += rows * m.cols * (4 if m.dtype == "f32" else 2) + (comp if wl.mode == "encode+decode" else 0)
             t1 = time.perf_counter()
             po.decode(*enc, N, K, b, l_np)
             t2 = time.perf_counter()
-            nbytes += rows * m.cols * 2 + (comp if wl.mode != "roundtrip" else 0)
+            nbytes += rows * m.cols * 2 + (comp if wl.mode in ("encode+decode", "decode") else 0)
             t += (t2 - t1) if wl.mode == "decode" else (t2 - t0)
         return nbytes, t
 
@@ -345,7 +354,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c5r"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -357,7 +366,8 @@ def main():
 
     wl = make_workload(args.config)
     metric = "pvq_%s_throughput" % wl.mode.replace("+", "_")
-    dirs = {"encode+decode": ["encode", "decode"], "decode": ["decode"], "roundtrip": ["roundtrip"]}[wl.mode]
+    dirs = {"encode+decode": ["encode", "decode"], "decode": ["decode"], "roundtrip": ["roundtrip"],
+            "rotate_roundtrip": ["rotate_roundtrip"]}[wl.mode]
     step_bytes = sum(algorithmic_bytes(wl, d) for d in dirs)
     config = {"workload": wl.name, "matrices": [[m.name, m.rows, m.cols, m.dtype] for m in wl.matrices],
               "N": wl.N, "index_bits": wl.index_bits, "scale_bits": wl.scale_bits, "mode": wl.mode,

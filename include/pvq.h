@@ -161,6 +161,27 @@ int pvq_roundtrip(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_
                   int scale_bits, const uint32_t* d_table, const float* d_edges,
                   const float* d_levels, void* d_out, int64_t ld_out, pvq_stream_t stream);
 
+/* Rotation on the fly (Sec. 2.3 "Hadamard coherence processing", Sec. 3.3 Step 1, along the
+ * input dimension; Sec. 4.3 for activations, which have to be rotated at run time): every
+ * row is multiplied elementwise by the signs d_signs[col % block] (+-1 as float, `block` of
+ * them) and every contiguous run of `block` columns by H_block / sqrt(block), H the
+ * Sylvester-Walsh-Hadamard matrix; the rotated row is then encoded (pvq_rotate_encode) or
+ * encoded and decoded (pvq_rotate_roundtrip) exactly as by pvq_encode / pvq_roundtrip on fp32
+ * input, without the rotated matrix ever being written to memory.
+ *   block      a power of two, a multiple of N, dividing cols, at most 16384.
+ * Arithmetic: fp32; the sign flip, then butterflies (a, b) -> (a + b, a - b) with strides
+ * 1, 2, 4, ..., block/2, one rounding each, then one multiplication by the fp32 nearest to
+ * 1/sqrt(block).  The other arguments are those of pvq_encode / pvq_roundtrip; the fused form
+ * needs K <= 127. */
+int pvq_rotate_encode(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int block,
+                      const float* d_signs, int N, int K, int scale_bits, const uint32_t* d_table,
+                      const float* d_edges, uint32_t* d_codes, uint8_t* d_scale_idx, float* d_row_norm,
+                      pvq_stream_t stream);
+int pvq_rotate_roundtrip(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int block,
+                         const float* d_signs, int N, int K, int scale_bits, const uint32_t* d_table,
+                         const float* d_edges, const float* d_levels, void* d_out, int64_t ld_out,
+                         pvq_stream_t stream);
+
 /* One matrix of a batched call.  Pointers are device pointers with the meaning and
  * alignment of the corresponding pvq_encode / pvq_decode arguments; d_edges / d_levels
  * belong to this matrix's G. */

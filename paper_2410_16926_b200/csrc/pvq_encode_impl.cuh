@@ -295,7 +295,59 @@ struct EncodeSmem {
     int idx_words;        // per buffer (there are two)
     int enum_mode;        // 2: U and 2V staged, 1: V only, 0: none (fused: the walk table serves)
     int walk_phases;
+    uint32_t signs_off;   // rotation: rot_block floats
+    uint32_t xbuf_off;    // rotation across more than a warp: threads * N floats
 };
+
+// Random-sign Hadamard rotation of a row tile held one group per thread (Sec. 2.3, Sec. 3.3
+// Step 1): x <- (x * s) H_B / sqrt(B) on every block of B = N * T consecutive columns.  The
+// Sylvester butterflies (a, b) -> (a + b, a - b) run with strides 1, 2, 4, ...: strides below
+// N inside the thread, strides N .. 16 N between threads of a warp by shuffle (T divides G,
+// so thread t and its partner t ^ d hold groups of the same block), larger ones through
+// shared memory.  Every sum is one fp32 addition, so the result does not depend on which of
+// these three ways a stage takes.
+template <int N>
+__device__ __forceinline__ void rotate_tile(float (&x)[N], const float* s_signs, int block, float scale,
+                                            int g, float* xbuf, int tid, int nthreads) {
+    const int col0 = (g * N) & (block - 1);
+#pragma unroll
+    for (int i = 0; i < N; ++i) x[i] = __fmul_rn(x[i], s_signs[col0 + i]);
+#pragma unroll
+    for (int h = 1; h < N; h <<= 1) {
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            if ((j & h) == 0) {
+                const float a = x[j], b2 = x[j + h];
+                x[j] = __fadd_rn(a, b2);
+                x[j + h] = __fsub_rn(a, b2);
+            }
+        }
+    }
+    const int T = block / N;  // threads per rotation block
+    for (int d = 1; d < T && d < 32; d <<= 1) {
+        const bool upper = (tid & d) != 0;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const float other = __shfl_xor_sync(kFull, x[i], d);
+            x[i] = upper ? __fsub_rn(other, x[i]) : __fadd_rn(x[i], other);
+        }
+    }
+    for (int d = 32; d < T; d <<= 1) {
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < N; ++i) xbuf[i * nthreads + tid] = x[i];
+        __syncthreads();
+        const bool upper = (tid & d) != 0;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const float other = xbuf[i * nthreads + (tid ^ d)];
+            x[i] = upper ? __fsub_rn(other, x[i]) : __fadd_rn(x[i], other);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) x[i] = __fmul_rn(x[i], scale);
+}
+
 
 // Where a thread works in a tile.
 struct TileLoc {
@@ -326,18 +378,30 @@ __device__ __forceinline__ TileLoc locate(const BatchArgs& a, unsigned tile) {
 // The two ss / scale-index buffers alternate between consecutive tiles, which leaves three
 // block-wide barriers per tile (two in the fused kernel); the input of the next tile is
 // requested as soon as the registers that held this tile's input are free.
-template <int N, int W, bool FUSED, typename YT, bool BF16>
+//
+// ROT: the tile is first rotated (rotate_tile); the kernel then works on the rotated fp32
+// values, whatever type the input has.
+template <int N, int W, bool FUSED, typename YT, bool BF16, bool ROT>
 __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ BatchArgs a,
                                                       const __grid_constant__ EncodeSmem sm) {
     extern __shared__ __align__(16) uint8_t smem[];
     constexpr int TW = W <= 2 ? W : (W <= 4 ? 4 : 6);
     constexpr int EB = TW * 4;
     constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
-    constexpr int RW = BF16 ? N / 2 : N;
+    constexpr int RW = BF16 ? N / 2 : N;      // words of a group as loaded
+    constexpr bool WBF16 = BF16 && !ROT;       // the form the kernel works on: packed bf16, or fp32
+    constexpr int WW = WBF16 ? N / 2 : N;
     const int K = a.K;
     const int b = a.scale_bits;
     const int nedges = (1 << b) - 1;
     const TableLayout L = table_layout(N, K, W);
+    float* s_signs = reinterpret_cast<float*>(smem + sm.signs_off);
+    float* s_xbuf = reinterpret_cast<float*>(smem + sm.xbuf_off);
+    float rot_scale = 1.0f;
+    if constexpr (ROT) {
+        for (int i = threadIdx.x; i < a.rot_block; i += blockDim.x) s_signs[i] = a.rot_signs[i];
+        rot_scale = static_cast<float>(1.0 / sqrt(static_cast<double>(a.rot_block)));
+    }
     float* s_ss2 = reinterpret_cast<float*>(smem + sm.ss_off);
     float* s_edges = reinterpret_cast<float*>(smem + sm.edges_off);
     float* s_levels = reinterpret_cast<float*>(smem + sm.levels_off);
@@ -372,12 +436,12 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     unsigned tile = blockIdx.x;
     if (tile >= a.total_tiles) return;
     TileLoc loc = locate(a, tile);
-    uint32_t raw[RW];
+    uint32_t pre[RW];  // the group as loaded; filled one tile ahead
 #pragma unroll
-    for (int i = 0; i < RW; ++i) raw[i] = 0u;
+    for (int i = 0; i < RW; ++i) pre[i] = 0u;
     if (loc.active) {
         const MatrixArgs& m0 = a.m[loc.mi];
-        load_raw<N, BF16>(m0.x, static_cast<size_t>(loc.row0 + loc.rl) * m0.ld + static_cast<size_t>(loc.g) * N, raw);
+        load_raw<N, BF16>(m0.x, static_cast<size_t>(loc.row0 + loc.rl) * m0.ld + static_cast<size_t>(loc.g) * N, pre);
     }
     __syncthreads();  // tables staged, index words cleared
 
@@ -391,16 +455,29 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
         float* s_ss = s_ss2 + buf * sm.ss_floats;
         uint32_t* s_idx = s_idx2 + buf * sm.idx_words;
 
+        uint32_t raw[WW];  // the group the kernel works on
+        if constexpr (ROT) {
+            float x[N];
+#pragma unroll
+            for (int i = 0; i < N; ++i) x[i] = raw_value<N, BF16>(pre, i);
+            rotate_tile<N>(x, s_signs, a.rot_block, rot_scale, g, s_xbuf, threadIdx.x, blockDim.x);
+#pragma unroll
+            for (int i = 0; i < N; ++i) raw[i] = __float_as_uint(x[i]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < WW; ++i) raw[i] = pre[i];
+        }
+
         // group norms; an inactive thread holds zeros
         float l1, ss;
         {
             float t[N];
 #pragma unroll
-            for (int i = 0; i < N; ++i) t[i] = fabsf(raw_value<N, BF16>(raw, i));
+            for (int i = 0; i < N; ++i) t[i] = fabsf(raw_value<N, WBF16>(raw, i));
             l1 = tree_sum<N>(t);
 #pragma unroll
             for (int i = 0; i < N; ++i) {
-                const float xi = raw_value<N, BF16>(raw, i);
+                const float xi = raw_value<N, WBF16>(raw, i);
                 t[i] = __fmul_rn(xi, xi);
             }
             ss = tree_sum<N>(t);
@@ -432,14 +509,14 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
 
         // direction; nothing here needs the row norm.  mag[i] carries the sign of x_i.
         float mag[N];
-        const bool has_dir = quantize_direction<N, BF16>(raw, l1, K, mag);
+        const bool has_dir = quantize_direction<N, WBF16>(raw, l1, K, mag);
         if (!has_dir) {  // (K, 0, ..., 0)
 #pragma unroll
             for (int i = 0; i < N; ++i) mag[i] = kMagic;
             mag[0] = __int_as_float(kMagicBits + K);
         }
 
-        // raw is dead: ask for the next tile's input now, it arrives while the index is computed
+        // the loaded group is dead: ask for the next tile's input now, it arrives while the index is computed
         const unsigned next_tile = tile + gridDim.x;
         const bool have_next = next_tile < a.total_tiles;
         TileLoc nloc = loc;
@@ -448,10 +525,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             if (nloc.active) {
                 const MatrixArgs& mn = a.m[nloc.mi];
                 load_raw<N, BF16>(mn.x, static_cast<size_t>(nloc.row0 + nloc.rl) * mn.ld + static_cast<size_t>(nloc.g) * N,
-                                  raw);
+                                  pre);
             } else {
 #pragma unroll
-                for (int i = 0; i < RW; ++i) raw[i] = 0u;
+                for (int i = 0; i < RW; ++i) pre[i] = 0u;
             }
         }
 
@@ -520,7 +597,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     }
 }
 
-template <int N, int W, bool FUSED, typename YT, bool BF16>
+template <int N, int W, bool FUSED, typename YT, bool BF16, bool ROT>
 static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
     // Block size: a multiple of 32 that wastes the fewest thread slots over the batch.
@@ -570,7 +647,11 @@ static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     const int sms = di.sms, smem_max = di.smem_max;
 
     const TableLayout L = table_layout(N, a.K, W);
-    const size_t small = (2 * static_cast<size_t>(ss_floats) + 256 + (FUSED ? 256 : 0) + 2 * max_idx_words) * 4u + 64u;
+    // rotation: the signs, and an exchange buffer when a rotation block spans more than a warp
+    const size_t rot_signs_b = ROT ? static_cast<size_t>(a.rot_block) * 4u : 0;
+    const size_t rot_xbuf_b = ROT && a.rot_block / N > 32 ? static_cast<size_t>(threads) * N * 4u : 0;
+    const size_t small = (2 * static_cast<size_t>(ss_floats) + 256 + (FUSED ? 256 : 0) + 2 * max_idx_words) * 4u + 64u +
+                         rot_signs_b + rot_xbuf_b;
     const size_t wbufs = FUSED ? static_cast<size_t>(threads) * YS : 0;
     const size_t enc_one = (L.enc_bytes + 127u) & ~size_t(127);
     EncodeSmem sm;
@@ -602,11 +683,13 @@ static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     sm.edges_off = sm.ss_off + 2u * ss_floats * 4u;
     sm.levels_off = sm.edges_off + 256u * 4u;
     sm.idx_off = sm.levels_off + (FUSED ? 256u * 4u : 0u);
-    sm.wbuf_off = (sm.idx_off + 2u * max_idx_words * 4u + 15u) & ~15u;
+    sm.signs_off = (sm.idx_off + 2u * max_idx_words * 4u + 15u) & ~15u;
+    sm.xbuf_off = sm.signs_off + static_cast<uint32_t>(rot_signs_b);
+    sm.wbuf_off = sm.xbuf_off + static_cast<uint32_t>(rot_xbuf_b);
     const size_t smem = sm.wbuf_off + wbufs;
     if (smem > static_cast<size_t>(smem_max)) return PVQ_ERR_UNSUPPORTED;
 
-    auto kern = encode_kernel<N, W, FUSED, YT, BF16>;
+    auto kern = encode_kernel<N, W, FUSED, YT, BF16, ROT>;
     int per_sm = 0;
     if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
@@ -618,9 +701,14 @@ static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
 
 template <int N, int W, bool BF16>
 static int launch_encode_nwb(BatchArgs& a, bool fused, cudaStream_t s) {
-    if (!fused) return launch_encode_t<N, W, false, int8_t, BF16>(a, s);
-    if (a.K <= 127) return launch_encode_t<N, W, true, int8_t, BF16>(a, s);
-    return launch_encode_t<N, W, true, int16_t, BF16>(a, s);
+    if (a.rot_block != 0) {  // rotating kernels are built for byte-sized slots only (K <= 127)
+        if (!fused) return launch_encode_t<N, W, false, int8_t, BF16, true>(a, s);
+        if (a.K <= 127) return launch_encode_t<N, W, true, int8_t, BF16, true>(a, s);
+        return PVQ_ERR_UNSUPPORTED;
+    }
+    if (!fused) return launch_encode_t<N, W, false, int8_t, BF16, false>(a, s);
+    if (a.K <= 127) return launch_encode_t<N, W, true, int8_t, BF16, false>(a, s);
+    return launch_encode_t<N, W, true, int16_t, BF16, false>(a, s);
 }
 
 template <int N, int W>

@@ -290,7 +290,7 @@ int fill_matrix(const pvq_matrix_desc& d, int need, int dtype, const Common& c, 
 
 int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int N, int K, int scale_bits,
               const uint32_t* d_table, uint32_t* d_status, int kind /*0 enc,1 dec,2 fused*/,
-              pvq_stream_t stream) {
+              pvq_stream_t stream, int rot_block = 0, const float* d_signs = nullptr) {
     if (!descs || count < 1 || count > kMaxBatch) return PVQ_ERR_INVALID_ARG;
     if (kind != 1 && dtype != PVQ_DTYPE_F32 && dtype != PVQ_DTYPE_BF16) return PVQ_ERR_INVALID_ARG;
     Common c;
@@ -305,6 +305,14 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
     a.status = d_status;
     a.c_one = 1u;
     a.c_minus_one = 0xffffffffu;
+    if (rot_block != 0) {
+        if (!d_signs || rot_block < N || (rot_block & (rot_block - 1)) != 0) return PVQ_ERR_INVALID_ARG;
+        if (rot_block > 16384) return PVQ_ERR_UNSUPPORTED;
+        for (int i = 0; i < count; ++i)
+            if (descs[i].cols % rot_block != 0) return PVQ_ERR_INVALID_ARG;
+        a.rot_block = rot_block;
+        a.rot_signs = d_signs;
+    }
     for (int i = 0; i < count; ++i) {
         st = fill_matrix(descs[i], need, dtype, c, &a.m[i]);
         if (st != PVQ_OK) return st;
@@ -378,4 +386,42 @@ extern "C" int pvq_decode_batched(const pvq_matrix_desc* descs, int count, int N
                                   const uint32_t* d_table, uint32_t* d_status, pvq_stream_t stream) {
     return run_batch(descs, count, NEED_OUT | NEED_CODES | NEED_LEVELS, PVQ_DTYPE_BF16, N, K, scale_bits,
                      d_table, d_status, 1, stream);
+}
+
+extern "C" int pvq_rotate_encode(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int block,
+                                 const float* d_signs, int N, int K, int scale_bits, const uint32_t* d_table,
+                                 const float* d_edges, uint32_t* d_codes, uint8_t* d_scale_idx,
+                                 float* d_row_norm, pvq_stream_t stream) {
+    if (block == 0) return PVQ_ERR_INVALID_ARG;
+    pvq_matrix_desc d;
+    std::memset(&d, 0, sizeof d);
+    d.d_x = d_x;
+    d.d_codes = d_codes;
+    d.d_scale_idx = d_scale_idx;
+    d.d_row_norm = d_row_norm;
+    d.d_edges = d_edges;
+    d.rows = rows;
+    d.cols = cols;
+    d.ld = ld;
+    return run_batch(&d, 1, NEED_X | NEED_CODES | NEED_EDGES, dtype, N, K, scale_bits, d_table, nullptr, 0,
+                     stream, block, d_signs);
+}
+
+extern "C" int pvq_rotate_roundtrip(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int block,
+                                    const float* d_signs, int N, int K, int scale_bits,
+                                    const uint32_t* d_table, const float* d_edges, const float* d_levels,
+                                    void* d_out, int64_t ld_out, pvq_stream_t stream) {
+    if (block == 0) return PVQ_ERR_INVALID_ARG;
+    pvq_matrix_desc d;
+    std::memset(&d, 0, sizeof d);
+    d.d_x = d_x;
+    d.d_out = d_out;
+    d.d_edges = d_edges;
+    d.d_levels = d_levels;
+    d.rows = rows;
+    d.cols = cols;
+    d.ld = ld;
+    d.ld_out = ld_out;
+    return run_batch(&d, 1, NEED_X | NEED_OUT | NEED_EDGES | NEED_LEVELS, dtype, N, K, scale_bits, d_table,
+                     nullptr, 2, stream, block, d_signs);
 }

@@ -44,6 +44,9 @@ struct BatchArgs {
     // see through stay multiply-adds, which run on the FMA pipe; the walk uses them for plain
     // moves, adds and subtracts to take load off the integer ALU pipe, its bottleneck.
     uint32_t c_one, c_minus_one;
+    // rotation in front of the encoder (Sec. 2.3 / Sec. 3.3 Step 1); rot_block = 0: none
+    const float* rot_signs;  // +-1, rot_block of them
+    int rot_block;           // power of two, a multiple of N, dividing every cols
 };
 
 // Layout of the table blob.  Section 0 is the count table as the paper defines it,
@@ -129,7 +132,7 @@ int prepare_kernel(const void* kern, int threads, size_t smem, int* blocks_per_s
 
 // launchers (one per kernel family); all return a pvq_status
 int launch_decode(const BatchArgs& args, int N, int W, cudaStream_t stream);
-int launch_encode(const BatchArgs& args, int dtype, int N, int W, bool fused, cudaStream_t stream);
+int launch_encode(const BatchArgs& args, int dtype, int N, int W, bool fused, cudaStream_t stream);  // rotates when args.rot_block != 0
 
 // ---------------------------------------------------------------- device bits
 

@@ -77,8 +77,10 @@ class Workload:
     N: int           # group size
     index_bits: int  # bits of one group's direction code
     scale_bits: int  # bits of one group's amplitude index
-    mode: str        # "encode+decode", "decode", "roundtrip"
+    mode: str        # "encode+decode", "decode", "roundtrip", "rotate_roundtrip"
     matrices: List[Matrix]
+    rot_block: int = 0          # "rotate_roundtrip": size of the Hadamard blocks applied on the fly
+    signs: np.ndarray = None    # ... and their +-1 signs (float32, rot_block of them)
 
     @property
     def weights(self) -> int:
@@ -146,3 +148,18 @@ def config5(tokens=16384, hidden=4096) -> Workload:
     x = hadamard_rows(x, hidden, _signs(rng, hidden))
     return Workload("c5_bf16_activations", 32, 64, 8, "roundtrip",
                     [Matrix("act", f32_to_bf16_bits(x), "bf16")])
+
+
+def config5_unrotated(tokens=16384, hidden=4096) -> Workload:
+    """config5's activations before their rotation (same seed, same draws): rows iid N(0,1)
+    with 0.1 % of the channels scaled by 20, in bf16, plus the signs of the hidden-point
+    random-sign Hadamard that the codec applies on the fly; N=32, 64-bit codes, 8-bit
+    amplitudes; rotate -> encode -> decode in one kernel."""
+    rng = _rng(5)
+    x = rng.standard_normal((tokens, hidden), dtype=np.float32)
+    n_out = max(int(round(hidden * 0.001)), 1)
+    ch = rng.choice(hidden, size=n_out, replace=False)
+    x[:, ch] *= np.float32(20.0)
+    signs = _signs(rng, hidden)
+    return Workload("c5r_bf16_activations_rotated_on_the_fly", 32, 64, 8, "rotate_roundtrip",
+                    [Matrix("act", f32_to_bf16_bits(x), "bf16")], rot_block=hidden, signs=signs)

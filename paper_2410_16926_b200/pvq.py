@@ -65,6 +65,8 @@ def lib():
         L.pvq_roundtrip.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, vp, vp, i64, vp]
         L.pvq_encode_batched.argtypes = [C.POINTER(MatrixDesc), i32, i32, i32, i32, i32, vp, vp]
         L.pvq_decode_batched.argtypes = [C.POINTER(MatrixDesc), i32, i32, i32, i32, vp, vp, vp]
+        L.pvq_rotate_encode.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.pvq_rotate_roundtrip.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, i32, i32, vp, vp, vp, vp, i64, vp]
         L.pvq_decode_static_table.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, i64, vp, vp]
         _lib = L
     return _lib
@@ -73,7 +75,7 @@ def lib():
 EXPORTS = ["pvq_strerror", "pvq_last_cuda_error", "pvq_index_bits", "pvq_max_pulses", "pvq_code_words",
            "pvq_count_table_bytes", "pvq_scale_row_stride", "pvq_build_count_table",
            "pvq_build_scale_codebook", "pvq_encode", "pvq_decode", "pvq_roundtrip", "pvq_encode_batched",
-           "pvq_decode_batched", "pvq_decode_static_table"]
+           "pvq_decode_batched", "pvq_decode_static_table", "pvq_rotate_encode", "pvq_rotate_roundtrip"]
 
 
 def _check(status, where):
@@ -220,6 +222,35 @@ def roundtrip(x, N, K, scale_bits, table, edges, levels, out=None):
                                _ptr(table, torch.int32), _ptr(edges, torch.float32),
                                _ptr(levels, torch.float32), _ptr(out, torch.bfloat16), out.stride(0),
                                _stream()), "pvq_roundtrip")
+    return out
+
+
+def rotate_encode(x, block, signs, N, K, scale_bits, table, edges, out=None):
+    """encode() of the rows of x rotated on the fly by the random-sign Hadamard of size `block`
+    (signs: float32 +-1, `block` of them)."""
+    rows, cols = x.shape
+    G = cols // N
+    if out is None:
+        out = alloc_encoded(rows, G, code_words(N, K), scale_bits, x.device)
+    codes, sidx, rnorm = out
+    _check(lib().pvq_rotate_encode(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), block,
+                                   _ptr(signs, torch.float32), N, K, scale_bits, _ptr(table, torch.int32),
+                                   _ptr(edges, torch.float32), _ptr(codes, torch.int32),
+                                   _ptr(sidx, torch.uint8), _ptr(rnorm, torch.float32), _stream()),
+           "pvq_rotate_encode")
+    return codes, sidx, rnorm
+
+
+def rotate_roundtrip(x, block, signs, N, K, scale_bits, table, edges, levels, out=None):
+    """roundtrip() of the rows of x rotated on the fly: bfloat16 [rows][cols] in the rotated basis."""
+    rows, cols = x.shape
+    if out is None:
+        out = torch.empty((rows, cols), dtype=torch.bfloat16, device=x.device)
+    _check(lib().pvq_rotate_roundtrip(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), block,
+                                      _ptr(signs, torch.float32), N, K, scale_bits,
+                                      _ptr(table, torch.int32), _ptr(edges, torch.float32),
+                                      _ptr(levels, torch.float32), _ptr(out, torch.bfloat16), out.stride(0),
+                                      _stream()), "pvq_rotate_roundtrip")
     return out
 
 

@@ -135,3 +135,23 @@ def test_c1_fp32_every_row():
     pvq.decode_batched(items, wl.N, K, wl.scale_bits, table)
     torch.cuda.synchronize()
     check_rows(wl, items, K, W, nrows=512, what=("codes", "out"))
+
+
+def test_c5r_activations_rotated_on_the_fly_sampled_rows():
+    wl = inputs.config5_unrotated()
+    K = pvq.max_pulses(wl.N, wl.index_bits)
+    W = pvq.code_words(wl.N, K)
+    table = pvq.build_count_table(wl.N, K)
+    items = workload_items(wl, K, W)
+    it = items[0]
+    signs = torch.from_numpy(wl.signs).to(DEV)
+    pvq.rotate_roundtrip(it["x"], wl.rot_block, signs, wl.N, K, wl.scale_bits, table, it["edges"], it["levels"],
+                         out=it["out"])
+    torch.cuda.synchronize()
+    m = wl.matrices[0]
+    rows = sample_rows(m.rows, 256, seed=55)
+    xr = po.rotate(np.ascontiguousarray(m.data[rows]), wl.rot_block, wl.signs)
+    enc = po.encode(xr, wl.N, K, wl.scale_bits, it["e_np"], W=W)
+    o_out, st = po.decode(*enc, wl.N, K, wl.scale_bits, it["l_np"])
+    r = torch.from_numpy(rows).to(DEV)
+    assert st == 0 and np.array_equal(bf16_bits(it["out"][r].contiguous()), o_out)

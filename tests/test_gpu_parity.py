@@ -307,3 +307,44 @@ def test_library_codebook_end_to_end():
     # uniform bin occupancy on Gaussian rows (Sec. 3.4): every 4-bit bin near 1/16
     occ = np.bincount(q.ravel(), minlength=16) / q.size
     assert np.all(np.abs(occ - 1 / 16) < 0.02)
+
+
+# ------------------------------------------------------------- rotation on the fly
+
+@pytest.mark.parametrize("N,bits,rows,cols,block,b,kind", [
+    (32, 64, 37, 4096, 4096, 8, "bf16"),     # a block spans 128 threads: shuffles and shared memory
+    (32, 96, 9, 14336, 512, 8, "bf16"),      # 16 threads per block: shuffles only; G = 448
+    (32, 64, 21, 512, 32, 8, "f32"),         # block = group: in-thread stages only
+    (16, 40, 11, 192, 64, 4, "f32"),         # G = 12, three blocks per row
+    (64, 192, 5, 3584, 512, 6, "bf16"),      # N = 64
+])
+def test_rotate_encode_and_roundtrip_parity(N, bits, rows, cols, block, b, kind):
+    rng = np.random.default_rng(block + rows)
+    x = rng.standard_normal((rows, cols)).astype(np.float32)
+    x[:, 3] *= 20.0                                            # an outlier channel to spread
+    x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+    signs = (rng.integers(0, 2, size=block) * 2 - 1).astype(np.float32)
+    cd = Codec(N, bits, cols // N, b)
+    xr = po.rotate(x_np, block, signs)                         # oracle: rotate, then the usual path
+    o_codes, o_sidx, o_rnorm = po.encode(xr, cd.N, cd.K, cd.b, cd.edges_np, W=cd.W)
+    o_out, _ = po.decode(o_codes, o_sidx, o_rnorm, cd.N, cd.K, cd.b, cd.levels_np)
+    x_dev = to_device(x_np, kind)
+    s_dev = torch.from_numpy(signs).to(DEV)
+    codes, sidx, rnorm = pvq.rotate_encode(x_dev, block, s_dev, cd.N, cd.K, cd.b, cd.table, cd.edges)
+    torch.cuda.synchronize()
+    assert np.array_equal(rnorm.cpu().numpy().view(np.uint32), o_rnorm.view(np.uint32)), "row norms"
+    assert np.array_equal(sidx.cpu().numpy(), o_sidx), "amplitude indices"
+    assert np.array_equal(as_u32(codes), o_codes), "codes"
+    if cd.K <= 127:
+        out = pvq.rotate_roundtrip(x_dev, block, s_dev, cd.N, cd.K, cd.b, cd.table, cd.edges, cd.levels)
+        torch.cuda.synchronize()
+        assert np.array_equal(bf16_bits(out), o_out), "fused round trip"
+
+
+def test_rotate_rejects_bad_blocks():
+    cd = Codec(32, 64, 8, 8)
+    x = torch.zeros((4, 256), dtype=torch.float32, device=DEV)
+    s = torch.ones(256, dtype=torch.float32, device=DEV)
+    for block in (0, 16, 48, 512):          # zero, below N, not a power of two, not dividing cols
+        with pytest.raises(pvq.PvqError):
+            pvq.rotate_encode(x, block, s, cd.N, cd.K, cd.b, cd.table, cd.edges)
