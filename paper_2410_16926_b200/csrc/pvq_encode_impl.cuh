@@ -306,12 +306,16 @@ struct EncodeSmem {
 // so thread t and its partner t ^ d hold groups of the same block), larger ones through
 // shared memory.  Every sum is one fp32 addition, so the result does not depend on which of
 // these three ways a stage takes.
+// s_signbits: the signs of a block packed N to a word (bit i of word j set: column j*N + i is
+// negated; for N = 64 two words per group).
 template <int N>
-__device__ __forceinline__ void rotate_tile(float (&x)[N], const float* s_signs, int block, float scale,
+__device__ __forceinline__ void rotate_tile(float (&x)[N], const uint32_t* s_signbits, int block, float scale,
                                             int g, float* xbuf, int tid, int nthreads) {
-    const int col0 = (g * N) & (block - 1);
+    const int T0 = block / N;
+    const uint32_t* sb = s_signbits + (g & (T0 - 1)) * ((N + 31) / 32);
 #pragma unroll
-    for (int i = 0; i < N; ++i) x[i] = __fmul_rn(x[i], s_signs[col0 + i]);
+    for (int i = 0; i < N; ++i)  // multiplying by -1 flips the sign bit
+        x[i] = __uint_as_float(__float_as_uint(x[i]) ^ ((sb[i / 32] >> (i % 32)) << 31));
 #pragma unroll
     for (int h = 1; h < N; h <<= 1) {
 #pragma unroll
@@ -324,12 +328,14 @@ __device__ __forceinline__ void rotate_tile(float (&x)[N], const float* s_signs,
         }
     }
     const int T = block / N;  // threads per rotation block
+    // a + b on the thread that holds a, a - b on the one that holds b: other + sgn * own with
+    // sgn = +-1 (the product is exact, so this is the one rounding of the sum or difference)
     for (int d = 1; d < T && d < 32; d <<= 1) {
-        const bool upper = (tid & d) != 0;
+        const float sgn = (tid & d) != 0 ? -1.0f : 1.0f;
 #pragma unroll
         for (int i = 0; i < N; ++i) {
             const float other = __shfl_xor_sync(kFull, x[i], d);
-            x[i] = upper ? __fsub_rn(other, x[i]) : __fadd_rn(x[i], other);
+            x[i] = __fmaf_rn(x[i], sgn, other);
         }
     }
     for (int d = 32; d < T; d <<= 1) {
@@ -337,12 +343,9 @@ __device__ __forceinline__ void rotate_tile(float (&x)[N], const float* s_signs,
 #pragma unroll
         for (int i = 0; i < N; ++i) xbuf[i * nthreads + tid] = x[i];
         __syncthreads();
-        const bool upper = (tid & d) != 0;
+        const float sgn = (tid & d) != 0 ? -1.0f : 1.0f;
 #pragma unroll
-        for (int i = 0; i < N; ++i) {
-            const float other = xbuf[i * nthreads + (tid ^ d)];
-            x[i] = upper ? __fsub_rn(other, x[i]) : __fadd_rn(x[i], other);
-        }
+        for (int i = 0; i < N; ++i) x[i] = __fmaf_rn(x[i], sgn, xbuf[i * nthreads + (tid ^ d)]);
     }
 #pragma unroll
     for (int i = 0; i < N; ++i) x[i] = __fmul_rn(x[i], scale);
@@ -395,11 +398,17 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     const int b = a.scale_bits;
     const int nedges = (1 << b) - 1;
     const TableLayout L = table_layout(N, K, W);
-    float* s_signs = reinterpret_cast<float*>(smem + sm.signs_off);
+    uint32_t* s_signs = reinterpret_cast<uint32_t*>(smem + sm.signs_off);
     float* s_xbuf = reinterpret_cast<float*>(smem + sm.xbuf_off);
     float rot_scale = 1.0f;
     if constexpr (ROT) {
-        for (int i = threadIdx.x; i < a.rot_block; i += blockDim.x) s_signs[i] = a.rot_signs[i];
+        constexpr int WPG = (N + 31) / 32;  // sign words per group
+        for (int j = threadIdx.x; j < a.rot_block / N * WPG; j += blockDim.x) {
+            uint32_t bits = 0;
+            const int col = j * (N / WPG);
+            for (int i = 0; i < N / WPG; ++i) bits |= (a.rot_signs[col + i] < 0.0f ? 1u : 0u) << i;
+            s_signs[j] = bits;
+        }
         rot_scale = static_cast<float>(1.0 / sqrt(static_cast<double>(a.rot_block)));
     }
     float* s_ss2 = reinterpret_cast<float*>(smem + sm.ss_off);
