@@ -16,6 +16,9 @@
  *   amplitude          Sec. 2.3 (amplitude = ||w||_2), Sec. 3.3 Step 5 and
  *                      Sec. 3.4 (quantile quantiser on s_g^2 / ||s||^2)
  *   reconstruction     Sec. 2.4 (projection of the pyramid point on the sphere)
+ *   16-bit amplitudes  Sec. 4.1 setting: the amplitude itself as IEEE binary16 (scale_bits = 16)
+ *   least squares      Sec. 3.3 Step 4 read as the least-squares scale of the unit
+ *                      direction, s = w_hat^T w / w_hat^T w_hat (amp_mode = 1)
  *   rotation           Sec. 2.3 "Hadamard coherence processing" / Sec. 3.3 Step 1, along
  *                      the input dimension: x <- (x * s) H_n / sqrt(n) per block of n
  *
@@ -218,6 +221,52 @@ static uint16_t f32_to_bf16_rne(float f) {
     u += 0x7fffu + lsb;
     return (uint16_t)(u >> 16);
 }
+
+/* IEEE binary16 <-> binary32; to binary16 rounds to nearest, ties to even, overflows to infinity */
+static uint16_t f32_to_f16_rne(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    uint32_t sign = (u >> 16) & 0x8000u;
+    uint32_t a = u & 0x7fffffffu;
+    if (a > 0x7f800000u) return (uint16_t)(sign | 0x7e00u);          /* NaN */
+    if (a >= 0x47800000u) return (uint16_t)(sign | 0x7c00u);         /* >= 65536: infinity (also from 65520 up, below) */
+    if (a < 0x33000000u) return (uint16_t)sign;                      /* below 2^-25: zero */
+    int e = (int)(a >> 23) - 127;                                    /* unbiased exponent */
+    uint32_t m = (a & 0x7fffffu) | 0x800000u;                        /* 24-bit significand */
+    int shift = e >= -14 ? 13 : 13 + (-14 - e);                      /* bits dropped */
+    uint32_t kept = m >> shift;
+    uint32_t rem = m & ((1u << shift) - 1u);
+    uint32_t half = 1u << (shift - 1);
+    if (rem > half || (rem == half && (kept & 1u))) kept += 1;
+    uint32_t h;
+    if (e >= -14)
+        h = ((uint32_t)(e + 15) << 10) + (kept - 0x400u);            /* a carry out of the significand moves into the exponent */
+    else
+        h = kept;                                                     /* subnormal (or the smallest normal after rounding up) */
+    if (h >= 0x7c00u) h = 0x7c00u;
+    return (uint16_t)(sign | h);
+}
+
+static float f16_to_f32(uint16_t h) {
+    uint32_t sign = ((uint32_t)h & 0x8000u) << 16;
+    uint32_t e = (h >> 10) & 0x1fu, m = h & 0x3ffu;
+    float f;
+    if (e == 0x1f) {
+        uint32_t u = sign | 0x7f800000u | (m << 13);
+        memcpy(&f, &u, 4);
+        return f;
+    }
+    if (e == 0) {
+        f = (float)m * 5.9604644775390625e-8f;                        /* m * 2^-24, exact */
+        return sign ? -f : f;
+    }
+    uint32_t u = sign | ((e + 112u) << 23) | (m << 13);
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+uint16_t pvqo_f32_to_f16(float f) { return f32_to_f16_rne(f); }
+float pvqo_f16_to_f32(uint16_t h) { return f16_to_f32(h); }
 
 /*
  * The one summation order of this build: a balanced tree over contiguous
@@ -440,11 +489,20 @@ static uint32_t get_bits(const uint8_t *row, int64_t bitpos, int nbits) {
  * Outputs: codes[(r*G+g)*W + w]; scale indices as an LSB-first bit stream per
  * row; row_norm[r].
  */
-int pvqo_encode(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
-                int scale_bits, int W, const float *edges, uint32_t *codes, uint8_t *scale_idx,
-                float *row_norm, int nthreads) {
+/*
+ * amp_mode 0: the amplitude of a group is ||x_g||_2 (Sec. 2.3), so u = ss / ss_row.
+ * amp_mode 1: least squares (Step 4): with y the chosen point and y_hat = y / ||y||_2,
+ *             a = y_hat^T x = (sum |y_i| |x_i|) / sqrt(sum y_i^2)   (y_i has the sign of x_i)
+ *             with the tree sum over i of the rounded products, and u = (a * a) / ss_row.
+ * scale_bits 1..8: q from the quantile edges as above.  scale_bits 16: the amplitude itself,
+ *             sqrt(ss) or a, rounded to IEEE binary16, 16 bits per group in the same stream.
+ */
+int pvqo_encode_amp(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+                    int scale_bits, int amp_mode, int W, const float *edges, uint32_t *codes,
+                    uint8_t *scale_idx, float *row_norm, int nthreads) {
     if (N < 1 || (N & (N - 1)) || cols % N || W < 1 || W > PVQO_MAXW) return -1;
-    if (scale_bits < 1 || scale_bits > 8) return -1;
+    if ((scale_bits < 1 || scale_bits > 8) && scale_bits != 16) return -1;
+    if (amp_mode != 0 && amp_mode != 1) return -1;
     big_t *t = count_table(N, K);
     if (!t) return -1;
     {
@@ -457,7 +515,7 @@ int pvqo_encode(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld
         }
     }
     int64_t G = cols / N;
-    int nedges = (1 << scale_bits) - 1;
+    int nedges = scale_bits <= 8 ? (1 << scale_bits) - 1 : 0;
     size_t sstride = scale_row_stride(G, scale_bits);
     memset(scale_idx, 0, sstride * (size_t)rows);
 #ifdef _OPENMP
@@ -486,12 +544,29 @@ int pvqo_encode(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld
         float ss_row = pvqo_tree_sum_padded(ss, (int)G);
         row_norm[r] = sqrtf(ss_row);
         for (int64_t g = 0; g < G; ++g) {
-            float u = ss_row > 0.0f ? ss[g] / ss_row : 0.0f;
-            uint32_t q = 0;
-            for (int j = 0; j < nedges; ++j)
-                if (u >= edges[j]) ++q;
-            put_bits(scale_idx + sstride * (size_t)r, g * scale_bits, scale_bits, q);
             quantize_direction(xs + g * N, l1[g], N, K, y);
+            float amp2 = ss[g];          /* squared amplitude */
+            float amp = sqrtf(ss[g]);
+            if (amp_mode == 1) {
+                long ssy = 0;
+                for (int i = 0; i < N; ++i) {
+                    int32_t m = y[i] < 0 ? -y[i] : y[i];
+                    ssy += (long)m * m;
+                    tmp[i] = (float)m * fabsf(xs[g * N + i]);
+                }
+                float dot = tree_sum(tmp, 0, N);
+                amp = dot / sqrtf((float)ssy);
+                amp2 = amp * amp;
+            }
+            uint32_t q = 0;
+            if (scale_bits == 16) {
+                q = f32_to_f16_rne(amp);
+            } else {
+                float u = ss_row > 0.0f ? amp2 / ss_row : 0.0f;
+                for (int j = 0; j < nedges; ++j)
+                    if (u >= edges[j]) ++q;
+            }
+            put_bits(scale_idx + sstride * (size_t)r, g * scale_bits, scale_bits, q);
             big_t c;
             enumerate(y, N, K, t, &c);
             memcpy(codes + ((size_t)r * (size_t)G + (size_t)g) * (size_t)W, c.w, 4u * (size_t)W);
@@ -506,6 +581,13 @@ int pvqo_encode(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld
     return 0;
 }
 
+int pvqo_encode(const void *x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+                int scale_bits, int W, const float *edges, uint32_t *codes, uint8_t *scale_idx,
+                float *row_norm, int nthreads) {
+    return pvqo_encode_amp(x, dtype, rows, cols, ld, N, K, scale_bits, 0, W, edges, codes, scale_idx, row_norm,
+                           nthreads);
+}
+
 /*
  * Decode to bf16.  Per group: de-enumerate; ssy = sum y_i^2 (exact);
  *   amp = row_norm * levels[q]           (levels = sqrt of the bin midpoints' quantiles)
@@ -518,7 +600,7 @@ int pvqo_decode(const uint32_t *codes, const uint8_t *scale_idx, const float *ro
                 int64_t cols, int N, int K, int scale_bits, int W, const float *levels,
                 uint16_t *out, int64_t ld_out, uint32_t *status, int nthreads) {
     if (N < 1 || (N & (N - 1)) || cols % N || W < 1 || W > PVQO_MAXW) return -1;
-    if (scale_bits < 1 || scale_bits > 8) return -1;
+    if ((scale_bits < 1 || scale_bits > 8) && scale_bits != 16) return -1;
     big_t *t = count_table(N, K);
     if (!t) return -1;
     int64_t G = cols / N;
@@ -544,7 +626,8 @@ int pvqo_decode(const uint32_t *codes, const uint8_t *scale_idx, const float *ro
             uint32_t q = get_bits(scale_idx + sstride * (size_t)r, g * scale_bits, scale_bits);
             long ssy = 0;
             for (int i = 0; i < N; ++i) ssy += (long)y[i] * y[i];
-            float amp = row_norm[r] * levels[q];
+            /* scale_bits 16: q is the amplitude itself as binary16 */
+            float amp = scale_bits == 16 ? f16_to_f32((uint16_t)q) : row_norm[r] * levels[q];
             float s = amp / sqrtf((float)ssy);
             for (int i = 0; i < N; ++i) o[i] = f32_to_bf16_rne((float)y[i] * s);
         }

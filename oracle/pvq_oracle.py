@@ -31,6 +31,11 @@ def lib():
         L.pvqo_deenumerate.argtypes = [vp, i32, i32, i32, vp]
         L.pvqo_scale_row_stride.argtypes = [i64, i32]
         L.pvqo_scale_row_stride.restype = C.c_size_t
+        L.pvqo_encode_amp.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, i32, i32, vp, vp, vp, vp, i32]
+        L.pvqo_f32_to_f16.argtypes = [C.c_float]
+        L.pvqo_f32_to_f16.restype = C.c_uint16
+        L.pvqo_f16_to_f32.argtypes = [C.c_uint16]
+        L.pvqo_f16_to_f32.restype = C.c_float
         L.pvqo_encode.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, vp, i32]
         L.pvqo_decode.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, i32, vp, vp, i64, vp, i32]
         L.pvqo_rotate.argtypes = [vp, i32, i64, i64, i64, i32, vp, vp]
@@ -111,9 +116,19 @@ def int_to_code(v: int, W: int) -> np.ndarray:
     return np.array([(v >> (32 * i)) & 0xFFFFFFFF for i in range(W)], dtype=np.uint32)
 
 
-def encode(x: np.ndarray, N: int, K: int, scale_bits: int, edges: np.ndarray, W: int = None,
-           nthreads: int = 0):
+def f32_to_f16(f) -> int:
+    return int(lib().pvqo_f32_to_f16(float(f)))
+
+
+def f16_to_f32(h) -> float:
+    return float(lib().pvqo_f16_to_f32(int(h)))
+
+
+def encode(x: np.ndarray, N: int, K: int, scale_bits: int, edges: np.ndarray = None, W: int = None,
+           nthreads: int = 0, amp_mode: int = 0):
     """x: 2-D float32 array, or uint16 array holding bf16 bit patterns.
+    scale_bits 1..8 with the quantile `edges`, or 16 (binary16 amplitudes, no edges);
+    amp_mode 0: amplitude ||x_g||, 1: least-squares amplitude of the chosen direction.
     Returns (codes uint32 [rows][G][W], scale_idx uint8 [rows][stride], row_norm f32 [rows])."""
     assert x.ndim == 2 and x.flags.c_contiguous
     if x.dtype == np.float32:
@@ -126,28 +141,34 @@ def encode(x: np.ndarray, N: int, K: int, scale_bits: int, edges: np.ndarray, W:
     G = cols // N
     if W is None:
         W = words_for_bits(index_bits(N, K))
-    edges = np.ascontiguousarray(edges, dtype=np.float32)
-    assert edges.size == (1 << scale_bits) - 1
+    if scale_bits == 16:
+        edges = np.zeros(1, dtype=np.float32)
+    else:
+        edges = np.ascontiguousarray(edges, dtype=np.float32)
+        assert edges.size == (1 << scale_bits) - 1
     codes = np.zeros((rows, G, W), dtype=np.uint32)
     sidx = np.zeros((rows, scale_row_stride(G, scale_bits)), dtype=np.uint8)
     rnorm = np.zeros(rows, dtype=np.float32)
-    rc = lib().pvqo_encode(_p(x), dtype, rows, cols, cols, N, K, scale_bits, W, _p(edges),
-                           _p(codes), _p(sidx), _p(rnorm), nthreads)
+    rc = lib().pvqo_encode_amp(_p(x), dtype, rows, cols, cols, N, K, scale_bits, amp_mode, W, _p(edges),
+                               _p(codes), _p(sidx), _p(rnorm), nthreads)
     if rc != 0:
         raise ValueError("oracle encode rejected its arguments")
     return codes, sidx, rnorm
 
 
 def decode(codes: np.ndarray, sidx: np.ndarray, rnorm: np.ndarray, N: int, K: int,
-           scale_bits: int, levels: np.ndarray, nthreads: int = 0):
+           scale_bits: int, levels: np.ndarray = None, nthreads: int = 0):
     """Returns (bf16 bit patterns uint16 [rows][cols], status word)."""
     rows, G, W = codes.shape
     cols = G * N
     codes = np.ascontiguousarray(codes, dtype=np.uint32)
     sidx = np.ascontiguousarray(sidx, dtype=np.uint8)
     rnorm = np.ascontiguousarray(rnorm, dtype=np.float32)
-    levels = np.ascontiguousarray(levels, dtype=np.float32)
-    assert levels.size == (1 << scale_bits)
+    if scale_bits == 16:
+        levels = np.zeros(1, dtype=np.float32)
+    else:
+        levels = np.ascontiguousarray(levels, dtype=np.float32)
+        assert levels.size == (1 << scale_bits)
     assert sidx.shape == (rows, scale_row_stride(G, scale_bits))
     out = np.zeros((rows, cols), dtype=np.uint16)
     status = np.zeros(1, dtype=np.uint32)

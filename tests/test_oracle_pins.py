@@ -16,6 +16,7 @@ import pytest
 from oracle import beta_codebook as bc
 from oracle import pvq_oracle as po
 from oracle import pvq_pyref as pr
+from paper_2410_16926_b200 import inputs
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -558,3 +559,67 @@ def test_rotation_of_bf16_input_widens_exactly():
     xb = inputs.f32_to_bf16_bits(x)
     s = np.ones(64, dtype=np.float32)
     assert np.array_equal(po.rotate(xb, 64, s), po.rotate(inputs.bf16_bits_to_f32(xb), 64, s))
+
+
+# --------------------------------------- 16-bit amplitudes and the least-squares amplitude
+
+def test_binary16_conversion_matches_numpy_on_every_half_and_on_ties():
+    # every binary16 value converts to itself; rounding of fp32 agrees with numpy's IEEE conversion
+    for h in list(range(0, 0x7c01, 37)) + [0x0001, 0x03ff, 0x0400, 0x7bff, 0x7c00, 0x8001, 0xfbff]:
+        f = np.array([h], dtype=np.uint16).view(np.float16)[0]
+        assert po.f32_to_f16(np.float32(f)) == h
+        assert np.float32(po.f16_to_f32(h)) == np.float32(f)
+    rng = np.random.default_rng(16)
+    vals = np.concatenate([rng.standard_normal(4000) * 10.0 ** rng.integers(-9, 6, 4000),
+                           [65504.0, 65519.9, 65520.0, 1e9, 5.96e-8, 2.98e-8, 2.9802325e-8, 6.1e-5, 0.0, -0.0,
+                            1.00048828125, 1.0009765625 + 2.0 ** -12]]).astype(np.float32)
+    with np.errstate(over="ignore"):
+        want = vals.astype(np.float16).view(np.uint16)
+    got = np.array([po.f32_to_f16(v) for v in vals], dtype=np.uint16)
+    assert np.array_equal(got, want)
+
+
+def test_binary16_amplitudes_round_trip_the_group_norm():
+    rng = np.random.default_rng(21)
+    N, K, rows, cols = 32, 22, 6, 256
+    x = (rng.standard_normal((rows, cols)) * 0.05).astype(np.float32)
+    codes, sidx, rnorm = po.encode(x, N, K, 16)
+    assert sidx.shape == (rows, 2 * (cols // N))                       # 16 bits per group
+    amp16 = sidx.view(np.uint16).reshape(rows, cols // N)
+    norms = np.sqrt((x.reshape(rows, -1, N).astype(np.float64) ** 2).sum(axis=2))
+    got = amp16.view(np.float16).astype(np.float64)
+    assert np.all(np.abs(got - norms) <= np.abs(norms) * 2.0 ** -11 + 1e-12)   # half an ulp of binary16 (+ fp32 sums)
+    out, st = po.decode(codes, sidx, rnorm, N, K, 16)
+    o = inputs.bf16_bits_to_f32(out).reshape(rows, -1, N).astype(np.float64)
+    # decoded groups have the stored amplitude as their norm (up to bf16 rounding of the elements)
+    assert st == 0 and np.allclose(np.sqrt((o ** 2).sum(axis=2)), got, rtol=6e-3)
+
+
+def test_least_squares_amplitude_is_the_projection_and_beats_the_norm():
+    rng = np.random.default_rng(22)
+    N, K, rows, cols = 16, 18, 8, 128
+    x = rng.standard_normal((rows, cols)).astype(np.float32)
+    c0, s0, r0 = po.encode(x, N, K, 16, amp_mode=0)
+    c1, s1, r1 = po.encode(x, N, K, 16, amp_mode=1)
+    assert np.array_equal(c0, c1)                                      # the direction does not depend on it
+    a0 = s0.view(np.uint16).view(np.float16).astype(np.float64).reshape(rows, -1)
+    a1 = s1.view(np.uint16).view(np.float16).astype(np.float64).reshape(rows, -1)
+    xg = x.reshape(rows, -1, N).astype(np.float64)
+    for r in range(rows):
+        for g in range(cols // N):
+            y, ok = po.deenumerate_code(c0[r, g], N, K)
+            yh = y / np.linalg.norm(y)
+            proj = float(yh @ xg[r, g])                                # argmin_a ||x - a y_hat||
+            assert abs(a1[r, g] - proj) <= abs(proj) * 2.0 ** -10
+            assert np.linalg.norm(xg[r, g] - a1[r, g] * yh) <= np.linalg.norm(xg[r, g] - a0[r, g] * yh) + 1e-3
+            assert a1[r, g] <= a0[r, g] * (1 + 2.0 ** -10)             # Cauchy-Schwarz
+
+
+def test_least_squares_amplitude_with_the_quantile_codebook():
+    rng = np.random.default_rng(23)
+    N, K, b, rows, cols = 32, 22, 8, 4, 1024
+    x = rng.standard_normal((rows, cols)).astype(np.float32)
+    e = bc.edges_f32(N, cols // N, b)
+    q0 = po.unpack_scale_idx(po.encode(x, N, K, b, e, amp_mode=0)[1], cols // N, b)
+    q1 = po.unpack_scale_idx(po.encode(x, N, K, b, e, amp_mode=1)[1], cols // N, b)
+    assert np.all(q1 <= q0) and np.mean(q1 < q0) > 0.5                 # smaller amplitudes, lower bins
