@@ -127,6 +127,7 @@ int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, f
  *   d_x        rows x cols values of `dtype`, leading dimension ld (elements); 16-byte
  *              aligned, ld a multiple of 8 (bf16) or 4 (fp32) elements.
  *   N, K       group size (power of two, 8..64) and pulses; cols % N == 0; G >= 2.
+ *   scale_bits 1..8 (quantile index), or 16 (see pvq_encode_amp).
  *   d_table    from pvq_build_count_table(N, K, ...).
  *   d_edges    2^scale_bits - 1 bin edges.
  *   d_codes    out, rows*G*W words.      d_scale_idx  out, rows * stride bytes.
@@ -160,6 +161,21 @@ int pvq_decode(const uint32_t* d_codes, const uint8_t* d_scale_idx, const float*
 int pvq_roundtrip(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
                   int scale_bits, const uint32_t* d_table, const float* d_edges,
                   const float* d_levels, void* d_out, int64_t ld_out, pvq_stream_t stream);
+
+/* pvq_encode with a choice of amplitude (Sec. 3.3 Step 4).
+ *   amp_mode 0  the amplitude of a group is ||x_g||_2, as in pvq_encode;
+ *   amp_mode 1  least squares: the projection of x_g on the chosen direction,
+ *               a = (sum_i |y_i| |x_i|) / sqrt(sum_i y_i^2)  (fp32, products rounded, summed by
+ *               the balanced tree), and u = a^2 / ||x_row||^2 for the quantile index.
+ * Everything else as pvq_encode; decoding does not depend on the mode.
+ *
+ * scale_bits = 16 (all encode / decode entry points): instead of a quantile index the stream
+ * holds the amplitude itself as IEEE binary16, rounded to nearest even, 16 bits per group
+ * (Sec. 4.1: 16-bit amplitudes); d_edges / d_levels are then unused and may be NULL, and
+ * the row norms are written but not read. */
+int pvq_encode_amp(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+                   int scale_bits, int amp_mode, const uint32_t* d_table, const float* d_edges,
+                   uint32_t* d_codes, uint8_t* d_scale_idx, float* d_row_norm, pvq_stream_t stream);
 
 /* Rotation on the fly (Sec. 2.3 "Hadamard coherence processing", Sec. 3.3 Step 1, along the
  * input dimension; Sec. 4.3 for activations, which have to be rotated at run time): every

@@ -6,6 +6,8 @@
 // memory, from where it scales it and writes its N bf16 values with 16-byte stores.
 #include <algorithm>
 
+#include <cuda_fp16.h>
+
 #include "pvq_walk.cuh"
 
 namespace pvq {
@@ -83,7 +85,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
                 unsigned bits = srow[bit >> 3];
                 if ((bit & 7u) + b > 8u) bits |= static_cast<unsigned>(srow[(bit >> 3) + 1]) << 8;
                 const unsigned q = (bits >> (bit & 7u)) & ((1u << b) - 1u);
-                amp = __fmul_rn(m.row_norm[row], m.levels[q]);
+                // 16 bits: the amplitude itself as binary16; else the quantile level times the row norm
+                amp = b == 16u ? __half2float(__ushort_as_half(static_cast<unsigned short>(q)))
+                               : __fmul_rn(m.row_norm[row], m.levels[q]);
             }
         }
         walk_code<N, W, YT>(c, wt, K, yslots);

@@ -6,6 +6,8 @@
 // of Sec. 3.3: group norms, row norm, direction (Step 3: l1 scale, floor,
 // greedy fix-up), Fischer index (Step 7, Algorithm 2), amplitude index (Step 5).
 #pragma once
+#include <cuda_fp16.h>
+
 #include <algorithm>
 
 #include "pvq_walk.cuh"
@@ -396,7 +398,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     constexpr int WW = WBF16 ? N / 2 : N;
     const int K = a.K;
     const int b = a.scale_bits;
-    const int nedges = (1 << b) - 1;
+    const int nedges = b <= 8 ? (1 << b) - 1 : 0;  // 16 bits: the amplitude itself, no codebook
     const TableLayout L = table_layout(N, K, W);
     uint32_t* s_signs = reinterpret_cast<uint32_t*>(smem + sm.signs_off);
     float* s_xbuf = reinterpret_cast<float*>(smem + sm.xbuf_off);
@@ -497,7 +499,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
         }
         __syncthreads();  // (1) group energies of this tile are in s_ss; nobody is in the previous tile
 
-        if (cur_edges != m.edges) {  // uniform across the block
+        if (nedges != 0 && cur_edges != m.edges) {  // uniform across the block
             for (int i = threadIdx.x; i < nedges; i += blockDim.x) s_edges[i] = m.edges[i];
             if constexpr (FUSED)
                 for (int i = threadIdx.x; i <= nedges; i += blockDim.x) s_levels[i] = m.levels[i];
@@ -523,6 +525,21 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
 #pragma unroll
             for (int i = 0; i < N; ++i) mag[i] = kMagic;
             mag[0] = __int_as_float(kMagicBits + K);
+        }
+
+        // Step 4 as least squares: the amplitude is the projection of x on the chosen direction,
+        // a = (sum |y_i| |x_i|) / sqrt(sum y_i^2), the sum of the rounded products by the fixed tree
+        float ls_amp = 0.0f;
+        if (a.amp_mode == 1) {
+            float t[N];
+            float ssy = 0.0f;
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+                const float mf = __fsub_rn(fabsf(mag[i]), kMagic);  // |y_i|, exact
+                ssy = __fadd_rn(ssy, __fmul_rn(mf, mf));            // integers below 2^24: exact
+                t[i] = __fmul_rn(mf, fabsf(raw_value<N, WBF16>(raw, i)));
+            }
+            ls_amp = __fdiv_rn(tree_sum<N>(t), __fsqrt_rn(ssy));
         }
 
         // the loaded group is dead: ask for the next tile's input now, it arrives while the index is computed
@@ -566,10 +583,16 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
         if (active) {
             const float ss_row = s_ss[rl * gp];
             rnorm = __fsqrt_rn(ss_row);
-            // Step 5: q = floor(CDF(u) 2^b) as the number of bin edges <= u
-            const float u = ss_row > 0.0f ? __fdiv_rn(ss, ss_row) : 0.0f;
-            for (int step = 1 << (b - 1); step >= 1; step >>= 1)
-                if (s_edges[q + step - 1] <= u) q += step;
+            if (b == 16) {  // the amplitude itself, as binary16
+                const float amp16 = a.amp_mode == 1 ? ls_amp : __fsqrt_rn(ss);
+                q = __half_as_ushort(__float2half_rn(amp16));
+            } else {
+                // Step 5: q = floor(CDF(u) 2^b) as the number of bin edges <= u
+                const float amp2 = a.amp_mode == 1 ? __fmul_rn(ls_amp, ls_amp) : ss;
+                const float u = ss_row > 0.0f ? __fdiv_rn(amp2, ss_row) : 0.0f;
+                for (int step = 1 << (b - 1); step >= 1; step >>= 1)
+                    if (s_edges[q + step - 1] <= u) q += step;
+            }
         }
 
         if constexpr (!FUSED) {
@@ -594,7 +617,9 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             }
         } else {
             // decode the code just made (every thread of the warp walks, in lockstep)
-            const float amp = active ? __fmul_rn(rnorm, s_levels[q]) : 0.0f;
+            const float amp = !active ? 0.0f
+                              : b == 16 ? __half2float(__ushort_as_half(static_cast<unsigned short>(q)))
+                                        : __fmul_rn(rnorm, s_levels[q]);
             if (!active) mp_zero(c);
             walk_code<N, W, YT>(c, wt, K, yslots);
             if (active) emit_group<N, YT>(m, yslots, amp, static_cast<unsigned>(row), static_cast<unsigned>(g));

@@ -216,7 +216,7 @@ extern "C" size_t pvq_count_table_bytes(int N, int K) {
 }
 
 extern "C" size_t pvq_scale_row_stride(int64_t G, int scale_bits) {
-    if (G < 1 || scale_bits < 1 || scale_bits > 8) return 0;
+    if (G < 1 || ((scale_bits < 1 || scale_bits > 8) && scale_bits != 16)) return 0;
     size_t bytes = static_cast<size_t>((G * scale_bits + 7) / 8);
     return (bytes + 3u) & ~static_cast<size_t>(3u);
 }
@@ -231,7 +231,7 @@ struct Common {
 
 int check_common(int N, int K, int scale_bits, const uint32_t* d_table, Common* out) {
     if (N < 2 || (N & (N - 1)) != 0 || K < 1) return PVQ_ERR_INVALID_ARG;
-    if (scale_bits < 1 || scale_bits > 8) return PVQ_ERR_INVALID_ARG;
+    if ((scale_bits < 1 || scale_bits > 8) && scale_bits != 16) return PVQ_ERR_INVALID_ARG;
     if (!d_table) return PVQ_ERR_INVALID_ARG;
     if (N < 8 || N > 64 || K > kMaxPulses) return PVQ_ERR_UNSUPPORTED;
     int W = code_words_for(N, K);
@@ -268,8 +268,9 @@ int fill_matrix(const pvq_matrix_desc& d, int need, int dtype, const Common& c, 
         if (!is_aligned(d.d_codes, 4) || !is_aligned(d.d_scale_idx, 4) || !is_aligned(d.d_row_norm, 4))
             return PVQ_ERR_ALIGNMENT;
     }
-    if ((need & NEED_EDGES) && !d.d_edges) return PVQ_ERR_INVALID_ARG;
-    if ((need & NEED_LEVELS) && !d.d_levels) return PVQ_ERR_INVALID_ARG;
+    // the quantile codebook is not used with 16-bit amplitudes
+    if ((need & NEED_EDGES) && c.scale_bits <= 8 && !d.d_edges) return PVQ_ERR_INVALID_ARG;
+    if ((need & NEED_LEVELS) && c.scale_bits <= 8 && !d.d_levels) return PVQ_ERR_INVALID_ARG;
     m->x = d.d_x;
     m->out = d.d_out;
     m->codes = d.d_codes;
@@ -290,7 +291,7 @@ int fill_matrix(const pvq_matrix_desc& d, int need, int dtype, const Common& c, 
 
 int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int N, int K, int scale_bits,
               const uint32_t* d_table, uint32_t* d_status, int kind /*0 enc,1 dec,2 fused*/,
-              pvq_stream_t stream, int rot_block = 0, const float* d_signs = nullptr) {
+              pvq_stream_t stream, int rot_block = 0, const float* d_signs = nullptr, int amp_mode = 0) {
     if (!descs || count < 1 || count > kMaxBatch) return PVQ_ERR_INVALID_ARG;
     if (kind != 1 && dtype != PVQ_DTYPE_F32 && dtype != PVQ_DTYPE_BF16) return PVQ_ERR_INVALID_ARG;
     Common c;
@@ -305,6 +306,8 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
     a.status = d_status;
     a.c_one = 1u;
     a.c_minus_one = 0xffffffffu;
+    if (amp_mode != 0 && amp_mode != 1) return PVQ_ERR_INVALID_ARG;
+    a.amp_mode = amp_mode;
     if (rot_block != 0) {
         if (!d_signs || rot_block < N || (rot_block & (rot_block - 1)) != 0) return PVQ_ERR_INVALID_ARG;
         if (rot_block > 16384) return PVQ_ERR_UNSUPPORTED;
@@ -424,4 +427,21 @@ extern "C" int pvq_rotate_roundtrip(const void* d_x, int dtype, int64_t rows, in
     d.ld_out = ld_out;
     return run_batch(&d, 1, NEED_X | NEED_OUT | NEED_EDGES | NEED_LEVELS, dtype, N, K, scale_bits, d_table,
                      nullptr, 2, stream, block, d_signs);
+}
+
+extern "C" int pvq_encode_amp(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int N, int K,
+                              int scale_bits, int amp_mode, const uint32_t* d_table, const float* d_edges,
+                              uint32_t* d_codes, uint8_t* d_scale_idx, float* d_row_norm, pvq_stream_t stream) {
+    pvq_matrix_desc d;
+    std::memset(&d, 0, sizeof d);
+    d.d_x = d_x;
+    d.d_codes = d_codes;
+    d.d_scale_idx = d_scale_idx;
+    d.d_row_norm = d_row_norm;
+    d.d_edges = d_edges;
+    d.rows = rows;
+    d.cols = cols;
+    d.ld = ld;
+    return run_batch(&d, 1, NEED_X | NEED_CODES | NEED_EDGES, dtype, N, K, scale_bits, d_table, nullptr, 0,
+                     stream, 0, nullptr, amp_mode);
 }

@@ -45,6 +45,7 @@ struct BatchArgs {
     // moves, adds and subtracts to take load off the integer ALU pipe, its bottleneck.
     uint32_t c_one, c_minus_one;
     // rotation in front of the encoder (Sec. 2.3 / Sec. 3.3 Step 1); rot_block = 0: none
+    int amp_mode;            // encode: 0 amplitude ||x_g||, 1 least-squares amplitude (Step 4)
     const float* rot_signs;  // +-1, rot_block of them
     int rot_block;           // power of two, a multiple of N, dividing every cols
 };

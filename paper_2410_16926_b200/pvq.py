@@ -65,6 +65,7 @@ def lib():
         L.pvq_roundtrip.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, vp, vp, vp, vp, i64, vp]
         L.pvq_encode_batched.argtypes = [C.POINTER(MatrixDesc), i32, i32, i32, i32, i32, vp, vp]
         L.pvq_decode_batched.argtypes = [C.POINTER(MatrixDesc), i32, i32, i32, i32, vp, vp, vp]
+        L.pvq_encode_amp.argtypes = [vp, i32, i64, i64, i64, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.pvq_rotate_encode.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.pvq_rotate_roundtrip.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, i32, i32, vp, vp, vp, vp, i64, vp]
         L.pvq_decode_static_table.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, i64, vp, vp]
@@ -75,7 +76,7 @@ def lib():
 EXPORTS = ["pvq_strerror", "pvq_last_cuda_error", "pvq_index_bits", "pvq_max_pulses", "pvq_code_words",
            "pvq_count_table_bytes", "pvq_scale_row_stride", "pvq_build_count_table",
            "pvq_build_scale_codebook", "pvq_encode", "pvq_decode", "pvq_roundtrip", "pvq_encode_batched",
-           "pvq_decode_batched", "pvq_decode_static_table", "pvq_rotate_encode", "pvq_rotate_roundtrip"]
+           "pvq_decode_batched", "pvq_decode_static_table", "pvq_rotate_encode", "pvq_rotate_roundtrip", "pvq_encode_amp"]
 
 
 def _check(status, where):
@@ -170,14 +171,21 @@ def alloc_encoded(rows, G, W, scale_bits, device="cuda"):
     return codes, sidx, rnorm
 
 
-def encode(x, N, K, scale_bits, table, edges, out=None):
+def encode(x, N, K, scale_bits, table, edges, out=None, amp_mode=None):
     """x [rows][cols] float32 / bfloat16 on the GPU -> (codes int32 [rows][G][W],
-    scale_idx uint8 [rows][stride], row_norm float32 [rows])."""
+    scale_idx uint8 [rows][stride], row_norm float32 [rows]).  amp_mode (0 / 1) goes through
+    pvq_encode_amp; scale_bits 16 takes no edges."""
     rows, cols = x.shape
     G = cols // N
     if out is None:
         out = alloc_encoded(rows, G, code_words(N, K), scale_bits, x.device)
     codes, sidx, rnorm = out
+    if amp_mode is not None:
+        _check(lib().pvq_encode_amp(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), N, K, scale_bits, amp_mode,
+                                    _ptr(table, torch.int32), _ptr(edges, torch.float32),
+                                    _ptr(codes, torch.int32), _ptr(sidx, torch.uint8),
+                                    _ptr(rnorm, torch.float32), _stream()), "pvq_encode_amp")
+        return codes, sidx, rnorm
     _check(lib().pvq_encode(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), N, K, scale_bits,
                             _ptr(table, torch.int32), _ptr(edges, torch.float32), _ptr(codes, torch.int32),
                             _ptr(sidx, torch.uint8), _ptr(rnorm, torch.float32), _stream()), "pvq_encode")

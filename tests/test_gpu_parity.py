@@ -348,3 +348,42 @@ def test_rotate_rejects_bad_blocks():
     for block in (0, 16, 48, 512):          # zero, below N, not a power of two, not dividing cols
         with pytest.raises(pvq.PvqError):
             pvq.rotate_encode(x, block, s, cd.N, cd.K, cd.b, cd.table, cd.edges)
+
+
+# ------------------------------------- 16-bit amplitudes and the least-squares amplitude
+
+@pytest.mark.parametrize("N,bits,rows,cols,b,amp_mode,kind", [
+    (32, 96, 19, 4096, 16, 0, "bf16"),
+    (32, 96, 19, 4096, 16, 1, "bf16"),
+    (32, 64, 33, 512, 8, 1, "f32"),
+    (16, 40, 9, 208, 16, 1, "f32"),       # G = 13
+    (64, 192, 5, 3584, 16, 0, "bf16"),
+    (32, 96, 7, 14336, 4, 1, "bf16"),
+])
+def test_amplitude_variants_parity(N, bits, rows, cols, b, amp_mode, kind):
+    rng = np.random.default_rng(rows * 7 + b + amp_mode)
+    x = (rng.standard_t(4.0, size=(rows, cols)) * 0.03).astype(np.float32)
+    x[0, :N] = 0.0                                             # a group without direction
+    x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+    G = cols // N
+    K = pvq.max_pulses(N, bits)
+    W = pvq.code_words(N, K)
+    table = pvq.build_count_table(N, K)
+    e_np = bc.edges_f32(N, G, b) if b <= 8 else None
+    l_np = bc.levels_amp_f32(N, G, b) if b <= 8 else None
+    edges = torch.from_numpy(e_np).to(DEV) if b <= 8 else None
+    levels = torch.from_numpy(l_np).to(DEV) if b <= 8 else None
+    o_codes, o_sidx, o_rnorm = po.encode(x_np, N, K, b, e_np, W=W, amp_mode=amp_mode)
+    o_out, _ = po.decode(o_codes, o_sidx, o_rnorm, N, K, b, l_np)
+    codes, sidx, rnorm = pvq.encode(to_device(x_np, kind), N, K, b, table, edges, amp_mode=amp_mode)
+    torch.cuda.synchronize()
+    assert np.array_equal(as_u32(codes), o_codes), "codes"
+    assert np.array_equal(sidx.cpu().numpy(), o_sidx), "amplitudes"
+    assert np.array_equal(rnorm.cpu().numpy().view(np.uint32), o_rnorm.view(np.uint32)), "row norms"
+    out = pvq.decode(codes, sidx, rnorm, N, K, b, table, levels)
+    torch.cuda.synchronize()
+    assert np.array_equal(bf16_bits(out), o_out), "decoded"
+    if amp_mode == 0 and K <= 127:                             # the fused kernel, 16-bit amplitudes included
+        rt = pvq.roundtrip(to_device(x_np, kind), N, K, b, table, edges, levels)
+        torch.cuda.synchronize()
+        assert np.array_equal(bf16_bits(rt), o_out), "fused"
