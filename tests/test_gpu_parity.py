@@ -387,3 +387,26 @@ def test_amplitude_variants_parity(N, bits, rows, cols, b, amp_mode, kind):
         rt = pvq.roundtrip(to_device(x_np, kind), N, K, b, table, edges, levels)
         torch.cuda.synchronize()
         assert np.array_equal(bf16_bits(rt), o_out), "fused"
+
+
+def test_qsnr_curve_on_a_gaussian_source_equals_the_oracles():
+    # the quality experiment of Sec. 2.6 / Fig. 3 (PVQ curve) through the CUDA path
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((128, 1024)).astype(np.float32)
+    xd = torch.from_numpy(x).to(DEV)
+    curve = []
+    for bpw in (2.0, 3.0, 4.0):
+        N, bits = 32, int(bpw * 32)
+        K = pvq.max_pulses(N, bits)
+        table = pvq.build_count_table(N, K)
+        enc = pvq.encode(xd, N, K, 16, table, None, amp_mode=1)
+        out = pvq.decode(*enc, N, K, 16, table, None).float()
+        torch.cuda.synchronize()
+        q_gpu = 10 * torch.log10((xd.double() ** 2).sum() / ((xd.double() - out.double()) ** 2).sum()).item()
+        c, s, r = po.encode(x, N, K, 16, W=(bits + 31) // 32, amp_mode=1)
+        o, _ = po.decode(c, s, r, N, K, 16)
+        xh = inputs.bf16_bits_to_f32(o).astype(np.float64)
+        q_cpu = 10 * np.log10((x.astype(np.float64) ** 2).sum() / ((x - xh) ** 2).sum())
+        assert abs(q_gpu - q_cpu) < 1e-9
+        curve.append(q_gpu)
+    assert curve[0] < curve[1] < curve[2] and 9.5 < curve[0] < 10.5

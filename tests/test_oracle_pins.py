@@ -623,3 +623,29 @@ def test_least_squares_amplitude_with_the_quantile_codebook():
     q0 = po.unpack_scale_idx(po.encode(x, N, K, b, e, amp_mode=0)[1], cols // N, b)
     q1 = po.unpack_scale_idx(po.encode(x, N, K, b, e, amp_mode=1)[1], cols // N, b)
     assert np.all(q1 <= q0) and np.mean(q1 < q0) > 0.5                 # smaller amplitudes, lower bins
+
+
+# ------------------------------------------------ QSNR on a Gaussian source (Sec. 2.6, Fig. 3)
+
+@pytest.mark.parametrize("N", [16, 32])
+def test_qsnr_on_a_gaussian_source_sits_under_the_rate_distortion_bound(N):
+    # A memoryless Gaussian source at R bits per sample cannot beat 6.02 R dB; a spherical code
+    # of this size stays within a few dB of it, gains about 6 dB per bit, and the least-squares
+    # amplitude is never worse than the norm.
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((128, 1024)).astype(np.float32)
+    prev = None
+    for bpw in (2.0, 3.0, 4.0):
+        bits = int(bpw * N)
+        K = po.max_pulses(N, bits)
+        q = []
+        for amp_mode in (0, 1):
+            c, s, r = po.encode(x, N, K, 16, W=(bits + 31) // 32, amp_mode=amp_mode)
+            out, _ = po.decode(c, s, r, N, K, 16)
+            xh = inputs.bf16_bits_to_f32(out).astype(np.float64)
+            q.append(10 * np.log10((x.astype(np.float64) ** 2).sum() / ((x - xh) ** 2).sum()))
+        assert q[1] >= q[0] - 1e-9
+        assert 6.02 * bpw - 2.6 < q[0] < 6.02 * (bpw + 16.0 / N)
+        if prev is not None:
+            assert 5.0 < q[0] - prev < 8.0          # per extra bit
+        prev = q[0]
