@@ -230,56 +230,98 @@ class GpuRun:
                for j, (name, _) in enumerate(phases)}
         return total_ms, per
 
+    def _new_set(self):
+        """One more device buffer set (the end-to-end leg wants at least two to overlap steps)."""
+        torch, pvq, wl = self.torch, self.pvq, self.wl
+        items = []
+        for m, h in zip(wl.matrices, self.host):
+            G = m.cols // wl.N
+            codes, sidx, rnorm = pvq.alloc_encoded(m.rows, G, self.W, wl.scale_bits, self.dev)
+            edges, levels = self.books[G]
+            items.append(dict(x=torch.empty_like(h, device=self.dev), codes=codes, scale_idx=sidx, row_norm=rnorm,
+                              edges=edges, levels=levels, cols=m.cols,
+                              out=torch.empty((m.rows, m.cols), dtype=torch.bfloat16, device=self.dev)))
+        return items
+
     def run_e2e(self, steps, warmup):
-        """Same step from pinned HOST buffers: H2D of the inputs and D2H of the results inside the
-        timed region.  Returns (ms per step, h2d bytes, d2h bytes)."""
+        """The same step from pinned HOST buffers, through the public API: every step copies its
+        inputs host -> device and its results device -> host inside the timed region.  Steps are
+        pipelined as a user streaming matrices through the codec would: copies in, kernels and
+        copies out run on three streams over two or three device buffer sets, so the transfer of
+        one step overlaps the kernels and the opposite transfer of its neighbours.
+        Returns (ms per step, h2d bytes, d2h bytes)."""
         torch = self.torch
-        wl, items = self.wl, self.sets[0]
+        wl = self.wl
+        while len(self.sets) < 2:
+            self.sets.append(self._new_set())
+        sets = self.sets[:3]
+        S = len(sets)
         host_out = [torch.empty((m.rows, m.cols), dtype=torch.bfloat16).pin_memory() for m in wl.matrices]
-        host_codes = [torch.empty_like(it["codes"], device="cpu").pin_memory() for it in items]
-        host_sidx = [torch.empty_like(it["scale_idx"], device="cpu").pin_memory() for it in items]
-        host_rn = [torch.empty_like(it["row_norm"], device="cpu").pin_memory() for it in items]
+        host_codes = [torch.empty_like(it["codes"], device="cpu").pin_memory() for it in sets[0]]
+        host_sidx = [torch.empty_like(it["scale_idx"], device="cpu").pin_memory() for it in sets[0]]
+        host_rn = [torch.empty_like(it["row_norm"], device="cpu").pin_memory() for it in sets[0]]
+        s_main = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = [torch.cuda.Event() for _ in range(S)]
+        ev_comp = [torch.cuda.Event() for _ in range(S)]
+        ev_free = [torch.cuda.Event() for _ in range(S)]
+        used = [False] * S
         h2d = d2h = 0
 
-        def step():
+        def step(i):
             nonlocal h2d, d2h
             h2d = d2h = 0
-            if wl.mode in ("encode+decode", "roundtrip", "rotate_roundtrip"):
-                for it, h in zip(items, self.host):
-                    it["x"].copy_(h, non_blocking=True)
-                    h2d += h.numel() * h.element_size()
-            if wl.mode == "decode":            # the compressed form comes from the host
-                for it, hc, hs, hr in zip(items, host_codes, host_sidx, host_rn):
-                    it["codes"].copy_(hc, non_blocking=True)
-                    it["scale_idx"].copy_(hs, non_blocking=True)
-                    it["row_norm"].copy_(hr, non_blocking=True)
-                    h2d += hc.numel() * 4 + hs.numel() + hr.numel() * 4
+            k = i % S
+            items = sets[k]
+            with torch.cuda.stream(s_in):
+                if used[k]:
+                    s_in.wait_event(ev_free[k])       # the set's previous results have left the device
+                if wl.mode in ("encode+decode", "roundtrip", "rotate_roundtrip"):
+                    for it, h in zip(items, self.host):
+                        it["x"].copy_(h, non_blocking=True)
+                        h2d += h.numel() * h.element_size()
+                if wl.mode == "decode":            # the compressed form comes from the host
+                    for it, hc, hs, hr in zip(items, host_codes, host_sidx, host_rn):
+                        it["codes"].copy_(hc, non_blocking=True)
+                        it["scale_idx"].copy_(hs, non_blocking=True)
+                        it["row_norm"].copy_(hr, non_blocking=True)
+                        h2d += hc.numel() * 4 + hs.numel() + hr.numel() * 4
+                ev_in[k].record(s_in)
+            s_main.wait_event(ev_in[k])
             for _, fn in self.phases():
                 fn(items)
-            if wl.mode == "encode+decode":
-                for it, hc, hs, hr in zip(items, host_codes, host_sidx, host_rn):
-                    hc.copy_(it["codes"], non_blocking=True)
-                    hs.copy_(it["scale_idx"], non_blocking=True)
-                    hr.copy_(it["row_norm"], non_blocking=True)
-                    d2h += hc.numel() * 4 + hs.numel() + hr.numel() * 4
-            for it, ho in zip(items, host_out):
-                ho.copy_(it["out"], non_blocking=True)
-                d2h += ho.numel() * 2
+            ev_comp[k].record(s_main)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_comp[k])
+                if wl.mode == "encode+decode":
+                    for it, hc, hs, hr in zip(items, host_codes, host_sidx, host_rn):
+                        hc.copy_(it["codes"], non_blocking=True)
+                        hs.copy_(it["scale_idx"], non_blocking=True)
+                        hr.copy_(it["row_norm"], non_blocking=True)
+                        d2h += hc.numel() * 4 + hs.numel() + hr.numel() * 4
+                for it, ho in zip(items, host_out):
+                    ho.copy_(it["out"], non_blocking=True)
+                    d2h += ho.numel() * 2
+                ev_free[k].record(s_out)
+            used[k] = True
 
         if wl.mode == "decode":
-            for it, hc, hs, hr in zip(items, host_codes, host_sidx, host_rn):
+            for it, hc, hs, hr in zip(sets[0], host_codes, host_sidx, host_rn):
                 hc.copy_(it["codes"])
                 hs.copy_(it["scale_idx"])
                 hr.copy_(it["row_norm"])
-        for _ in range(warmup):
-            step()
+        for i in range(warmup):
+            step(i)
         torch.cuda.synchronize()
         t0 = torch.cuda.Event(enable_timing=True)
         t1 = torch.cuda.Event(enable_timing=True)
-        t0.record()
-        for _ in range(steps):
-            step()
-        t1.record()
+        t0.record(s_main)
+        s_in.wait_event(t0)
+        for i in range(steps):
+            step(warmup + i)
+        s_main.wait_stream(s_in)
+        s_main.wait_stream(s_out)
+        t1.record(s_main)
         torch.cuda.synchronize()
         return t0.elapsed_time(t1) / steps, h2d, d2h
 
