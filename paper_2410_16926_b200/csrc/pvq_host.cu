@@ -233,7 +233,7 @@ int check_common(int N, int K, int scale_bits, const uint32_t* d_table, Common* 
     if (N < 2 || (N & (N - 1)) != 0 || K < 1) return PVQ_ERR_INVALID_ARG;
     if ((scale_bits < 1 || scale_bits > 8) && scale_bits != 16) return PVQ_ERR_INVALID_ARG;
     if (!d_table) return PVQ_ERR_INVALID_ARG;
-    if (N < 8 || N > 64 || K > kMaxPulses) return PVQ_ERR_UNSUPPORTED;
+    if (N < 8 || N > kMaxGroup || K > kMaxPulses) return PVQ_ERR_UNSUPPORTED;
     int W = code_words_for(N, K);
     if (W == 0) return PVQ_ERR_INVALID_ARG;
     if (W > kMaxWords) return PVQ_ERR_UNSUPPORTED;
@@ -321,6 +321,10 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
         if (st != PVQ_OK) return st;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c.N > 64) {  // large groups: encode and decode only
+        if (kind == 2 || rot_block != 0) return PVQ_ERR_UNSUPPORTED;
+        return launch_big(a, dtype, c.N, c.W, kind == 1, s);
+    }
     if (kind == 1) return launch_decode(a, c.N, c.W, s);
     return launch_encode(a, dtype, c.N, c.W, kind == 2, s);
 }

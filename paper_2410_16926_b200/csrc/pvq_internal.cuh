@@ -13,6 +13,7 @@ namespace pvq {
 
 constexpr int kMaxBatch = 32;     // matrices per launch
 constexpr int kMaxWords = 12;     // limbs per code the kernels are instantiated for
+constexpr int kMaxGroup = 128;    // largest group size; above 64 (or 6 limbs) the tables stay in global memory
 constexpr int kMaxPulses = 1023;  // table builder: one thread per k
 
 // One matrix as the kernels see it.
@@ -54,7 +55,7 @@ struct BatchArgs {
 // [n][k][W] words for n = 0..N-1, k = 0..K.  The other sections are the same numbers
 // rearranged for the kernels, so that a thread block can stage them with one flat copy:
 //
-//   bound       N(N,K) as 8 words (codes are valid below it)
+//   bound       N(N,K) as 16 words (codes are valid below it)
 //   walk[0]     rows by position i (row i holds N(N-1-i, .)), `rowlen` entries of
 //               `top_words` words each, entry (i, col) = N(N-1-i, col), zero padded
 //   walk[1]     same with 2-word entries, values from 2^62 up replaced by 2^62 (present when
@@ -85,7 +86,7 @@ struct TableLayout {
 
 __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
     TableLayout L;
-    if (N > 64 || W > 6) {  // no hot-path kernel for these: the blob is the plain count table
+    if (N > 128 || W > 12) {  // no kernel for these: the blob is the plain count table
         L.rowlen = 0;
         L.top_words = 0;
         L.bound_off = 0;
@@ -95,7 +96,7 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
         return L;
     }
     L.rowlen = (K + 2) & ~1;
-    L.top_words = W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : W));
+    L.top_words = W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : (W <= 8 ? 8 : 12)));
     uint32_t off = static_cast<uint32_t>(N) * (K + 1) * W * 4u;
     off = (off + 127u) & ~127u;
     L.bound_off = off;
@@ -133,6 +134,8 @@ int prepare_kernel(const void* kern, int threads, size_t smem, int* blocks_per_s
 
 // launchers (one per kernel family); all return a pvq_status
 int launch_decode(const BatchArgs& args, int N, int W, cudaStream_t stream);
+// large groups / wide codes (N = 128 or more than 6 words): tables in global memory
+int launch_big(const BatchArgs& args, int dtype, int N, int W, bool decode, cudaStream_t stream);
 int launch_encode(const BatchArgs& args, int dtype, int N, int W, bool fused, cudaStream_t stream);  // rotates when args.rot_block != 0
 
 // ---------------------------------------------------------------- device bits

@@ -144,13 +144,13 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         // N(N,K) = N(N-1,K) + 2 sum_{j=1..K} N(N-1,K-j)   (every point of P(N,K) by its first
         // coordinate: 0, or +-j with K-j pulses left for the other N-1)
-        uint32_t acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        uint32_t acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
         const uint32_t* row = blob + static_cast<size_t>(N - 1) * KP * W;
         for (int col = 0; col <= K; ++col) {
             const int times = col == K ? 1 : 2;
             for (int rep = 0; rep < times; ++rep) {
                 unsigned long long carry = 0;
-                for (int w = 0; w < 8; ++w) {
+                for (int w = 0; w < 16; ++w) {
                     const unsigned long long add = w < W ? row[col * W + w] : 0u;
                     const unsigned long long sum = static_cast<unsigned long long>(acc[w]) + add + carry;
                     acc[w] = static_cast<uint32_t>(sum);
@@ -158,7 +158,7 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
                 }
             }
         }
-        for (int w = 0; w < 8; ++w) blob[L.bound_off / 4 + w] = acc[w];
+        for (int w = 0; w < 16; ++w) blob[L.bound_off / 4 + w] = acc[w];
     }
 }
 

@@ -81,7 +81,7 @@ def _blob_layout(N, K, W):
     """Byte offsets of the sections that follow the count table (see include/pvq.h)."""
     up = lambda v: (v + 127) & ~127
     rowlen = (K + 2) & ~1
-    top = W if W <= 2 else (4 if W <= 4 else 6)
+    top = W if W <= 2 else (4 if W <= 4 else (6 if W <= 6 else (8 if W <= 8 else 12)))
     off = up(N * (K + 1) * W * 4)
     lay = {"bound": off, "rowlen": rowlen, "top": top}
     off += 128
@@ -95,7 +95,7 @@ def _blob_layout(N, K, W):
     return lay
 
 
-@pytest.mark.parametrize("N,K", [(8, 16), (16, 18), (32, 22), (32, 50), (32, 105), (64, 96), (64, 26)])
+@pytest.mark.parametrize("N,K", [(8, 16), (16, 18), (32, 22), (32, 50), (32, 105), (64, 96), (64, 26), (128, 40)])
 def test_table_blob_sections(N, K):
     """Every rearranged section of the table blob holds the numbers of the count table."""
     W = pvq.code_words(N, K)
@@ -107,7 +107,7 @@ def test_table_blob_sections(N, K):
     val = [[po.code_to_int(full[n, k]) for k in range(K + 1)] for n in range(N + 1)]
     mask = (1 << (32 * W)) - 1
     words = lambda v, nw: [(v >> (32 * w)) & 0xFFFFFFFF for w in range(nw)]
-    assert list(blob[lay["bound"] // 4: lay["bound"] // 4 + 8]) == words(val[N][K], 8)
+    assert list(blob[lay["bound"] // 4: lay["bound"] // 4 + 16]) == words(val[N][K], 16)
     rowlen, top = lay["rowlen"], lay["top"]
     for name, sat_bits in (("walk_top", None), ("walk2", 62), ("walk1", 30)):
         off, nw = lay[name]
@@ -410,3 +410,41 @@ def test_qsnr_curve_on_a_gaussian_source_equals_the_oracles():
         assert abs(q_gpu - q_cpu) < 1e-9
         curve.append(q_gpu)
     assert curve[0] < curve[1] < curve[2] and 9.5 < curve[0] < 10.5
+
+
+# ------------------------------------------------------------ large groups (N = 128)
+
+@pytest.mark.parametrize("bits,rows,cols,b,amp_mode,kind", [
+    (384, 9, 4096, 16, 0, "bf16"),      # the paper's 3 bits + 16-bit amplitudes at group size 128
+    (384, 5, 14336, 16, 1, "bf16"),     # G = 112, least-squares amplitudes
+    (256, 7, 1024, 8, 0, "f32"),        # 8-word codes, quantile amplitudes
+    (96, 6, 512, 4, 0, "f32"),          # few pulses: K below 128, byte slots
+])
+def test_large_group_parity(bits, rows, cols, b, amp_mode, kind):
+    N = 128
+    rng = np.random.default_rng(bits + rows)
+    x = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    x[1, :N] = 0.0
+    x[2, N:2 * N] = np.round(x[2, N:2 * N] * 200) / 200            # many equal magnitudes: ties
+    x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+    G = cols // N
+    K = pvq.max_pulses(N, bits)
+    W = pvq.code_words(N, K)
+    table = pvq.build_count_table(N, K)
+    e_np = bc.edges_f32(N, G, b) if b <= 8 else None
+    l_np = bc.levels_amp_f32(N, G, b) if b <= 8 else None
+    edges = torch.from_numpy(e_np).to(DEV) if b <= 8 else None
+    levels = torch.from_numpy(l_np).to(DEV) if b <= 8 else None
+    o_codes, o_sidx, o_rnorm = po.encode(x_np, N, K, b, e_np, W=W, amp_mode=amp_mode)
+    o_out, _ = po.decode(o_codes, o_sidx, o_rnorm, N, K, b, l_np)
+    codes, sidx, rnorm = pvq.encode(to_device(x_np, kind), N, K, b, table, edges, amp_mode=amp_mode)
+    torch.cuda.synchronize()
+    assert np.array_equal(rnorm.cpu().numpy().view(np.uint32), o_rnorm.view(np.uint32)), "row norms"
+    assert np.array_equal(sidx.cpu().numpy(), o_sidx), "amplitudes"
+    bad = np.argwhere(as_u32(codes) != o_codes)
+    assert bad.size == 0, "codes differ first at %s" % (bad[0],)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = pvq.decode(codes, sidx, rnorm, N, K, b, table, levels, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert np.array_equal(bf16_bits(out), o_out), "decoded"

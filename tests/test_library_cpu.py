@@ -90,7 +90,7 @@ def test_bad_arguments_are_rejected_without_a_gpu():
     assert enc(dt=7) == INVALID
     assert enc(ld=32) == INVALID            # ld < cols
     assert enc(cols=32, ld=32) == UNSUPPORTED   # one group per row: no quantile codebook
-    assert enc(N=128, cols=256, ld=256) == UNSUPPORTED
+    assert enc(N=256, cols=512, ld=512) == UNSUPPORTED
     assert enc(ld=68) == ALIGN
     assert enc(x=C.c_void_p(p.value + 2)) == ALIGN
     assert enc(tab=None) == INVALID
