@@ -88,7 +88,7 @@ def algorithmic_bytes(wl, direction):
 def make_workload(name):
     from paper_2410_16926_b200 import inputs
     return {"c1": inputs.config1, "c2": inputs.config2, "c3": inputs.config3, "c4": inputs.config4,
-            "c5": inputs.config5, "c5r": inputs.config5_unrotated}[name]()
+            "c5": inputs.config5, "c5r": inputs.config5_unrotated, "c6": inputs.config6}[name]()
 
 
 # ------------------------------------------------------------------------ clocks
@@ -159,8 +159,8 @@ class GpuRun:
         self.books = {}
         for m in wl.matrices:
             G = m.cols // N
-            if G not in self.books:
-                self.books[G] = pvq.build_scale_codebook(N, G, b, device)
+            if G not in self.books:      # 16-bit amplitudes use no codebook
+                self.books[G] = pvq.build_scale_codebook(N, G, b, device) if b <= 8 else (None, None)
         per_set = algorithmic_bytes(wl, "encode") + algorithmic_bytes(wl, "decode")
         self.nsets = max(1, min(16, -(-3 * L2_BYTES // per_set)))
         self.host = [self._host_tensor(m) for m in wl.matrices]
@@ -340,7 +340,7 @@ def oracle_sample(wl, target_seconds=12.0):
     for m in wl.matrices:
         G = m.cols // N
         if G not in books:
-            books[G] = (bc.edges_f32(N, G, b), bc.levels_amp_f32(N, G, b))
+            books[G] = (bc.edges_f32(N, G, b), bc.levels_amp_f32(N, G, b)) if b <= 8 else (None, None)
 
     def run(frac_rows):
         nbytes, t = 0, 0.0
@@ -396,7 +396,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c5r"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c5r", "c6"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

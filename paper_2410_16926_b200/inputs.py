@@ -163,3 +163,10 @@ def config5_unrotated(tokens=16384, hidden=4096) -> Workload:
     signs = _signs(rng, hidden)
     return Workload("c5r_bf16_activations_rotated_on_the_fly", 32, 64, 8, "rotate_roundtrip",
                     [Matrix("act", f32_to_bf16_bits(x), "bf16")], rot_block=hidden, signs=signs)
+
+
+def config6(rows=4096, cols=4096) -> Workload:
+    """The paper's weight-only setting of Sec. 4.1 on config2's matrix: group size 128, 3 bits per
+    weight of direction (384-bit codes, K = 187) and 16-bit amplitudes, 3.125 bits per weight."""
+    wl = config2(rows, cols)
+    return Workload("c6_bf16_q_proj_group128", 128, 384, 16, "encode+decode", wl.matrices)

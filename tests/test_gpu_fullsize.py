@@ -155,3 +155,25 @@ def test_c5r_activations_rotated_on_the_fly_sampled_rows():
     o_out, st = po.decode(*enc, wl.N, K, wl.scale_bits, it["l_np"])
     r = torch.from_numpy(rows).to(DEV)
     assert st == 0 and np.array_equal(bf16_bits(it["out"][r].contiguous()), o_out)
+
+
+def test_c6_group_128_sampled_rows():
+    wl = inputs.config6()
+    K = pvq.max_pulses(wl.N, wl.index_bits)
+    W = pvq.code_words(wl.N, K)
+    assert (K, W) == (187, 12)
+    table = pvq.build_count_table(wl.N, K)
+    m = wl.matrices[0]
+    G = m.cols // wl.N
+    x = dev_bf16(m.data)
+    codes, sidx, rnorm = pvq.encode(x, wl.N, K, 16, table, None)
+    out = pvq.decode(codes, sidx, rnorm, wl.N, K, 16, table, None)
+    torch.cuda.synchronize()
+    rows = sample_rows(m.rows, 128, seed=66)
+    o_codes, o_sidx, o_rnorm = po.encode(np.ascontiguousarray(m.data[rows]), wl.N, K, 16, W=W)
+    o_out, st = po.decode(o_codes, o_sidx, o_rnorm, wl.N, K, 16)
+    r = torch.from_numpy(rows).to(DEV)
+    assert st == 0
+    assert np.array_equal(codes[r].cpu().numpy().view(np.uint32), o_codes)
+    assert np.array_equal(sidx[r].cpu().numpy(), o_sidx)
+    assert np.array_equal(bf16_bits(out[r].contiguous()), o_out)
