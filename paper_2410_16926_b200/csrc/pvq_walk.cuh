@@ -336,6 +336,59 @@ __device__ __forceinline__ void walk_step_w6(uint32_t (&r)[6], uint32_t& p, int&
           "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
+// Middle phase for 5- and 6-word codes: once every r of the warp is below 2^126 the steps work
+// on four words (sign-bit compares) while still reading the 24-byte entries; an entry that
+// does not fit 126 bits is larger than any such r and fails its test.
+template <typename YT, int U>
+__device__ __forceinline__ void walk_step_4of6(mp<4>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                               const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, t2, t3, t4, t5, a0, a1, a2, a3, b0, b1, b2, b3, big, xh, val;\n\t"
+        "ld.shared.v2.u32 {t0, t1}, [%6+%10];\n\t"
+        "ld.shared.v2.u32 {t2, t3}, [%6+%11];\n\t"
+        "ld.shared.v2.u32 {t4, t5}, [%6+%12];\n\t"
+        "or.b32 big, t4, t5;\n\t"
+        "shr.u32 xh, t3, 30;\n\t"
+        "or.b32 big, big, xh;\n\t"             // non-zero: the entry is 2^126 or more
+        "sub.cc.u32 a0, %0, t0;\n\t"
+        "subc.cc.u32 a1, %1, t1;\n\t"
+        "subc.cc.u32 a2, %2, t2;\n\t"
+        "subc.u32 a3, %3, t3;\n\t"
+        "sub.cc.u32 b0, a0, t0;\n\t"
+        "subc.cc.u32 b1, a1, t1;\n\t"
+        "subc.cc.u32 b2, a2, t2;\n\t"
+        "subc.u32 b3, a3, t3;\n\t"
+        "setp.gt.s32 pl, %4, 0;\n\t"
+        "setp.ge.s32 g1, a3, 0;\n\t"
+        "setp.eq.and.u32 g1, big, 0, g1;\n\t"
+        "selp.u32 xh, b3, a3, pl;\n\t"
+        "setp.ge.and.s32 mo, xh, 0, g1;\n\t"
+        "and.pred ng, g1, pl;\n\t"
+        "and.pred m2, mo, pl;\n\t"
+        "@g1 mad.lo.u32 %0, a0, %7, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %7, 0;\n\t"
+        "@g1 mad.lo.u32 %2, a2, %7, 0;\n\t"
+        "@g1 mad.lo.u32 %3, a3, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %2, b2, %7, 0;\n\t"
+        "@m2 mad.lo.u32 %3, b3, %7, 0;\n\t"
+        "mad.lo.u32 val, %4, %7, %15;\n\t"
+        "@ng mad.lo.u32 val, %4, %8, %15;\n\t"
+        "st.shared.u%14 [%5], val;\n\t"
+        "@!mo add.u32 %5, %5, %13;\n\t"
+        "@!mo add.u32 %6, %6, %9;\n\t"
+        "mad.lo.u32 %4, %4, %7, %7;\n\t"
+        "@!mo mov.u32 %4, 0;\n\t"
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(r.w[3]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 24), "n"(-U * 24 + 8), "n"(-U * 24 + 16), "n"(SZ),
+          "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
 #undef PVQ_WIDE_TAIL
 
 template <int PW, int EB, bool HEADROOM, typename YT, int U>
@@ -345,6 +398,8 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
         walk_step_1<EB, YT, U>(r.w[0], p, v, y, D, f);
     else if constexpr (HEADROOM && PW == 2)
         walk_step_2<EB, YT, U>(r, p, v, y, D, f);
+    else if constexpr (HEADROOM && PW == 4 && EB == 24)
+        walk_step_4of6<YT, U>(r, p, v, y, D, f);
     else if constexpr (!HEADROOM && PW == 3)
         walk_step_w3<YT, U>(r, p, v, y, D, f);
     else if constexpr (!HEADROOM && PW == 4)
@@ -377,12 +432,18 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
 
     while (s + 8 <= S) {
         if (next_words > 0) {
-            // does r fit next_words words with the two top bits clear?
+            // does r fit next_words (4, 2 or 1) words with the two top bits clear?
             uint32_t hi = 0;
 #pragma unroll
-            for (int w = 2; w < PW; ++w) hi |= r.w[w];
-            if constexpr (PW > 1) hi |= next_words == 2 ? (r.w[1] >> 30) : r.w[1];
-            if (next_words == 1) hi |= r.w[0] >> 30;
+            for (int w = 4; w < PW; ++w) hi |= r.w[w];
+            if (next_words == 4) {
+                if constexpr (PW > 3) hi |= r.w[3] >> 30;
+            } else {
+#pragma unroll
+                for (int w = 2; w < PW && w < 4; ++w) hi |= r.w[w];
+                if constexpr (PW > 1) hi |= next_words == 2 ? (r.w[1] >> 30) : r.w[1];
+                if (next_words == 1) hi |= r.w[0] >> 30;
+            }
             if (__all_sync(kFull, hi == 0u)) break;
         }
         walk_step<PW, EB, HEADROOM, YT, 0>(r, p, v, y, D, f);
@@ -454,7 +515,11 @@ __device__ __forceinline__ void walk_code(mp<W>& c, const WalkTables& t, int K, 
     st.v = 0;
     st.y = st.y0 = shared_addr(yslots);
     int s = 0;
-    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, t.has2 ? 2 : (t.has1 ? 1 : 0), t.f);
+    const int narrow = t.has2 ? 2 : (t.has1 ? 1 : 0);
+    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, W > 4 ? 4 : narrow, t.f);
+    if constexpr (W > 4) {  // four-word arithmetic on the same table
+        if (s < S) s = walk_phase<4, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
+    }
     if constexpr (W > 2) {
         if (s < S && t.has2) s = walk_phase<2, 8, true, W, YT>(c, st, t.tab2, t.rowlen, K, s, S, t.has1 ? 1 : 0, t.f);
     }
