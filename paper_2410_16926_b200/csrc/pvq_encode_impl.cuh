@@ -386,7 +386,9 @@ __device__ __forceinline__ TileLoc locate(const BatchArgs& a, unsigned tile) {
 //
 // ROT: the tile is first rotated (rotate_tile); the kernel then works on the rotated fp32
 // values, whatever type the input has.
-template <int N, int W, bool FUSED, typename YT, bool BF16, bool ROT>
+// LS: the least-squares amplitude of Step 4 (a kernel of its own: its extra live values would
+// otherwise cost the common path registers).
+template <int N, int W, bool FUSED, typename YT, bool BF16, bool ROT, bool LS>
 __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ BatchArgs a,
                                                       const __grid_constant__ EncodeSmem sm) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -530,7 +532,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
         // Step 4 as least squares: the amplitude is the projection of x on the chosen direction,
         // a = (sum |y_i| |x_i|) / sqrt(sum y_i^2), the sum of the rounded products by the fixed tree
         float ls_amp = 0.0f;
-        if (a.amp_mode == 1) {
+        if constexpr (LS) {
             float t[N];
             float ssy = 0.0f;
 #pragma unroll
@@ -584,11 +586,11 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             const float ss_row = s_ss[rl * gp];
             rnorm = __fsqrt_rn(ss_row);
             if (b == 16) {  // the amplitude itself, as binary16
-                const float amp16 = a.amp_mode == 1 ? ls_amp : __fsqrt_rn(ss);
+                const float amp16 = LS ? ls_amp : __fsqrt_rn(ss);
                 q = __half_as_ushort(__float2half_rn(amp16));
             } else {
                 // Step 5: q = floor(CDF(u) 2^b) as the number of bin edges <= u
-                const float amp2 = a.amp_mode == 1 ? __fmul_rn(ls_amp, ls_amp) : ss;
+                const float amp2 = LS ? __fmul_rn(ls_amp, ls_amp) : ss;
                 const float u = ss_row > 0.0f ? __fdiv_rn(amp2, ss_row) : 0.0f;
                 for (int step = 1 << (b - 1); step >= 1; step >>= 1)
                     if (s_edges[q + step - 1] <= u) q += step;
@@ -631,7 +633,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     }
 }
 
-template <int N, int W, bool FUSED, typename YT, bool BF16, bool ROT>
+template <int N, int W, bool FUSED, typename YT, bool BF16, bool ROT, bool LS = false>
 static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
     // Block size: a multiple of 32 that wastes the fewest thread slots over the batch.
@@ -723,7 +725,7 @@ static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
     const size_t smem = sm.wbuf_off + wbufs;
     if (smem > static_cast<size_t>(smem_max)) return PVQ_ERR_UNSUPPORTED;
 
-    auto kern = encode_kernel<N, W, FUSED, YT, BF16, ROT>;
+    auto kern = encode_kernel<N, W, FUSED, YT, BF16, ROT, LS>;
     int per_sm = 0;
     if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
@@ -735,6 +737,10 @@ static int launch_encode_t(BatchArgs& a, cudaStream_t stream) {
 
 template <int N, int W, bool BF16>
 static int launch_encode_nwb(BatchArgs& a, bool fused, cudaStream_t s) {
+    if (a.amp_mode == 1) {  // least squares: the plain encoder only
+        if (fused || a.rot_block != 0) return PVQ_ERR_UNSUPPORTED;
+        return launch_encode_t<N, W, false, int8_t, BF16, false, true>(a, s);
+    }
     if (a.rot_block != 0) {  // rotating kernels are built for byte-sized slots only (K <= 127)
         if (!fused) return launch_encode_t<N, W, false, int8_t, BF16, true>(a, s);
         if (a.K <= 127) return launch_encode_t<N, W, true, int8_t, BF16, true>(a, s);
