@@ -38,9 +38,9 @@ FALLBACK_HBM_GBS = 6650.0
 # workload and launch configuration as this bench): DRAM bytes read + written, and warp
 # instructions executed.  Set an entry to None when its kernel changes until it is re-captured.
 NCU_COUNTERS = {
-    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_967_104 + 5_376, "warp_inst": 32_381_488},
-    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_651_136 + 5_120, "warp_inst": 40_036_062},
-    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_499_584 + 89_775_872, "warp_inst": 218_715_576},
+    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_968_384 + 2_816, "warp_inst": 32_554_608},
+    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_651_648 + 1_280, "warp_inst": 40_134_366},
+    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_529_536 + 89_149_440, "warp_inst": 219_689_144},
 }
 SMS, SCHEDULERS_PER_SM = 148, 4      # issue slots per cycle on the part = SMS * SCHEDULERS_PER_SM
 
@@ -366,8 +366,14 @@ def oracle_sample(wl, target_seconds=12.0):
     nb, t = run(probe)
     frac = min(1.0, probe * target_seconds / max(t, 1e-4))
     nb, t = run(frac)
+    reps = 1
+    if frac >= 1.0 and t < target_seconds / 4:       # the whole workload is quick: repeat it for a steadier figure
+        reps = int(min(20, max(1, target_seconds / 4 / max(t, 1e-4))))
+        for _ in range(reps - 1):
+            nb2, t2 = run(frac)
+            nb, t = nb + nb2, t + t2
     rows = [max(1, min(m.rows, int(round(m.rows * frac)))) for m in wl.matrices]
-    return nb / t / 1e9, po.threads(), "first %s rows of each matrix, %.1f s" % (rows, t), nb, t
+    return nb / t / 1e9, po.threads(), "first %s rows of each matrix, %d pass(es), %.1f s" % (rows, reps, t), nb, t
 
 
 # ----------------------------------------------------------------- over the ranks
