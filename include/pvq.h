@@ -77,6 +77,9 @@ typedef enum {
 
 /* bit 0 of the decode status word: some code was >= N(N,K) */
 #define PVQ_STATUS_INVALID_CODE 1u
+/* bit 1: a thread block gave up waiting for its tables to arrive in shared memory and wrote
+ * nothing (a bounded wait; not expected to happen) */
+#define PVQ_STATUS_STAGING_TIMEOUT 2u
 
 typedef void* pvq_stream_t; /* a cudaStream_t */
 

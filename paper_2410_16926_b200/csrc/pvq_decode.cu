@@ -24,10 +24,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
     const TableLayout L = table_layout(N, K, W);
     const uint32_t tab_bytes = walk_tables_bytes(L, a.walk_phases);
 
-    {   // stage the walk tables: one flat copy
-        const uint4* src = reinterpret_cast<const uint4*>(reinterpret_cast<const uint8_t*>(a.table) + L.walk_off[0]);
-        uint4* dst = reinterpret_cast<uint4*>(smem);
-        for (uint32_t q = threadIdx.x; q < tab_bytes / 16; q += blockDim.x) dst[q] = src[q];
+    // stage the walk tables: one flat bulk copy, waited for below
+    __shared__ uint64_t stage_bar;
+    const BulkStage stage = bulk_stage_begin(&stage_bar);
+    if (threadIdx.x == 0) {
+        bulk_stage_expect(stage, tab_bytes);
+        bulk_stage_copy(stage, smem, reinterpret_cast<const uint8_t*>(a.table) + L.walk_off[0], tab_bytes);
     }
     const WalkTables wt = walk_tables(L, shared_addr(smem), a.walk_phases, a);
 
@@ -41,7 +43,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
 #pragma unroll
     for (int w = 0; w < W; ++w) bound.w[w] = bw[w];
     const bool bound_wide = bw[W] != 0u;  // N(N,K) = 2^(32W) exactly: every W-word code is valid
-    __syncthreads();
+    if (!bulk_stage_wait(stage)) {  // the tables never arrived: report and leave
+        if (a.status && threadIdx.x == 0) atomicOr(a.status, PVQ_STATUS_STAGING_TIMEOUT);
+        return;
+    }
 
     const unsigned b = a.scale_bits;
     const unsigned warps_total = gridDim.x * (blockDim.x >> 5);

@@ -423,18 +423,17 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     const int warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
 
-    {   // stage the tables
+    // stage the tables with bulk copies; they land while the first tile's input is requested
+    __shared__ uint64_t stage_bar;
+    const BulkStage stage = bulk_stage_begin(&stage_bar);
+    if (threadIdx.x == 0) {
         const uint8_t* blob = reinterpret_cast<const uint8_t*>(a.table);
-        const uint4* src = reinterpret_cast<const uint4*>(blob + (sm.enum_mode == 2 ? L.enc_off[0] : L.enc_off[2]));
-        uint4* dst = reinterpret_cast<uint4*>(smem);
-        for (uint32_t q = threadIdx.x; q < sm.enc_bytes / 16; q += blockDim.x) dst[q] = src[q];
-        if constexpr (FUSED) {
-            const uint4* wsrc = reinterpret_cast<const uint4*>(blob + L.walk_off[0]);
-            uint4* wdst = reinterpret_cast<uint4*>(smem + sm.enc_bytes);
-            for (uint32_t q = threadIdx.x; q < sm.walk_bytes / 16; q += blockDim.x) wdst[q] = wsrc[q];
-        }
-        for (int i = threadIdx.x; i < 2 * sm.idx_words; i += blockDim.x) s_idx2[i] = 0u;
+        bulk_stage_expect(stage, sm.enc_bytes + (FUSED ? sm.walk_bytes : 0u));
+        if (sm.enc_bytes)
+            bulk_stage_copy(stage, smem, blob + (sm.enum_mode == 2 ? L.enc_off[0] : L.enc_off[2]), sm.enc_bytes);
+        if constexpr (FUSED) bulk_stage_copy(stage, smem + sm.enc_bytes, blob + L.walk_off[0], sm.walk_bytes);
     }
+    for (int i = threadIdx.x; i < 2 * sm.idx_words; i += blockDim.x) s_idx2[i] = 0u;
     const uint32_t tabA = shared_addr(smem);
     const uint32_t tabB = tabA + ((L.enc_bytes + 127u) & ~127u);  // 2V, when two tables are staged
     const int rowbytes = (K + 2) * EB;
@@ -456,7 +455,8 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
         const MatrixArgs& m0 = a.m[loc.mi];
         load_raw<N, BF16>(m0.x, static_cast<size_t>(loc.row0 + loc.rl) * m0.ld + static_cast<size_t>(loc.g) * N, pre);
     }
-    __syncthreads();  // tables staged, index words cleared
+    if (!bulk_stage_wait(stage)) return;  // the tables never arrived: leave rather than spin
+    __syncthreads();                      // index words cleared
 
     for (int buf = 0;; buf ^= 1) {
         const MatrixArgs& m = a.m[loc.mi];

@@ -101,6 +101,7 @@ int device_info(DeviceInfo* out) {
             return set_cuda_error(e);
         if ((e = cudaDeviceGetAttribute(&d.smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
             return set_cuda_error(e);
+        d.smem_max -= 256;  // room for the kernels' few bytes of static shared memory (an mbarrier)
         it = memo.emplace(dev, d).first;
     }
     *out = it->second;

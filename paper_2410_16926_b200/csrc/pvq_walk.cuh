@@ -35,6 +35,60 @@ __device__ __forceinline__ uint32_t shared_addr(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// Table staging with the bulk-copy engine (TMA, untiled form): thread 0 arms an mbarrier with
+// the byte count and issues the copies, global -> shared; the data lands while the block does
+// its other set-up, and every thread waits on the barrier before the first table read.
+// Source, destination and sizes are multiples of 16 bytes (the table blob's sections are
+// 128-byte aligned, the staged region starts the dynamic shared memory).
+struct BulkStage {
+    uint32_t bar;  // shared address of the mbarrier
+};
+
+__device__ __forceinline__ BulkStage bulk_stage_begin(uint64_t* bar_storage) {
+    BulkStage st;
+    st.bar = shared_addr(bar_storage);
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(st.bar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    return st;
+}
+
+// thread 0 only: announce `total` bytes, then copy the pieces with bulk_stage_copy
+__device__ __forceinline__ void bulk_stage_expect(const BulkStage& st, uint32_t total) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(st.bar), "r"(total) : "memory");
+}
+
+__device__ __forceinline__ void bulk_stage_copy(const BulkStage& st, void* dst, const void* src, uint32_t bytes) {
+    const uint32_t d = shared_addr(dst);
+    const uint8_t* s = static_cast<const uint8_t*>(src);
+    for (uint32_t off = 0; off < bytes; off += 32768u) {
+        const uint32_t n = bytes - off < 32768u ? bytes - off : 32768u;
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(d + off),
+                     "l"(s + off), "r"(n), "r"(st.bar)
+                     : "memory");
+    }
+}
+
+// every thread: true once the announced bytes have arrived; false if they have not after a
+// bounded number of polls (the caller then leaves the kernel instead of spinning)
+__device__ __forceinline__ bool bulk_stage_wait(const BulkStage& st) {
+    uint32_t done = 0;
+    for (int it = 0; it < (1 << 22) && !done; ++it) {
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(done)
+            : "r"(st.bar)
+            : "memory");
+    }
+    return done != 0u;
+}
+
 // Entry of PW words at shared address addr + OFF (OFF a compile-time byte offset).
 template <int PW, int OFF = 0>
 __device__ __forceinline__ mp<PW> load_entry(uint32_t addr) {
