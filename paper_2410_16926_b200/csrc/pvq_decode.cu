@@ -5,6 +5,7 @@
 // codes in lockstep (pvq_walk.cuh), each thread collecting its point in shared
 // memory, from where it scales it and writes its N bf16 values with 16-byte stores.
 #include <algorithm>
+#include <cmath>
 
 #include <cuda_fp16.h>
 
@@ -116,25 +117,39 @@ int launch_decode_t(BatchArgs& a, cudaStream_t stream) {
     int st = device_info(&di);
     if (st != PVQ_OK) return st;
     const int sms = di.sms, smem_max = di.smem_max;
-    // As many of the narrower walk tables as fit beside the widest one; fewer threads if even
-    // that leaves no room for their output slots.
-    int threads = kDecThreads;
-    int phases = 0;
+    // Block size: every tile costs the same, so the launch runs in rounds of one tile per
+    // resident warp and the last round is only partly filled.  Among block sizes of 12..16
+    // warps take the one that wastes the fewest warp slots over the rounds (with a small
+    // preference for more warps, which hide latency better); smaller blocks only when the
+    // tables leave no room for more output slots.  With each size go as many of the narrower
+    // walk tables as fit beside the widest one.
+    auto kern = decode_kernel<N, W, YT>;
+    int threads = 0, phases = 0, per_sm = 0;
     size_t smem = 0;
-    for (; threads >= 128; threads -= 32) {
-        const size_t wbufs = static_cast<size_t>(threads) * YS;
-        phases = walk_phases_that_fit(L, static_cast<size_t>(smem_max) - std::min<size_t>(smem_max, wbufs));
-        if (phases) {
-            smem = ((walk_tables_bytes(L, phases) + 15u) & ~size_t(15)) + wbufs;
-            break;
+    double best_score = -1.0;
+    for (int t = kDecThreads; t >= 128; t -= 32) {
+        if (t < 384 && threads != 0) break;
+        const size_t wbufs = static_cast<size_t>(t) * YS;
+        if (wbufs >= static_cast<size_t>(smem_max)) continue;
+        const int ph = walk_phases_that_fit(L, static_cast<size_t>(smem_max) - wbufs);
+        if (ph == 0) continue;
+        const size_t sm_bytes = ((walk_tables_bytes(L, ph) + 15u) & ~size_t(15)) + wbufs;
+        int bps = 0;
+        if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), t, sm_bytes, &bps)) != PVQ_OK) return st;
+        if (bps < 1) continue;
+        const double slots = static_cast<double>(sms) * bps * (t / 32);
+        const double rounds = std::ceil(tiles / slots);
+        const double score = tiles / (rounds * slots) * (1.0 - 0.01 * (kDecThreads - t) / 32);
+        if (score > best_score) {
+            best_score = score;
+            threads = t;
+            phases = ph;
+            per_sm = bps;
+            smem = sm_bytes;
         }
     }
-    if (phases == 0) return PVQ_ERR_UNSUPPORTED;
+    if (threads == 0) return PVQ_ERR_UNSUPPORTED;
     a.walk_phases = phases;
-    auto kern = decode_kernel<N, W, YT>;
-    int per_sm = 0;
-    if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
-    if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
     const unsigned warps_per_block = threads / 32;
     const unsigned blocks_needed = (tiles + warps_per_block - 1) / warps_per_block;
     const unsigned grid = std::max(1u, std::min<unsigned>(blocks_needed, static_cast<unsigned>(sms * per_sm)));
