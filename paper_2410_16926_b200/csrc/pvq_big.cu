@@ -71,6 +71,74 @@ __device__ __forceinline__ int walk_phase_g(mp<CW>& rfull, Walk& st, const uint8
 
 constexpr int kBigThreads = 256;
 
+// ---- bitonic merge of 32 values in registers (v bitonic on entry), descending or ascending
+template <bool DESC, int I, int J>
+__device__ __forceinline__ void merge_cx(float (&v)[32]) {
+    const float hi = fmaxf(v[I], v[J]), lo = fminf(v[I], v[J]);
+    v[I] = DESC ? hi : lo;
+    v[J] = DESC ? lo : hi;
+}
+
+template <bool DESC, int J, int I>
+__device__ __forceinline__ void merge_stage(float (&v)[32]) {  // pairs (i, i + J) for all i with bit J clear
+    if constexpr (I < 32) {
+        if constexpr ((I & J) == 0) merge_cx<DESC, I, I + J>(v);
+        merge_stage<DESC, J, I + 1>(v);
+    }
+}
+
+template <bool DESC>
+__device__ __forceinline__ void merge32(float (&v)[32]) {
+    merge_stage<DESC, 16, 0>(v);
+    merge_stage<DESC, 8, 0>(v);
+    merge_stage<DESC, 4, 0>(v);
+    merge_stage<DESC, 2, 0>(v);
+    merge_stage<DESC, 1, 0>(v);
+}
+
+// Sorts a column of N floats (es[i * T], N a multiple of 64) in descending order: chunks of 32
+// in registers (sorting network, then bitonic merges), the strides of 32 and more between
+// chunks in shared memory.
+template <int N>
+__device__ __forceinline__ void sort_column_desc(float* es, int T) {
+    float v[32];
+    for (int q = 0; q < N / 32; ++q) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] = es[(q * 32 + i) * T];
+        sort_desc<32>(v);
+        if (q & 1) {  // odd chunks ascending: neighbours then form bitonic runs of 64
+#pragma unroll
+            for (int i = 0; i < 32; ++i) es[(q * 32 + i) * T] = v[31 - i];
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) es[(q * 32 + i) * T] = v[i];
+        }
+    }
+    for (int k = 64; k <= N; k <<= 1) {
+        for (int j = k >> 1; j >= 32; j >>= 1) {
+            for (int p = 0; p < N / 2; ++p) {
+                const int i = ((p & ~(j - 1)) << 1) | (p & (j - 1));  // the p-th index with bit j clear
+                const int l = i | j;
+                const float x0 = es[i * T], x1 = es[l * T];
+                const bool desc = (i & k) == 0;
+                const float hi = fmaxf(x0, x1), lo = fminf(x0, x1);
+                es[i * T] = desc ? hi : lo;
+                es[l * T] = desc ? lo : hi;
+            }
+        }
+        for (int q = 0; q < N / 32; ++q) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = es[(q * 32 + i) * T];
+            if (((q * 32) & k) == 0)
+                merge32<true>(v);
+            else
+                merge32<false>(v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) es[(q * 32 + i) * T] = v[i];
+        }
+    }
+}
+
 template <int N, int W, typename YT>
 __global__ void __launch_bounds__(kBigThreads) decode_big_kernel(const __grid_constant__ BatchArgs a) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -276,20 +344,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 has_dir = d >= 0 && d <= N;
             }
             if (has_dir) {
-                // bitonic sort of the column, descending
-                for (int k = 2; k <= N; k <<= 1) {
-                    for (int j = k >> 1; j > 0; j >>= 1) {
-                        for (int q = 0; q < N / 2; ++q) {
-                            const int i = ((q & ~(j - 1)) << 1) | (q & (j - 1));  // the q-th index with bit j clear
-                            const int l = i | j;
-                            const float x0 = es[i * T], x1 = es[l * T];
-                            const bool desc = (i & k) == 0;
-                            const float hi = fmaxf(x0, x1), lo = fminf(x0, x1);
-                            es[i * T] = desc ? hi : lo;
-                            es[l * T] = desc ? lo : hi;
-                        }
-                    }
-                }
+                sort_column_desc<N>(es, T);
                 const float v = d > 0 ? es[(d - 1) * T] : 2.0f;
                 int cnt = 0;
                 for (int i = 0; i < N; ++i) {
