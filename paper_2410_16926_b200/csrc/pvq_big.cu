@@ -251,6 +251,53 @@ __device__ __forceinline__ float group_value(const void* gx, int i) {
         return __ldg(static_cast<const float*>(gx) + i);
 }
 
+// elements 8j .. 8j+7 of this thread's group with 16-byte loads (groups start 16-byte aligned)
+template <bool BF16>
+__device__ __forceinline__ void group_values8(const void* gx, int j, float (&x)[8]) {
+    if constexpr (BF16) {
+        const uint4 q = __ldg(static_cast<const uint4*>(gx) + j);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            x[2 * p] = __uint_as_float(w[p] << 16);
+            x[2 * p + 1] = __uint_as_float(w[p] & 0xffff0000u);
+        }
+    } else {
+        const float4 q0 = __ldg(static_cast<const float4*>(gx) + 2 * j);
+        const float4 q1 = __ldg(static_cast<const float4*>(gx) + 2 * j + 1);
+        x[0] = q0.x, x[1] = q0.y, x[2] = q0.z, x[3] = q0.w;
+        x[4] = q1.x, x[5] = q1.y, x[6] = q1.z, x[7] = q1.w;
+    }
+}
+
+// The low W words of an encoder-table entry (top_words_of(W) words long, so 16-, 8- or
+// 4-byte aligned and never shorter than the words the vector loads touch).
+template <int W>
+__device__ __forceinline__ mp<W> load_enc_entry(const uint8_t* p) {
+    constexpr int TW = top_words_of(W);
+    mp<W> t;
+    if constexpr (TW % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < (W + 3) / 4; ++v) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(p) + v);
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (4 * v + u < W) t.w[4 * v + u] = w[u];
+        }
+    } else if constexpr (TW % 2 == 0) {
+#pragma unroll
+        for (int v = 0; v < (W + 1) / 2; ++v) {
+            const uint2 q = __ldg(reinterpret_cast<const uint2*>(p) + v);
+            t.w[2 * v] = q.x;
+            if (2 * v + 1 < W) t.w[2 * v + 1] = q.y;
+        }
+    } else {
+        t = load_entry_g<W>(p);
+    }
+    return t;
+}
+
 // Encoder for large groups: the steps of encode_kernel with the per-thread arrays (residuals
 // to sort, the point) in shared memory columns es[i * T + t], ms[i * T + t], the input re-read
 // from global memory where it is needed, and the cumulative tables read from global memory.
@@ -300,14 +347,20 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
         // group norms by the balanced tree, run level by level in the es column
         float l1 = 0.0f, ss = 0.0f;
         if (active) {
-            for (int j = 0; j < N / 2; ++j)
-                es[j * T] = __fadd_rn(fabsf(group_value<BF16>(gx, 2 * j)), fabsf(group_value<BF16>(gx, 2 * j + 1)));
+            float x[8];
+            for (int j = 0; j < N / 8; ++j) {
+                group_values8<BF16>(gx, j, x);
+#pragma unroll
+                for (int p = 0; p < 4; ++p) es[(4 * j + p) * T] = __fadd_rn(fabsf(x[2 * p]), fabsf(x[2 * p + 1]));
+            }
             for (int len = N / 4; len >= 1; len >>= 1)
                 for (int j = 0; j < len; ++j) es[j * T] = __fadd_rn(es[2 * j * T], es[(2 * j + 1) * T]);
             l1 = es[0];
-            for (int j = 0; j < N / 2; ++j) {
-                const float x0 = group_value<BF16>(gx, 2 * j), x1 = group_value<BF16>(gx, 2 * j + 1);
-                es[j * T] = __fadd_rn(__fmul_rn(x0, x0), __fmul_rn(x1, x1));
+            for (int j = 0; j < N / 8; ++j) {
+                group_values8<BF16>(gx, j, x);
+#pragma unroll
+                for (int p = 0; p < 4; ++p)
+                    es[(4 * j + p) * T] = __fadd_rn(__fmul_rn(x[2 * p], x[2 * p]), __fmul_rn(x[2 * p + 1], x[2 * p + 1]));
             }
             for (int len = N / 4; len >= 1; len >>= 1)
                 for (int j = 0; j < len; ++j) es[j * T] = __fadd_rn(es[2 * j * T], es[(2 * j + 1) * T]);
@@ -333,12 +386,17 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
             int d = 0;
             if (has_dir) {
                 float sumf = 0.0f;
-                for (int i = 0; i < N; ++i) {
-                    const float av = __fmul_rn(fabsf(group_value<BF16>(gx, i)), gsc);
-                    const float tt = __fadd_rd(av, kMagic);
-                    const float f = __fsub_rn(tt, kMagic);
-                    es[i * T] = __fsub_rn(av, f);
-                    sumf = __fadd_rn(sumf, f);
+                float x[8];
+                for (int j = 0; j < N / 8; ++j) {
+                    group_values8<BF16>(gx, j, x);
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) {
+                        const float av = __fmul_rn(fabsf(x[p]), gsc);
+                        const float tt = __fadd_rd(av, kMagic);
+                        const float f = __fsub_rn(tt, kMagic);
+                        es[(8 * j + p) * T] = __fsub_rn(av, f);
+                        sumf = __fadd_rn(sumf, f);
+                    }
                 }
                 d = K - static_cast<int>(sumf);
                 has_dir = d >= 0 && d <= N;
@@ -347,15 +405,19 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 sort_column_desc<N>(es, T);
                 const float v = d > 0 ? es[(d - 1) * T] : 2.0f;
                 int cnt = 0;
-                for (int i = 0; i < N; ++i) {
-                    const float xi = group_value<BF16>(gx, i);
-                    const float av = __fmul_rn(fabsf(xi), gsc);
-                    const float tt = __fadd_rd(av, kMagic);
-                    const float e = __fsub_rn(av, __fsub_rn(tt, kMagic));
-                    const int one = e >= v ? 1 : 0;
-                    const int mi = __float_as_int(tt) - kMagicBits + one;
-                    ms[i * T] = static_cast<short>(__float_as_int(xi) < 0 ? -mi : mi);
-                    cnt += one;
+                float x[8];
+                for (int j = 0; j < N / 8; ++j) {
+                    group_values8<BF16>(gx, j, x);
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) {
+                        const float av = __fmul_rn(fabsf(x[p]), gsc);
+                        const float tt = __fadd_rd(av, kMagic);
+                        const float e = __fsub_rn(av, __fsub_rn(tt, kMagic));
+                        const int one = e >= v ? 1 : 0;
+                        const int mi = __float_as_int(tt) - kMagicBits + one;
+                        ms[(8 * j + p) * T] = static_cast<short>(__float_as_int(x[p]) < 0 ? -mi : mi);
+                        cnt += one;
+                    }
                 }
                 int excess = cnt - d;
                 for (int i = N - 1; i >= 0 && excess > 0; --i) {  // equal residuals straddle the cut
@@ -374,11 +436,16 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
 
             if (a.amp_mode == 1) {  // least-squares amplitude: tree of |y_i| |x_i| in the es column
                 float ssy = 0.0f;
-                for (int j = 0; j < N / 2; ++j) {
-                    const float m0 = fabsf(static_cast<float>(ms[2 * j * T])), m1 = fabsf(static_cast<float>(ms[(2 * j + 1) * T]));
-                    ssy = __fadd_rn(ssy, __fadd_rn(__fmul_rn(m0, m0), __fmul_rn(m1, m1)));
-                    es[j * T] = __fadd_rn(__fmul_rn(m0, fabsf(group_value<BF16>(gx, 2 * j))),
-                                          __fmul_rn(m1, fabsf(group_value<BF16>(gx, 2 * j + 1))));
+                float x[8];
+                for (int j8 = 0; j8 < N / 8; ++j8) {
+                    group_values8<BF16>(gx, j8, x);
+#pragma unroll
+                    for (int p = 0; p < 4; ++p) {
+                        const int j = 4 * j8 + p;
+                        const float m0 = fabsf(static_cast<float>(ms[2 * j * T])), m1 = fabsf(static_cast<float>(ms[(2 * j + 1) * T]));
+                        ssy = __fadd_rn(ssy, __fadd_rn(__fmul_rn(m0, m0), __fmul_rn(m1, m1)));
+                        es[j * T] = __fadd_rn(__fmul_rn(m0, fabsf(x[2 * p])), __fmul_rn(m1, fabsf(x[2 * p + 1])));
+                    }
                 }
                 for (int len = N / 4; len >= 1; len >>= 1)
                     for (int j = 0; j < len; ++j) es[j * T] = __fadd_rn(es[2 * j * T], es[(2 * j + 1) * T]);
@@ -396,8 +463,8 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 const int k2 = k - abs(y);
                 const uint8_t* ru = tabU + (i * rowwords + static_cast<size_t>(k + 1) * TW) * 4;
                 const uint8_t* rx = (y <= 0 ? tabU : tab2V) + (i * rowwords + static_cast<size_t>(k2 + 1) * TW) * 4;
-                mp_add<W>(plus, load_entry_g<W>(ru));
-                mp_add<W>(minus, load_entry_g<W>(rx));
+                mp_add<W>(plus, load_enc_entry<W>(ru));
+                mp_add<W>(minus, load_enc_entry<W>(rx));
                 k = k2;
             }
             mp_sub_borrow<W>(c, plus, minus);

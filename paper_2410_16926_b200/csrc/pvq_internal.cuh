@@ -73,6 +73,11 @@ struct BatchArgs {
 //                 enc[0]  U(n,col) = V(n,col) + V(n,col-1)
 //                 enc[1]  2 V(n,col)
 //                 enc[2]  V(n,col)
+// words per entry of the widest tables for W-word codes
+__host__ __device__ constexpr int top_words_of(int W) {
+    return W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : (W <= 8 ? 8 : 12)));
+}
+
 struct TableLayout {
     int rowlen;
     int top_words;
@@ -96,7 +101,7 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
         return L;
     }
     L.rowlen = (K + 2) & ~1;
-    L.top_words = W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : (W <= 8 ? 8 : 12)));
+    L.top_words = top_words_of(W);
     uint32_t off = static_cast<uint32_t>(N) * (K + 1) * W * 4u;
     off = (off + 127u) & ~127u;
     L.bound_off = off;
