@@ -238,7 +238,7 @@ int launch_decode_big_t(BatchArgs& a, cudaStream_t stream) {
 // ------------------------------------------------------------------------- encode
 
 struct BigSmem {
-    uint32_t es_off, ms_off, ss_off, edges_off, idx_off;
+    uint32_t es_off, ss_off, edges_off, idx_off;
     int ss_floats, idx_words;
 };
 
@@ -299,7 +299,7 @@ __device__ __forceinline__ mp<W> load_enc_entry(const uint8_t* p) {
 }
 
 // Encoder for large groups: the steps of encode_kernel with the per-thread arrays (residuals
-// to sort, the point) in shared memory columns es[i * T + t], ms[i * T + t], the input re-read
+// to sort, the point) in shared memory columns es[i * T + t], the input re-read
 // from global memory where it is needed, and the cumulative tables read from global memory.
 template <int N, int W, bool BF16>
 __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_constant__ BatchArgs a,
@@ -308,7 +308,12 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
     const int T = blockDim.x;
     const int t = threadIdx.x;
     float* es = reinterpret_cast<float*>(smem + sm.es_off) + t;         // column of this thread, stride T
-    short* ms = reinterpret_cast<short*>(smem + sm.ms_off) + t;
+    // The point lies over the upper half of this thread's es column, two entries to a word: that
+    // half is dead once the cut value has been read from the sorted residuals (the least-squares
+    // tree uses the lower half).
+    auto ms = [es, T](int i) -> short& {
+        return reinterpret_cast<short*>(es + (N / 2 + (i >> 1)) * T)[i & 1];
+    };
     float* s_ss = reinterpret_cast<float*>(smem + sm.ss_off);
     float* s_edges = reinterpret_cast<float*>(smem + sm.edges_off);
     uint32_t* s_idx = reinterpret_cast<uint32_t*>(smem + sm.idx_off);
@@ -404,6 +409,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
             if (has_dir) {
                 sort_column_desc<N>(es, T);
                 const float v = d > 0 ? es[(d - 1) * T] : 2.0f;
+                asm volatile("" ::: "memory");  // the point's column reuses the residuals' memory from here on
                 int cnt = 0;
                 float x[8];
                 for (int j = 0; j < N / 8; ++j) {
@@ -415,7 +421,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                         const float e = __fsub_rn(av, __fsub_rn(tt, kMagic));
                         const int one = e >= v ? 1 : 0;
                         const int mi = __float_as_int(tt) - kMagicBits + one;
-                        ms[(8 * j + p) * T] = static_cast<short>(__float_as_int(x[p]) < 0 ? -mi : mi);
+                        ms(8 * j + p) = static_cast<short>(__float_as_int(x[p]) < 0 ? -mi : mi);
                         cnt += one;
                     }
                 }
@@ -425,13 +431,13 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                     const float av = __fmul_rn(fabsf(xi), gsc);
                     const float tt = __fadd_rd(av, kMagic);
                     if (__fsub_rn(av, __fsub_rn(tt, kMagic)) == v) {
-                        ms[i * T] += __float_as_int(xi) < 0 ? 1 : -1;
+                        ms(i) += __float_as_int(xi) < 0 ? 1 : -1;
                         --excess;
                     }
                 }
             } else {
-                for (int i = 0; i < N; ++i) ms[i * T] = 0;
-                ms[0] = static_cast<short>(K);
+                for (int i = 0; i < N; ++i) ms(i) = 0;
+                ms(0) = static_cast<short>(K);
             }
 
             if (a.amp_mode == 1) {  // least-squares amplitude: tree of |y_i| |x_i| in the es column
@@ -442,7 +448,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
                         const int j = 4 * j8 + p;
-                        const float m0 = fabsf(static_cast<float>(ms[2 * j * T])), m1 = fabsf(static_cast<float>(ms[(2 * j + 1) * T]));
+                        const float m0 = fabsf(static_cast<float>(ms(2 * j))), m1 = fabsf(static_cast<float>(ms(2 * j + 1)));
                         ssy = __fadd_rn(ssy, __fadd_rn(__fmul_rn(m0, m0), __fmul_rn(m1, m1)));
                         es[j * T] = __fadd_rn(__fmul_rn(m0, fabsf(x[2 * p])), __fmul_rn(m1, fabsf(x[2 * p + 1])));
                     }
@@ -459,7 +465,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
             int k = K;
             const size_t rowwords = static_cast<size_t>(K + 2) * TW;
             for (int i = 0; i < N; ++i) {
-                const int y = ms[i * T];
+                const int y = ms(i);
                 const int k2 = k - abs(y);
                 const uint8_t* ru = tabU + (i * rowwords + static_cast<size_t>(k + 1) * TW) * 4;
                 const uint8_t* rx = (y <= 0 ? tabU : tab2V) + (i * rowwords + static_cast<size_t>(k2 + 1) * TW) * 4;
@@ -536,8 +542,7 @@ int launch_encode_big_t(BatchArgs& a, cudaStream_t stream) {
     a.total_tiles = tiles;
     BigSmem sm;
     sm.es_off = 0;
-    sm.ms_off = static_cast<uint32_t>(threads) * N * 4u;
-    sm.ss_off = sm.ms_off + static_cast<uint32_t>(threads) * N * 2u;
+    sm.ss_off = static_cast<uint32_t>(threads) * N * 4u;
     sm.edges_off = sm.ss_off + ss_floats * 4u;
     sm.idx_off = sm.edges_off + 256u * 4u;
     sm.ss_floats = ss_floats;
