@@ -25,6 +25,34 @@ __device__ __forceinline__ mp<PW> load_entry_g(const uint8_t* p) {
     return t;
 }
 
+// The low W words of a table entry in global memory.  Entries are top_words_of(W) words long,
+// so 16-, 8- or 4-byte aligned and never shorter than the words the vector loads touch.
+template <int W>
+__device__ __forceinline__ mp<W> load_entry_v(const uint8_t* p) {
+    constexpr int TW = top_words_of(W);
+    mp<W> t;
+    if constexpr (TW % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < (W + 3) / 4; ++v) {
+            const uint4 q = __ldg(reinterpret_cast<const uint4*>(p) + v);
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (4 * v + u < W) t.w[4 * v + u] = w[u];
+        }
+    } else if constexpr (TW % 2 == 0) {
+#pragma unroll
+        for (int v = 0; v < (W + 1) / 2; ++v) {
+            const uint2 q = __ldg(reinterpret_cast<const uint2*>(p) + v);
+            t.w[2 * v] = q.x;
+            if (2 * v + 1 < W) t.w[2 * v + 1] = q.y;
+        }
+    } else {
+        t = load_entry_g<W>(p);
+    }
+    return t;
+}
+
 // One phase of the decode walk (see pvq_walk.cuh) with the table in global memory.
 template <int PW, int CW, typename YT>
 __device__ __forceinline__ int walk_phase_g(mp<CW>& rfull, Walk& st, const uint8_t* tab, int EB, int rowlen,
@@ -46,7 +74,7 @@ __device__ __forceinline__ int walk_phase_g(mp<CW>& rfull, Walk& st, const uint8
             if (next_words == 1) hi |= r.w[0] >> 30;
             if (__all_sync(kFull, hi == 0u)) break;
         }
-        const mp<PW> t = load_entry_g<PW>(p);
+        const mp<PW> t = load_entry_v<PW>(p);
         mp<PW> d2, d1;
         const bool lt1 = mp_sub_borrow<PW>(d2, r, t);
         const bool lt2 = mp_sub_borrow<PW>(d1, d2, t);
@@ -270,33 +298,6 @@ __device__ __forceinline__ void group_values8(const void* gx, int j, float (&x)[
     }
 }
 
-// The low W words of an encoder-table entry (top_words_of(W) words long, so 16-, 8- or
-// 4-byte aligned and never shorter than the words the vector loads touch).
-template <int W>
-__device__ __forceinline__ mp<W> load_enc_entry(const uint8_t* p) {
-    constexpr int TW = top_words_of(W);
-    mp<W> t;
-    if constexpr (TW % 4 == 0) {
-#pragma unroll
-        for (int v = 0; v < (W + 3) / 4; ++v) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4*>(p) + v);
-            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (4 * v + u < W) t.w[4 * v + u] = w[u];
-        }
-    } else if constexpr (TW % 2 == 0) {
-#pragma unroll
-        for (int v = 0; v < (W + 1) / 2; ++v) {
-            const uint2 q = __ldg(reinterpret_cast<const uint2*>(p) + v);
-            t.w[2 * v] = q.x;
-            if (2 * v + 1 < W) t.w[2 * v + 1] = q.y;
-        }
-    } else {
-        t = load_entry_g<W>(p);
-    }
-    return t;
-}
 
 // Encoder for large groups: the steps of encode_kernel with the per-thread arrays (residuals
 // to sort, the point) in shared memory columns es[i * T + t], the input re-read
@@ -469,8 +470,8 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 const int k2 = k - abs(y);
                 const uint8_t* ru = tabU + (i * rowwords + static_cast<size_t>(k + 1) * TW) * 4;
                 const uint8_t* rx = (y <= 0 ? tabU : tab2V) + (i * rowwords + static_cast<size_t>(k2 + 1) * TW) * 4;
-                mp_add<W>(plus, load_enc_entry<W>(ru));
-                mp_add<W>(minus, load_enc_entry<W>(rx));
+                mp_add<W>(plus, load_entry_v<W>(ru));
+                mp_add<W>(minus, load_entry_v<W>(rx));
                 k = k2;
             }
             mp_sub_borrow<W>(c, plus, minus);
