@@ -34,13 +34,13 @@
  *   count table uint32 pvq_count_table_bytes(N,K) bytes, 16-byte aligned, written by
  *                      pvq_build_count_table.  It opens with the table of the paper,
  *                      table[(n*(K+1) + k)*W + w] = word w of N(n,k) for n = 0..N-1
- *                      (dimensions left after a position) and k = 0..K.  For N <= 128
- *                      and W <= 12 the same numbers follow, rearranged for the kernels
+ *                      (dimensions left after a position) and k = 0..K.  For N <= 256
+ *                      and W <= 32 the same numbers follow, rearranged for the kernels
  *                      (each section starts on a 128-byte boundary, in this order):
- *                        N(N,K) as 16 words;
+ *                        N(N,K) as 16 words (64 words when W > 12);
  *                        the decoder's tables, rows by position i (row i = N(N-1-i, .)),
  *                        K+1 rounded up to even entries per row: one with entries of
- *                        1, 2, 4, 6, 8 or 12 words (the first that holds W), then, when W > 2,
+ *                        1, 2, 4, 6, 8, 12, 16, 20, ... words (the first that holds W), then, when W > 2,
  *                        one with 2-word entries where values from 2^62 up are
  *                        replaced by 2^62, and, when W > 1, one with 1-word entries
  *                        where values from 2^30 up are replaced by 2^30;
@@ -129,9 +129,12 @@ int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, f
 /* Encode (Sec. 3.3 Steps 3, 4, 5, 7; Algorithms 1 and 2).
  *   d_x        rows x cols values of `dtype`, leading dimension ld (elements); 16-byte
  *              aligned, ld a multiple of 8 (bf16) or 4 (fp32) elements.
- *   N, K       group size (power of two, 8..128) and pulses; cols % N == 0; G >= 2.  N = 128
- *              (codes of up to 12 words) runs on slower kernels that keep the tables in
- *              global memory; the fused and rotating entry points stop at N = 64.
+ *   N, K       group size (power of two, 8..256) and pulses (up to 1023, codes of up to 32
+ *              words); cols % N == 0; G >= 2.  Codes of up to 2, 3, 4, 6 words at N = 8, 16,
+ *              32, 64 run on the kernels with the tables in shared memory.  Wider codes at
+ *              N >= 16, and N = 128 and 256, run on slower kernels that keep the tables in
+ *              global memory (the paper's grid of group sizes and direction bits, Sec. 4.1);
+ *              the fused and rotating entry points have only the former.
  *   scale_bits 1..8 (quantile index), or 16 (see pvq_encode_amp).
  *   d_table    from pvq_build_count_table(N, K, ...).
  *   d_edges    2^scale_bits - 1 bin edges.

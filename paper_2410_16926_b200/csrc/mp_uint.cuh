@@ -13,13 +13,31 @@ struct mp {
     uint32_t w[W];
 };
 
-// a += b (the caller knows the sum fits W limbs)
+// a += b (the caller knows the sum fits W limbs).  Widths 1..12 are specialised below; wider
+// numbers take this plain form, whose carries the compiler turns into the same chain.
 template <int W>
-__device__ __forceinline__ void mp_add(mp<W>& a, const mp<W>& b);
+__device__ __forceinline__ void mp_add(mp<W>& a, const mp<W>& b) {
+    uint64_t c = 0;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+        const uint64_t s = static_cast<uint64_t>(a.w[w]) + b.w[w] + c;
+        a.w[w] = static_cast<uint32_t>(s);
+        c = s >> 32;
+    }
+}
 
 // d = a - b; returns true when a < b (a borrow leaves the top limb)
 template <int W>
-__device__ __forceinline__ bool mp_sub_borrow(mp<W>& d, const mp<W>& a, const mp<W>& b);
+__device__ __forceinline__ bool mp_sub_borrow(mp<W>& d, const mp<W>& a, const mp<W>& b) {
+    uint64_t brw = 0;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+        const uint64_t s = static_cast<uint64_t>(a.w[w]) - b.w[w] - brw;
+        d.w[w] = static_cast<uint32_t>(s);
+        brw = (s >> 32) & 1u;
+    }
+    return brw != 0u;
+}
 
 template <>
 __device__ __forceinline__ void mp_add<1>(mp<1>& a, const mp<1>& b) {

@@ -302,6 +302,7 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
     std::memset(&a, 0, sizeof a);
     a.count = count;
     a.K = K;
+    a.code_words = c.W;
     a.scale_bits = scale_bits;
     a.table = d_table;
     a.status = d_status;
@@ -322,7 +323,9 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
         if (st != PVQ_OK) return st;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (c.N > 64) {  // large groups: encode and decode only
+    // codes the shared-memory kernels are built for, by group size
+    const int fast_words = c.N == 8 ? 2 : (c.N == 16 ? 3 : (c.N == 32 ? 4 : (c.N == 64 ? 6 : 0)));
+    if (c.W > fast_words) {  // large groups, wide codes: encode and decode only
         if (kind == 2 || rot_block != 0) return PVQ_ERR_UNSUPPORTED;
         return launch_big(a, dtype, c.N, c.W, kind == 1, s);
     }

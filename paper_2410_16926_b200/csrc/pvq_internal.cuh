@@ -12,8 +12,8 @@
 namespace pvq {
 
 constexpr int kMaxBatch = 32;     // matrices per launch
-constexpr int kMaxWords = 12;     // limbs per code the kernels are instantiated for
-constexpr int kMaxGroup = 128;    // largest group size; above 64 (or 6 limbs) the tables stay in global memory
+constexpr int kMaxWords = 32;     // limbs per code (1024-bit codes)
+constexpr int kMaxGroup = 256;    // largest group size; above 64 (or 6 limbs) the tables stay in global memory
 constexpr int kMaxPulses = 1023;  // table builder: one thread per k
 
 // One matrix as the kernels see it.
@@ -38,6 +38,7 @@ struct BatchArgs {
     unsigned total_tiles;
     int K;
     int scale_bits;
+    int code_words;         // W: 32-bit words of one code in memory (kernels may compute in more)
     const uint32_t* table;  // the blob written by pvq_build_count_table (see TableLayout)
     uint32_t* status;
     int walk_phases;        // decode: how many of the walk tables are staged in shared memory (1..3)
@@ -55,7 +56,8 @@ struct BatchArgs {
 // [n][k][W] words for n = 0..N-1, k = 0..K.  The other sections are the same numbers
 // rearranged for the kernels, so that a thread block can stage them with one flat copy:
 //
-//   bound       N(N,K) as 16 words (codes are valid below it)
+//   bound       N(N,K) as 16 words, 64 words for codes of more than 12 words (codes are valid
+//               below it)
 //   walk[0]     rows by position i (row i holds N(N-1-i, .)), `rowlen` entries of
 //               `top_words` words each, entry (i, col) = N(N-1-i, col), zero padded
 //   walk[1]     same with 2-word entries, values from 2^62 up replaced by 2^62 (present when
@@ -75,8 +77,11 @@ struct BatchArgs {
 //                 enc[2]  V(n,col)
 // words per entry of the widest tables for W-word codes
 __host__ __device__ constexpr int top_words_of(int W) {
-    return W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : (W <= 8 ? 8 : 12)));
+    return W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : (W <= 8 ? 8 : (W <= 12 ? 12 : ((W + 3) & ~3)))));
 }
+
+// words of the blob's copy of N(N,K)
+__host__ __device__ constexpr int bound_words_of(int W) { return W <= 12 ? 16 : 64; }
 
 struct TableLayout {
     int rowlen;
@@ -91,7 +96,7 @@ struct TableLayout {
 
 __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
     TableLayout L;
-    if (N > 128 || W > 12) {  // no kernel for these: the blob is the plain count table
+    if (N > kMaxGroup || W > kMaxWords) {  // no kernel for these: the blob is the plain count table
         L.rowlen = 0;
         L.top_words = 0;
         L.bound_off = 0;
@@ -105,7 +110,7 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
     uint32_t off = static_cast<uint32_t>(N) * (K + 1) * W * 4u;
     off = (off + 127u) & ~127u;
     L.bound_off = off;
-    off += 128u;
+    off += (static_cast<uint32_t>(bound_words_of(W)) * 4u + 127u) & ~127u;
     const uint32_t entries = static_cast<uint32_t>(N) * L.rowlen;
     const int words[3] = {L.top_words, L.top_words > 2 ? 2 : 0, L.top_words > 1 ? 1 : 0};
     for (int p = 0; p < 3; ++p) {

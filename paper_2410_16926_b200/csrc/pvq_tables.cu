@@ -16,8 +16,9 @@ namespace pvq {
 // along k.  The prefix sum is a Hillis-Steele scan through shared memory.  A
 // table of this size never needs more than one block, so there is no
 // inter-block barrier.
+// W is the width the kernel computes in, Wc <= W the words of an entry in memory.
 template <int W>
-__global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, uint32_t* __restrict__ table) {
+__global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, int Wc, uint32_t* __restrict__ table) {
     extern __shared__ uint32_t sm[];  // two buffers of (K+1) entries of W words
     const int k = threadIdx.x;
     const int KP = K + 1;
@@ -32,7 +33,8 @@ __global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, uint32_
     for (int n = 0; n < N; ++n) {
         if (live) {
 #pragma unroll
-            for (int w = 0; w < W; ++w) table[(static_cast<size_t>(n) * KP + k) * W + w] = v.w[w];
+            for (int w = 0; w < W; ++w)
+                if (w < Wc) table[(static_cast<size_t>(n) * KP + k) * Wc + w] = v.w[w];
 #pragma unroll
             for (int w = 0; w < W; ++w) buf0[k * W + w] = v.w[w];
         }
@@ -72,8 +74,8 @@ __global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, uint32_
 // The other sections of the blob (TableLayout): the same numbers re-laid for the decode walk,
 // narrow copies saturated at their width, and N(N,K) itself.
 template <int W>
-__global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) {
-    const TableLayout L = table_layout(N, K, W);
+__global__ void derive_tables_kernel(int N, int K, int Wc, uint32_t* __restrict__ blob) {
+    const TableLayout L = table_layout(N, K, Wc);
     if (L.rowlen == 0) return;
     const int KP = K + 1;
     const int entries = N * L.rowlen;
@@ -84,7 +86,7 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
         uint32_t v[W];
 #pragma unroll
         for (int w = 0; w < W; ++w)
-            v[w] = pad ? 0xffffffffu : blob[(static_cast<size_t>(N - 1 - i) * KP + col) * W + w];
+            v[w] = pad ? 0xffffffffu : (w < Wc ? blob[(static_cast<size_t>(N - 1 - i) * KP + col) * Wc + w] : 0u);
         uint32_t* top = blob + L.walk_off[0] / 4 + static_cast<size_t>(e) * L.top_words;
         for (int w = 0; w < L.top_words; ++w) top[w] = w < W ? v[w] : 0u;
         if (L.walk_bytes[1]) {  // two-word copy: values from 2^62 up become 2^62
@@ -107,7 +109,7 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
     }
     // encoder tables: one thread per position runs the prefix sum V(n,k) = V(n,k-1) + N(n,k)
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) {
-        const uint32_t* row = blob + static_cast<size_t>(N - 1 - i) * KP * W;
+        const uint32_t* row = blob + static_cast<size_t>(N - 1 - i) * KP * Wc;
         const int TW = L.top_words;
         uint32_t* eu = blob + L.enc_off[0] / 4 + static_cast<size_t>(i) * (K + 2) * TW;
         uint32_t* e2 = blob + L.enc_off[1] / 4 + static_cast<size_t>(i) * (K + 2) * TW;
@@ -122,8 +124,9 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
                 unsigned long long carry = 0;
 #pragma unroll
                 for (int w = 0; w < W; ++w) {
-                    const unsigned long long sum = static_cast<unsigned long long>(v[w]) + row[c * W + w] + carry;
-                    v[w] = static_cast<uint32_t>(sum);
+                    const uint32_t add = w < Wc ? row[c * Wc + w] : 0u;
+                    const unsigned long long sum = static_cast<unsigned long long>(v[w]) + add + carry;
+                    v[w] = w < Wc ? static_cast<uint32_t>(sum) : 0u;  // modulo 2^(32 Wc)
                     carry = sum >> 32;
                 }
             }
@@ -134,7 +137,7 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
                 const unsigned long long s2 = static_cast<unsigned long long>(a) + a + c2;
                 cu = su >> 32;
                 c2 = s2 >> 32;
-                const bool in = w < W;  // words beyond W stay zero: the sums are kept modulo 2^(32 W)
+                const bool in = w < Wc;  // words beyond Wc stay zero: the sums are kept modulo 2^(32 Wc)
                 eu[(c + 1) * TW + w] = in ? static_cast<uint32_t>(su) : 0u;
                 e2[(c + 1) * TW + w] = in ? static_cast<uint32_t>(s2) : 0u;
                 ev[(c + 1) * TW + w] = a;
@@ -144,38 +147,44 @@ __global__ void derive_tables_kernel(int N, int K, uint32_t* __restrict__ blob) 
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         // N(N,K) = N(N-1,K) + 2 sum_{j=1..K} N(N-1,K-j)   (every point of P(N,K) by its first
         // coordinate: 0, or +-j with K-j pulses left for the other N-1)
-        uint32_t acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-        const uint32_t* row = blob + static_cast<size_t>(N - 1) * KP * W;
+        constexpr int BW = bound_words_of(W);
+        uint32_t acc[BW];
+        for (int w = 0; w < BW; ++w) acc[w] = 0u;
+        const uint32_t* row = blob + static_cast<size_t>(N - 1) * KP * Wc;
         for (int col = 0; col <= K; ++col) {
             const int times = col == K ? 1 : 2;
             for (int rep = 0; rep < times; ++rep) {
                 unsigned long long carry = 0;
-                for (int w = 0; w < 16; ++w) {
-                    const unsigned long long add = w < W ? row[col * W + w] : 0u;
+                for (int w = 0; w < BW; ++w) {
+                    const unsigned long long add = w < Wc ? row[col * Wc + w] : 0u;
                     const unsigned long long sum = static_cast<unsigned long long>(acc[w]) + add + carry;
                     acc[w] = static_cast<uint32_t>(sum);
                     carry = sum >> 32;
                 }
             }
         }
-        for (int w = 0; w < 16; ++w) blob[L.bound_off / 4 + w] = acc[w];
+        for (int w = 0; w < BW; ++w) blob[L.bound_off / 4 + w] = acc[w];
     }
 }
 
 template <int W>
-static int launch_count_table(int N, int K, uint32_t* d_table, cudaStream_t s) {
+static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStream_t s) {
     const int threads = ((K + 1 + 31) / 32) * 32;
     const size_t smem = 2u * static_cast<size_t>(K + 1) * W * sizeof(uint32_t);
+    DeviceInfo di;
+    const int st = device_info(&di);
+    if (st != PVQ_OK) return st;
+    if (smem > static_cast<size_t>(di.smem_max)) return PVQ_ERR_UNSUPPORTED;
     if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(count_table_kernel<W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              static_cast<int>(smem));
         if (e != cudaSuccess) return set_cuda_error(e);
     }
-    count_table_kernel<W><<<1, threads, smem, s>>>(N, K, d_table);
+    count_table_kernel<W><<<1, threads, smem, s>>>(N, K, Wc, d_table);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error(e);
-    if (table_layout(N, K, W).rowlen != 0) {
-        derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, d_table);
+    if (table_layout(N, K, Wc).rowlen != 0) {
+        derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table);
         e = cudaGetLastError();
     }
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
@@ -241,20 +250,24 @@ extern "C" int pvq_build_count_table(int N, int K, uint32_t* d_table, size_t byt
     if (bytes < pvq_count_table_bytes(N, K)) return PVQ_ERR_TABLE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (W) {
-        case 1: return launch_count_table<1>(N, K, d_table, s);
-        case 2: return launch_count_table<2>(N, K, d_table, s);
-        case 3: return launch_count_table<3>(N, K, d_table, s);
-        case 4: return launch_count_table<4>(N, K, d_table, s);
-        case 5: return launch_count_table<5>(N, K, d_table, s);
-        case 6: return launch_count_table<6>(N, K, d_table, s);
-        case 7: return launch_count_table<7>(N, K, d_table, s);
-        case 8: return launch_count_table<8>(N, K, d_table, s);
-        case 9: return launch_count_table<9>(N, K, d_table, s);
-        case 10: return launch_count_table<10>(N, K, d_table, s);
-        case 11: return launch_count_table<11>(N, K, d_table, s);
-        case 12: return launch_count_table<12>(N, K, d_table, s);
-        default: return PVQ_ERR_UNSUPPORTED;
+        case 1: return launch_count_table<1>(N, K, W, d_table, s);
+        case 2: return launch_count_table<2>(N, K, W, d_table, s);
+        case 3: return launch_count_table<3>(N, K, W, d_table, s);
+        case 4: return launch_count_table<4>(N, K, W, d_table, s);
+        case 5: return launch_count_table<5>(N, K, W, d_table, s);
+        case 6: return launch_count_table<6>(N, K, W, d_table, s);
+        case 7: return launch_count_table<7>(N, K, W, d_table, s);
+        case 8: return launch_count_table<8>(N, K, W, d_table, s);
+        case 9: return launch_count_table<9>(N, K, W, d_table, s);
+        case 10: return launch_count_table<10>(N, K, W, d_table, s);
+        case 11: return launch_count_table<11>(N, K, W, d_table, s);
+        case 12: return launch_count_table<12>(N, K, W, d_table, s);
+        default: break;
     }
+    // wider codes: computed in the next of 16, 24, 32 words
+    if (W <= 16) return launch_count_table<16>(N, K, W, d_table, s);
+    if (W <= 24) return launch_count_table<24>(N, K, W, d_table, s);
+    return launch_count_table<32>(N, K, W, d_table, s);
 }
 
 extern "C" int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, float* d_levels,

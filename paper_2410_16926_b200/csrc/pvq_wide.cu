@@ -1,0 +1,33 @@
+// Codes wider than the shared-memory kernels take (group sizes 16 to 64) or than 12 words
+// (group size 128), and group size 256: the global-table kernels computing in the next of
+// 8, 16 or 32 words (the paper's grid of group sizes and direction bits, Sec. 4.1).
+#include "pvq_big_impl.cuh"
+
+namespace pvq {
+
+int launch_wide(BatchArgs& a, int dtype, int N, int W, bool decode, cudaStream_t s) {
+    const int WB = W <= 8 ? 8 : (W <= 16 ? 16 : 32);
+    switch (N) {
+        case 16:
+            if (WB == 8) return launch_big_w<16, 8, false>(a, dtype, decode, s);
+            break;
+        case 32:
+            if (WB == 8) return launch_big_w<32, 8, false>(a, dtype, decode, s);
+            break;
+        case 64:
+            if (WB == 8) return launch_big_w<64, 8, false>(a, dtype, decode, s);
+            if (WB == 16) return launch_big_w<64, 16, false>(a, dtype, decode, s);
+            break;
+        case 128:
+            if (WB <= 16) return launch_big_w<128, 16, false>(a, dtype, decode, s);
+            return launch_big_w<128, 32, false>(a, dtype, decode, s);
+        case 256:
+            if (WB == 8) return launch_big_w<256, 8, false>(a, dtype, decode, s);
+            if (WB == 16) return launch_big_w<256, 16, false>(a, dtype, decode, s);
+            return launch_big_w<256, 32, false>(a, dtype, decode, s);
+        default: break;
+    }
+    return PVQ_ERR_UNSUPPORTED;
+}
+
+}  // namespace pvq

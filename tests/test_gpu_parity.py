@@ -68,7 +68,8 @@ def check_decode(cd, enc_dev, enc_np):
 
 # ------------------------------------------------------------------ set-up kernels
 
-@pytest.mark.parametrize("N,K", [(8, 6), (8, 40), (16, 18), (32, 22), (32, 50), (64, 96), (32, 1), (128, 187)])
+@pytest.mark.parametrize("N,K", [(8, 6), (8, 40), (16, 18), (32, 22), (32, 50), (64, 96), (32, 1), (128, 187),
+                                 (64, 405), (128, 386), (128, 782), (256, 369), (256, 760)])
 def test_count_table_word_for_word(N, K):
     W = pvq.code_words(N, K)
     t = pvq.build_count_table(N, K)
@@ -81,10 +82,11 @@ def _blob_layout(N, K, W):
     """Byte offsets of the sections that follow the count table (see include/pvq.h)."""
     up = lambda v: (v + 127) & ~127
     rowlen = (K + 2) & ~1
-    top = W if W <= 2 else (4 if W <= 4 else (6 if W <= 6 else (8 if W <= 8 else 12)))
+    top = W if W <= 2 else (4 if W <= 4 else (6 if W <= 6 else (8 if W <= 8 else (12 if W <= 12 else (W + 3) & ~3))))
+    bound_words = 16 if W <= 12 else 64
     off = up(N * (K + 1) * W * 4)
-    lay = {"bound": off, "rowlen": rowlen, "top": top}
-    off += 128
+    lay = {"bound": off, "bound_words": bound_words, "rowlen": rowlen, "top": top}
+    off += up(bound_words * 4)
     for name, words in (("walk_top", top), ("walk2", 2 if top > 2 else 0), ("walk1", 1 if top > 1 else 0)):
         lay[name] = (off, words)
         off += up(N * rowlen * words * 4)
@@ -95,7 +97,8 @@ def _blob_layout(N, K, W):
     return lay
 
 
-@pytest.mark.parametrize("N,K", [(8, 16), (16, 18), (32, 22), (32, 50), (32, 105), (64, 96), (64, 26), (128, 40)])
+@pytest.mark.parametrize("N,K", [(8, 16), (16, 18), (32, 22), (32, 50), (32, 105), (64, 96), (64, 26), (128, 40),
+                                 (64, 230), (128, 300), (256, 200)])
 def test_table_blob_sections(N, K):
     """Every rearranged section of the table blob holds the numbers of the count table."""
     W = pvq.code_words(N, K)
@@ -107,7 +110,8 @@ def test_table_blob_sections(N, K):
     val = [[po.code_to_int(full[n, k]) for k in range(K + 1)] for n in range(N + 1)]
     mask = (1 << (32 * W)) - 1
     words = lambda v, nw: [(v >> (32 * w)) & 0xFFFFFFFF for w in range(nw)]
-    assert list(blob[lay["bound"] // 4: lay["bound"] // 4 + 16]) == words(val[N][K], 16)
+    bwn = lay["bound_words"]
+    assert list(blob[lay["bound"] // 4: lay["bound"] // 4 + bwn]) == words(val[N][K], bwn)
     rowlen, top = lay["rowlen"], lay["top"]
     for name, sat_bits in (("walk_top", None), ("walk2", 62), ("walk1", 30)):
         off, nw = lay[name]
@@ -412,16 +416,26 @@ def test_qsnr_curve_on_a_gaussian_source_equals_the_oracles():
     assert curve[0] < curve[1] < curve[2] and 9.5 < curve[0] < 10.5
 
 
-# ------------------------------------------------------------ large groups (N = 128)
+# -------------------------------------- large groups and wide codes (tables in global memory)
 
-@pytest.mark.parametrize("bits,rows,cols,b,amp_mode,kind", [
-    (384, 9, 4096, 16, 0, "bf16"),      # the paper's 3 bits + 16-bit amplitudes at group size 128
-    (384, 5, 14336, 16, 1, "bf16"),     # G = 112, least-squares amplitudes
-    (256, 7, 1024, 8, 0, "f32"),        # 8-word codes, quantile amplitudes
-    (96, 6, 512, 4, 0, "f32"),          # few pulses: K below 128, byte slots
+@pytest.mark.parametrize("N,bits,rows,cols,b,amp_mode,kind", [
+    (128, 384, 9, 4096, 16, 0, "bf16"),      # the paper's 3 bits + 16-bit amplitudes at group size 128
+    (128, 384, 5, 14336, 16, 1, "bf16"),     # G = 112, least-squares amplitudes
+    (128, 256, 7, 1024, 8, 0, "f32"),        # 8-word codes, quantile amplitudes
+    (128, 96, 6, 512, 4, 0, "f32"),          # few pulses: K below 128, byte slots
+    # the rest of the paper's grid of group sizes and direction bits (Sec. 4.1) that fits 1023 pulses
+    (16, 112, 6, 256, 4, 0, "f32"),          # 7 bits per weight at group size 16: 4 words
+    (32, 160, 7, 512, 8, 0, "bf16"),         # 5 bits per weight: 5 words
+    (32, 192, 3, 256, 16, 1, "bf16"),        # 6 bits per weight
+    (64, 256, 5, 1024, 6, 1, "bf16"),        # 4 bits per weight: 8 words
+    (64, 320, 4, 512, 16, 0, "f32"),         # 5 bits per weight: 10 words, computed in 16
+    (128, 512, 5, 1024, 16, 0, "bf16"),      # 4 bits per weight: 16 words
+    (128, 640, 3, 512, 16, 0, "f32"),        # 5 bits per weight: 20 words, computed in 32
+    (256, 768, 3, 1024, 16, 0, "bf16"),      # group size 256 at 3 bits per weight: 24 words
+    (256, 1024, 3, 512, 16, 1, "f32"),       # 4 bits per weight: 32 words
+    (256, 192, 4, 512, 8, 0, "bf16"),        # group size 256 with a short code
 ])
-def test_large_group_parity(bits, rows, cols, b, amp_mode, kind):
-    N = 128
+def test_large_group_parity(N, bits, rows, cols, b, amp_mode, kind):
     rng = np.random.default_rng(bits + rows)
     x = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
     x[1, :N] = 0.0

@@ -34,7 +34,7 @@ def test_strerror():
     assert b"OK" in pvq.lib().pvq_strerror(0)
 
 
-@pytest.mark.parametrize("N,bits", [(32, 64), (32, 96), (64, 192), (16, 40), (8, 24), (128, 384)])
+@pytest.mark.parametrize("N,bits", [(32, 64), (32, 96), (64, 192), (16, 40), (8, 24), (128, 384), (64, 320), (128, 512), (256, 768)])
 def test_pulse_selection_matches_oracle(N, bits):
     K = pvq.max_pulses(N, bits)
     assert K == po.max_pulses(N, bits)
@@ -90,7 +90,7 @@ def test_bad_arguments_are_rejected_without_a_gpu():
     assert enc(dt=7) == INVALID
     assert enc(ld=32) == INVALID            # ld < cols
     assert enc(cols=32, ld=32) == UNSUPPORTED   # one group per row: no quantile codebook
-    assert enc(N=256, cols=512, ld=512) == UNSUPPORTED
+    assert enc(N=512, cols=1024, ld=1024) == UNSUPPORTED
     assert enc(ld=68) == ALIGN
     assert enc(x=C.c_void_p(p.value + 2)) == ALIGN
     assert enc(tab=None) == INVALID
