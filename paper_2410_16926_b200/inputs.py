@@ -170,3 +170,17 @@ def config6(rows=4096, cols=4096) -> Workload:
     weight of direction (384-bit codes, K = 187) and 16-bit amplitudes, 3.125 bits per weight."""
     wl = config2(rows, cols)
     return Workload("c6_bf16_q_proj_group128", 128, 384, 16, "encode+decode", wl.matrices)
+
+
+def config7(rows=4096, cols=4096) -> Workload:
+    """Sec. 4.1's grid at a higher rate on config2's matrix: group size 64, 4 bits per weight of
+    direction (256-bit codes, K = 199) and 16-bit amplitudes."""
+    wl = config2(rows, cols)
+    return Workload("c7_bf16_q_proj_group64_4bit", 64, 256, 16, "encode+decode", wl.matrices)
+
+
+def config8(rows=4096, cols=4096) -> Workload:
+    """Sec. 4.1's largest group size on config2's matrix: group size 256, 3 bits per weight of
+    direction (768-bit codes, K = 369) and 16-bit amplitudes."""
+    wl = config2(rows, cols)
+    return Workload("c8_bf16_q_proj_group256", 256, 768, 16, "encode+decode", wl.matrices)

@@ -157,11 +157,14 @@ def test_c5r_activations_rotated_on_the_fly_sampled_rows():
     assert st == 0 and np.array_equal(bf16_bits(it["out"][r].contiguous()), o_out)
 
 
-def test_c6_group_128_sampled_rows():
-    wl = inputs.config6()
+@pytest.mark.parametrize("config,expect", [(inputs.config6, (187, 12)), (inputs.config7, (199, 8)),
+                                           (inputs.config8, (369, 24))])
+def test_global_table_kernels_sampled_rows(config, expect):
+    """Group sizes and code widths of Sec. 4.1 that run with the tables in global memory."""
+    wl = config()
     K = pvq.max_pulses(wl.N, wl.index_bits)
     W = pvq.code_words(wl.N, K)
-    assert (K, W) == (187, 12)
+    assert (K, W) == expect
     table = pvq.build_count_table(wl.N, K)
     m = wl.matrices[0]
     G = m.cols // wl.N
