@@ -38,9 +38,9 @@ FALLBACK_HBM_GBS = 6650.0
 # workload and launch configuration as this bench): DRAM bytes read + written, and warp
 # instructions executed.  Set an entry to None when its kernel changes until it is re-captured.
 NCU_COUNTERS = {
-    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_968_384 + 2_816, "warp_inst": 32_554_608},
-    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_651_648 + 1_280, "warp_inst": 40_134_366},
-    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_529_536 + 89_149_440, "warp_inst": 219_689_144},
+    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_665_536 + 5_888, "warp_inst": 32_246_845},
+    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_651_904 + 450_048, "warp_inst": 39_675_358},
+    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_744_832 + 87_227_904, "warp_inst": 219_468_744},
 }
 SMS, SCHEDULERS_PER_SM = 148, 4      # issue slots per cycle on the part = SMS * SCHEDULERS_PER_SM
 
