@@ -214,6 +214,41 @@ def test_degenerate_inputs():
         check_decode(cd, enc_dev, enc_np)
 
 
+@pytest.mark.parametrize("N,bits,b", [(32, 64, 8), (64, 192, 6), (128, 384, 16), (64, 256, 16)])
+def test_non_finite_inputs_give_valid_codes(N, bits, b):
+    """NaN, infinities and sums that overflow are outside the method (their result is left open), but
+    every code written must be a valid one and the other rows must not notice."""
+    rows, cols = 10, 8 * N
+    rng = np.random.default_rng(N + b)
+    x = (rng.standard_normal((rows, cols)) * 0.02).astype(np.float32)
+    x[1, 5] = np.nan
+    x[3, N + 1] = np.inf
+    x[3, 3 * N] = -np.inf
+    x[5, :] = np.nan
+    x[7, 2 * N: 3 * N] = 3e38                          # finite values, sums overflow
+    x[8, 7] = -np.inf
+    x[8, 9] = np.nan
+    finite = np.array([0, 2, 4, 6, 9])
+    K = pvq.max_pulses(N, bits)
+    W = pvq.code_words(N, K)
+    table = pvq.build_count_table(N, K)
+    e_np = bc.edges_f32(N, cols // N, b) if b <= 8 else None
+    l_np = bc.levels_amp_f32(N, cols // N, b) if b <= 8 else None
+    edges = torch.from_numpy(e_np).to(DEV) if b <= 8 else None
+    levels = torch.from_numpy(l_np).to(DEV) if b <= 8 else None
+    codes, sidx, rnorm = pvq.encode(torch.from_numpy(x).to(DEV), N, K, b, table, edges)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = pvq.decode(codes, sidx, rnorm, N, K, b, table, levels, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0                     # every code is below N(N,K)
+    o_codes, o_sidx, o_rnorm = po.encode(np.ascontiguousarray(x[finite]), N, K, b, e_np, W=W)
+    o_out, _ = po.decode(o_codes, o_sidx, o_rnorm, N, K, b, l_np)
+    f = torch.from_numpy(finite).to(DEV)
+    assert np.array_equal(as_u32(codes[f]), o_codes)
+    assert np.array_equal(sidx[f].cpu().numpy(), o_sidx)
+    assert np.array_equal(bf16_bits(out[f].contiguous()), o_out)
+
+
 def test_leading_dimensions():
     N, rows, cols, ld, ldo = 32, 10, 256, 320, 288
     rng = np.random.default_rng(8)
