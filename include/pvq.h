@@ -114,7 +114,7 @@ size_t pvq_scale_row_stride(int64_t G, int scale_bits);
 /* Fill d_table with N(n,k), n = 0..N-1, k = 0..K (Sec. 2.4 recurrence; built a row at a
  * time with a parallel prefix sum over k as in App. C.2 / Algorithm 4, by one thread
  * block).  `bytes` is the size of d_table and must be at least
- * pvq_count_table_bytes(N,K).  Requires 1 <= N <= 256, 1 <= K <= 1023, W <= 12. */
+ * pvq_count_table_bytes(N,K).  Requires 1 <= N <= 256, 1 <= K <= 8191, W <= 32. */
 int pvq_build_count_table(int N, int K, uint32_t* d_table, size_t bytes, pvq_stream_t stream);
 
 /* Fill d_edges (2^b - 1 floats) and d_levels (2^b floats) for group size N, G groups per
@@ -129,7 +129,7 @@ int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, f
 /* Encode (Sec. 3.3 Steps 3, 4, 5, 7; Algorithms 1 and 2).
  *   d_x        rows x cols values of `dtype`, leading dimension ld (elements); 16-byte
  *              aligned, ld a multiple of 8 (bf16) or 4 (fp32) elements.
- *   N, K       group size (power of two, 8..256) and pulses (up to 1023, codes of up to 32
+ *   N, K       group size (power of two, 8..256) and pulses (up to 8191, codes of up to 32
  *              words); cols % N == 0; G >= 2.  Codes of up to 2, 3, 4, 6 words at N = 8, 16,
  *              32, 64 run on the kernels with the tables in shared memory.  Wider codes at
  *              N >= 16, and N = 128 and 256, run on slower kernels that keep the tables in

@@ -455,21 +455,22 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
             }
 
             if (a.amp_mode == 1) {  // least-squares amplitude: tree of |y_i| |x_i| in the es column
-                float ssy = 0.0f;
+                int ssy = 0;  // exact; converted once (it can pass 2^24 when K > 4095)
                 float x[8];
                 for (int j8 = 0; j8 < N / 8; ++j8) {
                     group_values8<BF16>(gx, j8, x);
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
                         const int j = 4 * j8 + p;
-                        const float m0 = fabsf(static_cast<float>(ms(2 * j))), m1 = fabsf(static_cast<float>(ms(2 * j + 1)));
-                        ssy = __fadd_rn(ssy, __fadd_rn(__fmul_rn(m0, m0), __fmul_rn(m1, m1)));
+                        const int y0 = ms(2 * j), y1 = ms(2 * j + 1);
+                        const float m0 = fabsf(static_cast<float>(y0)), m1 = fabsf(static_cast<float>(y1));
+                        ssy += y0 * y0 + y1 * y1;
                         es[j * T] = __fadd_rn(__fmul_rn(m0, fabsf(x[2 * p])), __fmul_rn(m1, fabsf(x[2 * p + 1])));
                     }
                 }
                 for (int len = N / 4; len >= 1; len >>= 1)
                     for (int j = 0; j < len; ++j) es[j * T] = __fadd_rn(es[2 * j * T], es[(2 * j + 1) * T]);
-                ls_amp = __fdiv_rn(es[0], __fsqrt_rn(ssy));
+                ls_amp = __fdiv_rn(es[0], __fsqrt_rn(static_cast<float>(ssy)));
             }
 
             // Algorithm 2 with the cumulative tables (see enumerate_uv)

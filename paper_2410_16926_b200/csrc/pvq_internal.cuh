@@ -14,7 +14,7 @@ namespace pvq {
 constexpr int kMaxBatch = 32;     // matrices per launch
 constexpr int kMaxWords = 32;     // limbs per code (1024-bit codes)
 constexpr int kMaxGroup = 256;    // largest group size; above 64 (or 6 limbs) the tables stay in global memory
-constexpr int kMaxPulses = 1023;  // table builder: one thread per k
+constexpr int kMaxPulses = 8191;  // y_i fits 16 bits with room, a_i < 2^23 (up to 1023: one builder thread per k)
 
 // One matrix as the kernels see it.
 struct MatrixArgs {

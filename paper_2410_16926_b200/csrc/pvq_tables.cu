@@ -71,6 +71,63 @@ __global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, int Wc,
     }
 }
 
+// The same table for more pulses than a block has threads (K up to kMaxPulses).  One block;
+// thread t owns the `chunk` consecutive columns from t * chunk.  Row n is the inclusive prefix
+// sum over k of a_k = N(n-1,k) + N(n-1,k-1), read back from the row the block has just
+// written: each thread sums its chunk, the block scans the threads' totals in shared memory,
+// and a second pass over the chunk writes the row.  Still no inter-block barrier.
+template <int W>
+__global__ void __launch_bounds__(1024) count_table_chunked_kernel(int N, int K, int Wc, int chunk,
+                                                                   uint32_t* __restrict__ table) {
+    extern __shared__ uint32_t tot[];  // blockDim.x entries of W words
+    const int t = threadIdx.x;
+    const int KP = K + 1;
+    const int k0 = t * chunk;
+    const int k1 = k0 + chunk < KP ? k0 + chunk : KP;
+    auto load = [Wc](const uint32_t* row, int k) {
+        mp<W> v;
+#pragma unroll
+        for (int w = 0; w < W; ++w) v.w[w] = w < Wc ? row[static_cast<size_t>(k) * Wc + w] : 0u;
+        return v;
+    };
+    for (int k = k0; k < k1; ++k)  // row 0: N(0,0) = 1, N(0,k>=1) = 0
+        for (int w = 0; w < Wc; ++w) table[static_cast<size_t>(k) * Wc + w] = (k == 0 && w == 0) ? 1u : 0u;
+    __syncthreads();
+    for (int n = 1; n < N; ++n) {
+        const uint32_t* prev = table + static_cast<size_t>(n - 1) * KP * Wc;
+        uint32_t* cur = table + static_cast<size_t>(n) * KP * Wc;
+        mp<W> run;
+        mp_zero(run);
+        for (int k = k0; k < k1; ++k) {
+            mp_add<W>(run, load(prev, k));
+            if (k > 0) mp_add<W>(run, load(prev, k - 1));
+        }
+        // inclusive scan of the threads' totals
+        mp<W> v = run;
+#pragma unroll
+        for (int w = 0; w < W; ++w) tot[t * W + w] = v.w[w];
+        __syncthreads();
+        for (int off = 1; off < static_cast<int>(blockDim.x); off <<= 1) {
+            mp<W> o;
+            mp_zero(o);
+            if (t >= off) o = mp_load<W>(tot + (t - off) * W);
+            __syncthreads();
+            mp_add<W>(v, o);
+#pragma unroll
+            for (int w = 0; w < W; ++w) tot[t * W + w] = v.w[w];
+            __syncthreads();
+        }
+        mp_zero(run);
+        if (t > 0) run = mp_load<W>(tot + (t - 1) * W);  // everything left of this chunk
+        for (int k = k0; k < k1; ++k) {
+            mp_add<W>(run, load(prev, k));
+            if (k > 0) mp_add<W>(run, load(prev, k - 1));
+            for (int w = 0; w < Wc; ++w) cur[static_cast<size_t>(k) * Wc + w] = run.w[w];
+        }
+        __syncthreads();  // the row is complete (and the totals free) before the next one starts
+    }
+}
+
 // The other sections of the blob (TableLayout): the same numbers re-laid for the decode walk,
 // narrow copies saturated at their width, and N(N,K) itself.
 template <int W>
@@ -190,6 +247,23 @@ static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStrea
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 
+template <int W>
+static int launch_count_table_chunked(int N, int K, int Wc, uint32_t* d_table, cudaStream_t s) {
+    const int threads = 1024;
+    const int chunk = (K + 1 + threads - 1) / threads;
+    const size_t smem = static_cast<size_t>(threads) * W * sizeof(uint32_t);
+    cudaError_t e = cudaFuncSetAttribute(count_table_chunked_kernel<W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         static_cast<int>(smem));
+    if (e != cudaSuccess) return set_cuda_error(e);
+    count_table_chunked_kernel<W><<<1, threads, smem, s>>>(N, K, Wc, chunk, d_table);
+    if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
+    if (table_layout(N, K, Wc).rowlen != 0) {
+        derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table);
+        e = cudaGetLastError();
+    }
+    return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
+}
+
 // ---------------------------------------------------------- scale codebook
 //
 // u = ||x_g||^2 / ||x_row||^2 ~ Beta(a, b) with a = N/2, b = N(G-1)/2, both
@@ -249,6 +323,11 @@ extern "C" int pvq_build_count_table(int N, int K, uint32_t* d_table, size_t byt
     if (!is_aligned(d_table, 16)) return PVQ_ERR_ALIGNMENT;
     if (bytes < pvq_count_table_bytes(N, K)) return PVQ_ERR_TABLE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (K > 1023) {  // more pulses than threads of a block: the chunked builder, in 8, 16 or 32 words
+        if (W <= 8) return launch_count_table_chunked<8>(N, K, W, d_table, s);
+        if (W <= 16) return launch_count_table_chunked<16>(N, K, W, d_table, s);
+        return launch_count_table_chunked<32>(N, K, W, d_table, s);
+    }
     switch (W) {
         case 1: return launch_count_table<1>(N, K, W, d_table, s);
         case 2: return launch_count_table<2>(N, K, W, d_table, s);

@@ -69,7 +69,8 @@ def check_decode(cd, enc_dev, enc_np):
 # ------------------------------------------------------------------ set-up kernels
 
 @pytest.mark.parametrize("N,K", [(8, 6), (8, 40), (16, 18), (32, 22), (32, 50), (64, 96), (32, 1), (128, 187),
-                                 (64, 405), (128, 386), (128, 782), (256, 369), (256, 760)])
+                                 (64, 405), (128, 386), (128, 782), (256, 369), (256, 760),
+                                 (16, 1136), (32, 1858), (64, 3359), (128, 1576), (128, 6378), (32, 1024)])
 def test_count_table_word_for_word(N, K):
     W = pvq.code_words(N, K)
     t = pvq.build_count_table(N, K)
@@ -469,6 +470,12 @@ def test_qsnr_curve_on_a_gaussian_source_equals_the_oracles():
     (256, 768, 3, 1024, 16, 0, "bf16"),      # group size 256 at 3 bits per weight: 24 words
     (256, 1024, 3, 512, 16, 1, "f32"),       # 4 bits per weight: 32 words
     (256, 192, 4, 512, 8, 0, "bf16"),        # group size 256 with a short code
+    # more than 1023 pulses: the high-rate end of the grid
+    (16, 128, 5, 256, 8, 0, "bf16"),         # 8 bits per weight at group size 16: K = 1136
+    (32, 256, 4, 256, 16, 1, "f32"),         # 8 bits per weight at group size 32: K = 1858
+    (64, 512, 3, 512, 16, 0, "bf16"),        # 8 bits per weight at group size 64: K = 3359, 16 words
+    (128, 768, 3, 512, 16, 1, "f32"),        # 6 bits per weight at group size 128: K = 1576, 24 words
+    (128, 1024, 3, 512, 16, 1, "bf16"),      # 8 bits per weight at group size 128: K = 6378, 32 words
 ])
 def test_large_group_parity(N, bits, rows, cols, b, amp_mode, kind):
     rng = np.random.default_rng(bits + rows)

@@ -34,7 +34,7 @@ def test_strerror():
     assert b"OK" in pvq.lib().pvq_strerror(0)
 
 
-@pytest.mark.parametrize("N,bits", [(32, 64), (32, 96), (64, 192), (16, 40), (8, 24), (128, 384), (64, 320), (128, 512), (256, 768)])
+@pytest.mark.parametrize("N,bits", [(32, 64), (32, 96), (64, 192), (16, 40), (8, 24), (128, 384), (64, 320), (128, 512), (256, 768), (32, 256), (128, 768)])
 def test_pulse_selection_matches_oracle(N, bits):
     K = pvq.max_pulses(N, bits)
     assert K == po.max_pulses(N, bits)
@@ -73,7 +73,7 @@ def test_bad_arguments_are_rejected_without_a_gpu():
     assert L.pvq_build_count_table(32, 22, None, 1 << 20, None) == INVALID
     assert L.pvq_build_count_table(0, 22, p, 1 << 20, None) == INVALID
     assert L.pvq_build_count_table(32, 22, p, 16, None) == SMALL
-    assert L.pvq_build_count_table(32, 5000, p, 1 << 30, None) == UNSUPPORTED
+    assert L.pvq_build_count_table(32, 9000, p, 1 << 30, None) == UNSUPPORTED
     assert L.pvq_build_count_table(32, 22, C.c_void_p(p.value + 4), 1 << 20, None) == ALIGN
     # codebook
     assert L.pvq_build_scale_codebook(32, 1, 4, p, p, None) == INVALID
