@@ -184,3 +184,11 @@ def config8(rows=4096, cols=4096) -> Workload:
     direction (768-bit codes, K = 369) and 16-bit amplitudes."""
     wl = config2(rows, cols)
     return Workload("c8_bf16_q_proj_group256", 256, 768, 16, "encode+decode", wl.matrices)
+
+
+def config9(rows=4096, cols=4096) -> Workload:
+    """The setting of the paper's headline result (abstract; weight-only tables of Sec. 4: 3 bits of
+    direction and 4-bit amplitudes at group size 16, 3.25 bits per weight) on config2's matrix:
+    48-bit codes, K = 27."""
+    wl = config2(rows, cols)
+    return Workload("c9_bf16_q_proj_group16", 16, 48, 4, "encode+decode", wl.matrices)

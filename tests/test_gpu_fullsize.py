@@ -137,6 +137,21 @@ def test_c1_fp32_every_row():
     check_rows(wl, items, K, W, nrows=512, what=("codes", "out"))
 
 
+def test_c9_group_16_sampled_rows():
+    wl = inputs.config9()
+    K = pvq.max_pulses(wl.N, wl.index_bits)
+    W = pvq.code_words(wl.N, K)
+    assert (K, W) == (27, 2)
+    table = pvq.build_count_table(wl.N, K)
+    items = workload_items(wl, K, W)
+    pvq.encode_batched(items, torch.bfloat16, wl.N, K, wl.scale_bits, table)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    pvq.decode_batched(items, wl.N, K, wl.scale_bits, table, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    check_rows(wl, items, K, W, nrows=128, what=("codes", "out"))
+
+
 def test_c5r_activations_rotated_on_the_fly_sampled_rows():
     wl = inputs.config5_unrotated()
     K = pvq.max_pulses(wl.N, wl.index_bits)
