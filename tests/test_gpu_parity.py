@@ -504,3 +504,56 @@ def test_large_group_parity(N, bits, rows, cols, b, amp_mode, kind):
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert np.array_equal(bf16_bits(out), o_out), "decoded"
+
+
+# ------------------------------------------------------------ seeded random configurations
+
+def _random_case(seed):
+    rng = np.random.default_rng(9000 + seed)
+    N = int(rng.choice([8, 16, 32, 64, 128, 256]))
+    max_bits = {8: 64, 16: 128, 32: 256, 64: 512, 128: 1024, 256: 1024}[N]
+    bits = int(rng.integers(max(N // 2, 8), max_bits + 1))
+    G = int(rng.integers(2, 24))
+    rows = int(rng.integers(1, 8))
+    b = int(rng.choice([1, 2, 3, 4, 5, 6, 7, 8, 16]))
+    kind = str(rng.choice(["f32", "bf16"]))
+    amp_mode = int(rng.integers(0, 2))
+    dist = str(rng.choice(["gauss", "student", "sparse"]))
+    return N, bits, G, rows, b, kind, amp_mode, dist
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_configuration_parity(seed):
+    N, bits, G, rows, b, kind, amp_mode, dist = _random_case(seed)
+    K = pvq.max_pulses(N, bits)
+    if K < 1:
+        pytest.skip("no pulse fits %d bits at N = %d" % (bits, N))
+    W = pvq.code_words(N, K)
+    rng = np.random.default_rng(seed)
+    cols = N * G
+    if dist == "gauss":
+        x = rng.standard_normal((rows, cols)) * 0.02
+    elif dist == "student":
+        x = rng.standard_t(3.0, size=(rows, cols))
+    else:
+        x = rng.standard_normal((rows, cols)) * (rng.random((rows, cols)) < 0.15)
+    x = x.astype(np.float32)
+    x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+    table = pvq.build_count_table(N, K)
+    e_np = bc.edges_f32(N, G, b) if b <= 8 else None
+    l_np = bc.levels_amp_f32(N, G, b) if b <= 8 else None
+    edges = torch.from_numpy(e_np).to(DEV) if b <= 8 else None
+    levels = torch.from_numpy(l_np).to(DEV) if b <= 8 else None
+    o_codes, o_sidx, o_rnorm = po.encode(x_np, N, K, b, e_np, W=W, amp_mode=amp_mode)
+    o_out, o_st = po.decode(o_codes, o_sidx, o_rnorm, N, K, b, l_np)
+    codes, sidx, rnorm = pvq.encode(to_device(x_np, kind), N, K, b, table, edges, amp_mode=amp_mode)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = pvq.decode(codes, sidx, rnorm, N, K, b, table, levels, status=status)
+    torch.cuda.synchronize()
+    what = "N=%d bits=%d K=%d W=%d G=%d rows=%d b=%d %s amp_mode=%d %s" % (N, bits, K, W, G, rows, b, kind, amp_mode, dist)
+    assert np.array_equal(rnorm.cpu().numpy().view(np.uint32), o_rnorm.view(np.uint32)), what
+    assert np.array_equal(sidx.cpu().numpy(), o_sidx), what
+    assert np.array_equal(as_u32(codes), o_codes), what
+    assert int(status.item()) == o_st == 0, what
+    assert np.array_equal(bf16_bits(out), o_out), what
+
