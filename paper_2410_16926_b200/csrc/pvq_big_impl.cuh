@@ -50,14 +50,23 @@ __device__ __forceinline__ mp<W> load_entry_v(const uint8_t* p, int TW) {
     return t;
 }
 
-// One phase of the decode walk (see pvq_walk.cuh) with the table in global memory.
+// One phase of the decode walk (see pvq_walk.cuh) with the table in global memory, computing
+// in PW words on entries of TW words.  The phase ends when every lane can go on in
+// next_words words: on a narrow table whose large values are saturated (next_same false:
+// the remainder must be two bits below the width), or on this table with fewer words
+// (next_same true: the remainder and the entry just read fit next_words words; the entries
+// along a path never grow, N(n,k) being monotone in n and k).
 template <int PW, int CW, typename YT>
 __device__ __forceinline__ int walk_phase_g(mp<CW>& rfull, Walk& st, const uint8_t* tab, int TW, int rowlen,
-                                            int K, int s, const int S, const int next_words) {
+                                            int K, int s, const int S, const int next_words,
+                                            const bool next_same) {
     const int EB = TW * 4;  // bytes per entry
-    mp<PW> r;
+    mp<PW> r, t;
 #pragma unroll
-    for (int w = 0; w < PW; ++w) r.w[w] = rfull.w[w];
+    for (int w = 0; w < PW; ++w) {
+        r.w[w] = rfull.w[w];
+        t.w[w] = 0xffffffffu;  // no entry read yet
+    }
     const int D = (rowlen + 1) * EB;
     const int i0 = static_cast<int>(st.y - st.y0) / static_cast<int>(sizeof(YT));
     const uint8_t* p = tab + static_cast<size_t>(i0) * D + (K - s) * EB;
@@ -67,12 +76,16 @@ __device__ __forceinline__ int walk_phase_g(mp<CW>& rfull, Walk& st, const uint8
         if (next_words > 0 && (s & 7) == 0) {
             uint32_t hi = 0;
 #pragma unroll
-            for (int w = 2; w < PW; ++w) hi |= r.w[w];
-            if constexpr (PW > 1) hi |= next_words == 2 ? (r.w[1] >> 30) : r.w[1];
-            if (next_words == 1) hi |= r.w[0] >> 30;
+            for (int w = 1; w < PW; ++w)
+                if (w >= next_words) hi |= next_same ? (r.w[w] | t.w[w]) : r.w[w];
+            if (!next_same) {
+#pragma unroll
+                for (int w = 0; w < PW; ++w)
+                    if (w == next_words - 1) hi |= r.w[w] >> 30;
+            }
             if (__all_sync(kFull, hi == 0u)) break;
         }
-        const mp<PW> t = load_entry_v<PW>(p, TW);
+        t = load_entry_v<PW>(p, TW);
         mp<PW> d2, d1;
         const bool lt1 = mp_sub_borrow<PW>(d2, r, t);
         const bool lt2 = mp_sub_borrow<PW>(d1, d2, t);
@@ -93,6 +106,21 @@ __device__ __forceinline__ int walk_phase_g(mp<CW>& rfull, Walk& st, const uint8
     st.v = v;
     st.y = y;
     return s;
+}
+
+// The phases on the full-width table: PW words, then 16, 8 and 4 as the remainder shrinks
+// (about one bit per step), the last of them handing over to the narrow tables (sat_next).
+template <int PW, int CW, typename YT>
+__device__ __forceinline__ int walk_wide_phases(mp<CW>& c, Walk& st, const uint8_t* tab, int TW, int rowlen, int K,
+                                                int s, const int S, const int sat_next) {
+    constexpr int NEXT = PW > 16 ? 16 : (PW > 8 ? 8 : (PW > 4 ? 4 : 0));
+    if constexpr (NEXT == 0) {
+        return walk_phase_g<PW, CW, YT>(c, st, tab, TW, rowlen, K, s, S, sat_next, false);
+    } else {
+        s = walk_phase_g<PW, CW, YT>(c, st, tab, TW, rowlen, K, s, S, NEXT, true);
+        if (s < S) s = walk_wide_phases<NEXT, CW, YT>(c, st, tab, TW, rowlen, K, s, S, sat_next);
+        return s;
+    }
 }
 
 constexpr int kBigThreads = 256;
@@ -235,14 +263,14 @@ __global__ void __launch_bounds__(kBigThreads) decode_big_kernel(const __grid_co
         st.y = st.y0 = shared_addr(yslots);
         int s = 0;
         const bool has2 = L.walk_bytes[1] != 0, has1 = L.walk_bytes[2] != 0;
-        s = walk_phase_g<W, W, YT>(c, st, blob + L.walk_off[0], TW, L.rowlen, K, s, S,
-                                   has2 ? 2 : (has1 ? 1 : 0));
+        s = walk_wide_phases<W, W, YT>(c, st, blob + L.walk_off[0], TW, L.rowlen, K, s, S,
+                                       has2 ? 2 : (has1 ? 1 : 0));
         if constexpr (W > 2) {
             if (s < S && has2)
-                s = walk_phase_g<2, W, YT>(c, st, blob + L.walk_off[1], 2, L.rowlen, K, s, S, has1 ? 1 : 0);
+                s = walk_phase_g<2, W, YT>(c, st, blob + L.walk_off[1], 2, L.rowlen, K, s, S, has1 ? 1 : 0, false);
         }
         if constexpr (W > 1) {
-            if (s < S && has1) s = walk_phase_g<1, W, YT>(c, st, blob + L.walk_off[2], 1, L.rowlen, K, s, S, 0);
+            if (s < S && has1) s = walk_phase_g<1, W, YT>(c, st, blob + L.walk_off[2], 1, L.rowlen, K, s, S, 0, false);
         }
         if (active) emit_group<N, YT>(m, yslots, amp, row, g);
         __syncwarp();
