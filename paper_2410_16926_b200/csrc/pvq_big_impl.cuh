@@ -507,14 +507,17 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
             mp_zero(minus);
             int k = K;
             const size_t rowwords = static_cast<size_t>(K + 2) * TW;
+#pragma unroll 4
             for (int i = 0; i < N; ++i) {
                 const int y = ms(i);
-                const int k2 = k - abs(y);
-                const uint8_t* ru = tabU + (i * rowwords + static_cast<size_t>(k + 1) * TW) * 4;
-                const uint8_t* rx = (y <= 0 ? tabU : tab2V) + (i * rowwords + static_cast<size_t>(k2 + 1) * TW) * 4;
-                mp_add<W>(plus, load_entry_v<W>(ru, TW));
-                mp_add<W>(minus, load_entry_v<W>(rx, TW));
-                k = k2;
+                if (y != 0) {  // a zero adds and subtracts the same entry
+                    const int k2 = k - abs(y);
+                    const uint8_t* ru = tabU + (i * rowwords + static_cast<size_t>(k + 1) * TW) * 4;
+                    const uint8_t* rx = (y < 0 ? tabU : tab2V) + (i * rowwords + static_cast<size_t>(k2 + 1) * TW) * 4;
+                    mp_add<W>(plus, load_entry_v<W>(ru, TW));
+                    mp_add<W>(minus, load_entry_v<W>(rx, TW));
+                    k = k2;
+                }
             }
             mp_sub_borrow<W>(c, plus, minus);
         }
