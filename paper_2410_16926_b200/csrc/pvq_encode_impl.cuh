@@ -380,8 +380,9 @@ __device__ __forceinline__ TileLoc locate(const BatchArgs& a, unsigned tile) {
 
 // Shared memory: [encoder tables][walk tables (fused)][2 x ss per thread slot, padded rows]
 //                [edges][levels (fused)][2 x scale-index words][per-warp slots (fused)]
-// The two ss / scale-index buffers alternate between consecutive tiles, which leaves three
-// block-wide barriers per tile (two in the fused kernel); the input of the next tile is
+// The two ss / scale-index buffers alternate between consecutive tiles, and a tile's index
+// words are written out behind the next tile's first barrier, which leaves two block-wide
+// barriers per tile; the input of the next tile is
 // requested as soon as the registers that held this tile's input are free.
 //
 // ROT: the tile is first rotated (rotate_tile); the kernel then works on the rotated fp32
@@ -457,6 +458,11 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     }
     if (!bulk_stage_wait(stage)) return;  // the tables never arrived: leave rather than spin
     __syncthreads();                      // index words cleared
+    struct {
+        bool valid;
+        int mi, rpt;
+        long long row0;
+    } prev = {false, 0, 0, 0};  // the tile whose index words are still to be written out
 
     for (int buf = 0;; buf ^= 1) {
         const MatrixArgs& m = a.m[loc.mi];
@@ -507,8 +513,21 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
                 for (int i = threadIdx.x; i <= nedges; i += blockDim.x) s_levels[i] = m.levels[i];
             cur_edges = m.edges;
         }
-        if constexpr (!FUSED) {  // the other buffer's index words, for the next tile
+        if constexpr (!FUSED) {
+            // The previous tile's index words (the other buffer) are complete: every thread added
+            // its bits before it came to barrier (1).  Write them out and clear them for the next tile.
             uint32_t* other = s_idx2 + (buf ^ 1) * sm.idx_words;
+            if (prev.valid) {
+                const MatrixArgs& pm = a.m[prev.mi];
+                const int piw = pm.sstride >> 2;
+                for (int i = threadIdx.x; i < prev.rpt * piw; i += blockDim.x) {
+                    const int r2 = i / piw;
+                    const long long row2 = prev.row0 + r2;
+                    if (row2 < pm.rows)
+                        reinterpret_cast<uint32_t*>(pm.scale_idx + static_cast<size_t>(row2) * pm.sstride)[i - r2 * piw] =
+                            other[i];
+                }
+            }
             for (int i = threadIdx.x; i < sm.idx_words; i += blockDim.x) other[i] = 0u;
         }
         // row energy: balanced tree over the (zero padded) groups of each row, one warp per row
@@ -609,14 +628,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
                 if (sh + b > 32u)
                     atomicOr(&s_idx[rl * idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));
             }
-            __syncthreads();  // (3) the tile's index words are complete
-            for (int i = threadIdx.x; i < rpt * idx_words; i += blockDim.x) {
-                const int r2 = i / idx_words;
-                const long long row2 = row0 + r2;
-                if (row2 < m.rows)
-                    reinterpret_cast<uint32_t*>(m.scale_idx + static_cast<size_t>(row2) * m.sstride)[i - r2 * idx_words] =
-                        s_idx[i];
-            }
+            prev.valid = true;  // written out after the next tile's first barrier, or after the loop
+            prev.mi = loc.mi;
+            prev.rpt = rpt;
+            prev.row0 = row0;
         } else {
             // decode the code just made (every thread of the warp walks, in lockstep)
             const float amp = !active ? 0.0f
@@ -627,7 +642,19 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             if (active) emit_group<N, YT>(m, yslots, amp, static_cast<unsigned>(row), static_cast<unsigned>(g));
         }
 
-        if (!have_next) break;
+        if (!have_next) {
+            if constexpr (!FUSED) {
+                __syncthreads();  // the last tile's index words are complete
+                for (int i = threadIdx.x; i < rpt * idx_words; i += blockDim.x) {
+                    const int r2 = i / idx_words;
+                    const long long row2 = row0 + r2;
+                    if (row2 < m.rows)
+                        reinterpret_cast<uint32_t*>(m.scale_idx + static_cast<size_t>(row2) * m.sstride)[i - r2 * idx_words] =
+                            s_idx[i];
+                }
+            }
+            break;
+        }
         tile = next_tile;
         loc = nloc;
     }
