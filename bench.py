@@ -231,6 +231,35 @@ class GpuRun:
                for j, (name, _) in enumerate(phases)}
         return total_ms, per
 
+    def run_graph(self, steps, warmup):
+        """The same steps replayed from a CUDA graph (one step per buffer set captured through the
+        library's calls): the device time of a step without the host's launch work, which is what
+        a launch-bound workload otherwise measures.  Returns ms per step."""
+        torch = self.torch
+        phases = self.phases()
+        stream = torch.cuda.Stream()
+        stream.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            for items in self.sets:                    # kernel attributes are set on first use
+                for _, fn in phases:
+                    fn(items)
+            stream.synchronize()
+            with torch.cuda.graph(graph, stream=stream):
+                for items in self.sets:
+                    for _, fn in phases:
+                        fn(items)
+            replays = max(1, (steps + self.nsets - 1) // self.nsets)
+            for _ in range(max(1, warmup // self.nsets)):
+                graph.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(replays):
+                graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+        return e0.elapsed_time(e1) / (replays * self.nsets)
+
     def _new_set(self):
         """One more device buffer set (the end-to-end leg wants at least two to overlap steps)."""
         torch, pvq, wl = self.torch, self.pvq, self.wl
@@ -406,6 +435,8 @@ def main():
     ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c5r", "c6", "c7", "c8", "c9"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--graph", action="store_true",
+                    help="also time the steps replayed from a CUDA graph (for launch-bound workloads)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     warmup = max(args.warmup, 3)
@@ -465,6 +496,8 @@ def main():
     total_ms = max_over_ranks(total_ms, world, device)
     value = whole_job_value(step_bytes, args.steps, world, total_ms)
 
+    graph_ms = run.run_graph(args.steps, warmup) if args.graph else None
+
     e2e = None
     if not args.no_e2e:
         e_steps = max(3, min(args.steps, 20))
@@ -517,6 +550,8 @@ def main():
             "config": config, "Gweights_per_s": wl.weights * args.steps * world / (total_ms * 1e-3) / 1e9,
             "kernels": kernels, "roofline": roofline, "issue": issue, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
             "gpu_launches": len(per) * args.steps}
+    if graph_ms is not None:
+        line["graph_replay"] = {"ms_per_step": graph_ms, "GBps": step_bytes / (graph_ms * 1e-3) / 1e9}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
