@@ -134,7 +134,7 @@ int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, f
  *              32, 64 run on the kernels with the tables in shared memory.  Wider codes at
  *              N >= 16, and N = 128 and 256, run on slower kernels that keep the tables in
  *              global memory (the paper's grid of group sizes and direction bits, Sec. 4.1);
- *              the fused and rotating entry points have only the former.
+ *              the rotating entry points have only the former.
  *   scale_bits 1..8 (quantile index), or 16 (see pvq_encode_amp).
  *   d_table    from pvq_build_count_table(N, K, ...).
  *   d_edges    2^scale_bits - 1 bin edges.

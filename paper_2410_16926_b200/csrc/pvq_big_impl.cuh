@@ -342,7 +342,7 @@ __device__ __forceinline__ void group_values8(const void* gx, int j, float (&x)[
 // Encoder for large groups: the steps of encode_kernel with the per-thread arrays (residuals
 // to sort, the point) in shared memory columns es[i * T + t], the input re-read
 // from global memory where it is needed, and the cumulative tables read from global memory.
-template <int N, int W, bool EXACT, bool BF16>
+template <int N, int W, bool EXACT, bool BF16, bool FUSED>
 __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_constant__ BatchArgs a,
                                                                   const __grid_constant__ BigSmem sm) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -523,6 +523,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
         }
 
         __syncthreads();  // row energies are in s_ss[r * gp]
+        float amp = 0.0f;     // round trip: the dequantised amplitude
         if (active) {
             const float ss_row = s_ss[rl * gp];
             const float rnorm = __fsqrt_rn(ss_row);
@@ -535,15 +536,47 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 for (int step = 1 << (b - 1); step >= 1; step >>= 1)
                     if (s_edges[q + step - 1] <= u) q += step;
             }
-            if (g == 0) m.row_norm[row] = rnorm;
-            uint32_t* cp = m.codes + (static_cast<size_t>(row) * G + g) * Wc;
+            if constexpr (FUSED) {
+                amp = b == 16 ? __half2float(__ushort_as_half(static_cast<unsigned short>(q)))
+                              : __fmul_rn(rnorm, m.levels[q]);
+            } else {
+                if (g == 0) m.row_norm[row] = rnorm;
+                uint32_t* cp = m.codes + (static_cast<size_t>(row) * G + g) * Wc;
 #pragma unroll
-            for (int w = 0; w < W; ++w)
-                if (w < Wc) cp[w] = c.w[w];
-            const unsigned bit = static_cast<unsigned>(g) * b;
-            const unsigned sh = bit & 31u;
-            atomicOr(&s_idx[rl * idx_words + (bit >> 5)], static_cast<uint32_t>(q) << sh);
-            if (sh + b > 32u) atomicOr(&s_idx[rl * idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));
+                for (int w = 0; w < W; ++w)
+                    if (w < Wc) cp[w] = c.w[w];
+                const unsigned bit = static_cast<unsigned>(g) * b;
+                const unsigned sh = bit & 31u;
+                atomicOr(&s_idx[rl * idx_words + (bit >> 5)], static_cast<uint32_t>(q) << sh);
+                if (sh + b > 32u)
+                    atomicOr(&s_idx[rl * idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));
+            }
+        }
+        if constexpr (FUSED) {
+            // Round trip (activations, Sec. 4.3): decode the code just made.  Every thread is past
+            // the enumeration (the barrier above), so the columns are free: each thread collects
+            // its point in its own slots there, as decode_big_kernel does.
+            constexpr int YS = N * 2 + 4;
+            short* yslots = reinterpret_cast<short*>(smem + sm.es_off + static_cast<size_t>(t) * YS);
+            Walk st;
+            st.v = 0;
+            st.y = st.y0 = shared_addr(yslots);
+            const int S = N + K;
+            int s = 0;
+            const bool has2 = L.walk_bytes[1] != 0, has1 = L.walk_bytes[2] != 0;
+            s = walk_wide_phases<W, W, short>(c, st, blob + L.walk_off[0], TW, L.rowlen, K, s, S,
+                                              has2 ? 2 : (has1 ? 1 : 0));
+            if constexpr (W > 2) {
+                if (s < S && has2)
+                    s = walk_phase_g<2, W, short>(c, st, blob + L.walk_off[1], 2, L.rowlen, K, s, S, has1 ? 1 : 0, false);
+            }
+            if constexpr (W > 1) {
+                if (s < S && has1)
+                    s = walk_phase_g<1, W, short>(c, st, blob + L.walk_off[2], 1, L.rowlen, K, s, S, 0, false);
+            }
+            if (active)
+                emit_group<N, short>(m, yslots, amp, static_cast<unsigned>(row), static_cast<unsigned>(g));
+            continue;  // the barrier at the top of the loop frees the slots
         }
         __syncthreads();
         for (int i = t; i < rpt * idx_words; i += T) {
@@ -555,7 +588,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
     }
 }
 
-template <int N, int W, bool EXACT, bool BF16>
+template <int N, int W, bool EXACT, bool BF16, bool FUSED>
 int launch_encode_big_t(BatchArgs& a, cudaStream_t stream) {
     DeviceInfo di;
     int st = device_info(&di);
@@ -601,7 +634,7 @@ int launch_encode_big_t(BatchArgs& a, cudaStream_t stream) {
     sm.idx_words = idx_words;
     const size_t smem = sm.idx_off + idx_words * 4u;
     if (smem > static_cast<size_t>(di.smem_max)) return PVQ_ERR_UNSUPPORTED;
-    auto kern = encode_big_kernel<N, W, EXACT, BF16>;
+    auto kern = encode_big_kernel<N, W, EXACT, BF16, FUSED>;
     int per_sm = 0;
     if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
@@ -616,8 +649,11 @@ int launch_big_w(BatchArgs& a, int dtype, bool decode, cudaStream_t s) {
     if (decode)
         return a.K <= 127 ? launch_decode_big_t<N, W, EXACT, int8_t>(a, s)
                           : launch_decode_big_t<N, W, EXACT, int16_t>(a, s);
-    return dtype == PVQ_DTYPE_BF16 ? launch_encode_big_t<N, W, EXACT, true>(a, s)
-                                   : launch_encode_big_t<N, W, EXACT, false>(a, s);
+    if (a.fused)
+        return dtype == PVQ_DTYPE_BF16 ? launch_encode_big_t<N, W, EXACT, true, true>(a, s)
+                                       : launch_encode_big_t<N, W, EXACT, false, true>(a, s);
+    return dtype == PVQ_DTYPE_BF16 ? launch_encode_big_t<N, W, EXACT, true, false>(a, s)
+                                   : launch_encode_big_t<N, W, EXACT, false, false>(a, s);
 }
 
 }  // namespace

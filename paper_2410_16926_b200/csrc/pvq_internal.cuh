@@ -48,6 +48,7 @@ struct BatchArgs {
     uint32_t c_one, c_minus_one;
     // rotation in front of the encoder (Sec. 2.3 / Sec. 3.3 Step 1); rot_block = 0: none
     int amp_mode;            // encode: 0 amplitude ||x_g||, 1 least-squares amplitude (Step 4)
+    int fused;               // global-table encoder: decode the code just made instead of storing it
     const float* rot_signs;  // +-1, rot_block of them
     int rot_block;           // power of two, a multiple of N, dividing every cols
 };
@@ -145,7 +146,7 @@ int prepare_kernel(const void* kern, int threads, size_t smem, int* blocks_per_s
 // launchers (one per kernel family); all return a pvq_status
 int launch_decode(const BatchArgs& args, int N, int W, cudaStream_t stream);
 // large groups / wide codes (N = 128 or more than 6 words): tables in global memory
-int launch_big(const BatchArgs& args, int dtype, int N, int W, bool decode, cudaStream_t stream);
+int launch_big(const BatchArgs& args, int dtype, int N, int W, bool decode, cudaStream_t stream);  // args.fused: round trip
 int launch_encode(const BatchArgs& args, int dtype, int N, int W, bool fused, cudaStream_t stream);  // rotates when args.rot_block != 0
 
 // ---------------------------------------------------------------- device bits

@@ -297,6 +297,32 @@ def test_fused_roundtrip_equals_encode_then_decode():
         assert np.array_equal(bf16_bits(out), o_out)
 
 
+@pytest.mark.parametrize("N,bits,rows,cols,b,kind", [
+    (128, 512, 6, 1024, 8, "bf16"),      # activations at group size 128, 4 bits of direction (Sec. 4.3)
+    (128, 384, 9, 4096, 16, "bf16"),
+    (64, 256, 5, 512, 6, "f32"),         # computed in 8 words
+    (256, 768, 3, 1024, 16, "bf16"),     # computed in 32 words
+    (128, 96, 4, 512, 4, "f32"),         # few pulses
+])
+def test_fused_roundtrip_global_table_kernels(N, bits, rows, cols, b, kind):
+    rng = np.random.default_rng(rows + N)
+    x = rng.standard_normal((rows, cols)).astype(np.float32)
+    x[1, :N] = 0.0
+    x_np = inputs.f32_to_bf16_bits(x) if kind == "bf16" else x
+    K = pvq.max_pulses(N, bits)
+    W = pvq.code_words(N, K)
+    table = pvq.build_count_table(N, K)
+    e_np = bc.edges_f32(N, cols // N, b) if b <= 8 else None
+    l_np = bc.levels_amp_f32(N, cols // N, b) if b <= 8 else None
+    edges = torch.from_numpy(e_np).to(DEV) if b <= 8 else None
+    levels = torch.from_numpy(l_np).to(DEV) if b <= 8 else None
+    out = pvq.roundtrip(to_device(x_np, kind), N, K, b, table, edges, levels)
+    torch.cuda.synchronize()
+    enc = po.encode(x_np, N, K, b, e_np, W=W)
+    o_out, _ = po.decode(*enc, N, K, b, l_np)
+    assert np.array_equal(bf16_bits(out), o_out)
+
+
 def test_batched_calls_match_single_calls():
     wl = inputs.config3(scale_div=256)       # the seven matrices of a layer, 1/256 of the rows
     N, b = wl.N, wl.scale_bits
