@@ -192,3 +192,11 @@ def config9(rows=4096, cols=4096) -> Workload:
     48-bit codes, K = 27."""
     wl = config2(rows, cols)
     return Workload("c9_bf16_q_proj_group16", 16, 48, 4, "encode+decode", wl.matrices)
+
+
+def config10(tokens=16384, hidden=4096) -> Workload:
+    """config5's activations at the setting of the paper's weight-and-activation results (Sec. 4.3:
+    4.125 bits per activation at group size 128): 4 bits of direction per value (512-bit codes,
+    K = 386) and 16-bit amplitudes; fused encode -> decode."""
+    wl = config5(tokens, hidden)
+    return Workload("c10_bf16_activations_group128", 128, 512, 16, "roundtrip", wl.matrices)

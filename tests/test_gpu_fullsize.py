@@ -39,9 +39,11 @@ def workload_items(wl, K, W):
     items, books = [], {}
     for m in wl.matrices:
         G = m.cols // N
-        if G not in books:
+        if G not in books and b <= 8:
             e_np, l_np = bc.edges_f32(N, G, b), bc.levels_amp_f32(N, G, b)
             books[G] = (e_np, l_np, torch.from_numpy(e_np).to(DEV), torch.from_numpy(l_np).to(DEV))
+        elif G not in books:                # 16-bit amplitudes use no codebook
+            books[G] = (None, None, None, None)
         e_np, l_np, e_d, l_d = books[G]
         codes, sidx, rnorm = pvq.alloc_encoded(m.rows, G, W, b)
         x = dev_bf16(m.data) if m.dtype == "bf16" else torch.from_numpy(m.data).to(DEV)
@@ -135,6 +137,19 @@ def test_c1_fp32_every_row():
     pvq.decode_batched(items, wl.N, K, wl.scale_bits, table)
     torch.cuda.synchronize()
     check_rows(wl, items, K, W, nrows=512, what=("codes", "out"))
+
+
+def test_c10_activations_group_128_fused_sampled_rows():
+    wl = inputs.config10()
+    K = pvq.max_pulses(wl.N, wl.index_bits)
+    W = pvq.code_words(wl.N, K)
+    assert (K, W) == (386, 16)
+    table = pvq.build_count_table(wl.N, K)
+    items = workload_items(wl, K, W)
+    it = items[0]
+    pvq.roundtrip(it["x"], wl.N, K, wl.scale_bits, table, it["edges"], it["levels"], out=it["out"])
+    torch.cuda.synchronize()
+    check_rows(wl, items, K, W, nrows=96, what=("out",))
 
 
 def test_c9_group_16_sampled_rows():
