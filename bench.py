@@ -147,7 +147,7 @@ class ClockSampler:
 
 # --------------------------------------------------------------------- GPU runner
 
-class GpuRun:
+class DeviceRun:
     """Device state of one workload: tables, codebooks, S rotating buffer sets."""
 
     def __init__(self, wl, device):
@@ -478,7 +478,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
-    run = GpuRun(wl, device)
+    run = DeviceRun(wl, device)
     config["buffer_sets"] = run.nsets
     config["l2"] = "rotating %d buffer sets, %.0f MB in total, larger than the 126 MB L2" % (
         run.nsets, run.nsets * step_bytes / 1e6)

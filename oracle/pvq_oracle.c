@@ -30,7 +30,7 @@
  *
  * Parity unpinned by the paper (it prints no value for them): the order of
  * the fp32 roundings and the bit packing of the amplitude indices.  Both are
- * conventions of this build.
+ * conventions of this codec.
  */
 #include <math.h>
 #include <stdint.h>
@@ -269,7 +269,7 @@ uint16_t pvqo_f32_to_f16(float f) { return f32_to_f16_rne(f); }
 float pvqo_f16_to_f32(uint16_t h) { return f16_to_f32(h); }
 
 /*
- * The one summation order of this build: a balanced tree over contiguous
+ * The one summation order of this codec: a balanced tree over contiguous
  * halves, tree(lo,hi) = tree(lo,mid) + tree(mid,hi), mid the midpoint, each
  * addition rounded to binary32.  n must be a power of two.
  */
@@ -649,7 +649,7 @@ int pvqo_decode(const uint32_t *codes, const uint8_t *scale_idx, const float *ro
  * H is applied as log2(block) stages of butterflies with strides 1, 2, 4, ...:
  * (a, b) -> (a + b, a - b) on elements j and j + stride, each sum rounded to
  * binary32; the scale is the binary32 nearest to 1/sqrt(block), applied last
- * with one multiplication.  That order is a convention of this build (parity
+ * with one multiplication.  That order is a convention of this codec (parity
  * unpinned by the paper); the result is pinned to H by exact cases.
  * dtype 0 = fp32 in, 1 = bf16 in; out is fp32 [rows][cols].
  */
