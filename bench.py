@@ -518,7 +518,8 @@ def main():
     for name, ms_list in per.items():
         avg = sum(ms_list) / len(ms_list)
         nbytes = algorithmic_bytes(wl, name)
-        kernels[name] = {"avg_ms": avg, "min_ms": min(ms_list), "algorithmic_bytes": nbytes,
+        kernels[name] = {"avg_ms": avg, "median_ms": sorted(ms_list)[len(ms_list) // 2], "min_ms": min(ms_list),
+                         "algorithmic_bytes": nbytes,
                          "GBps": nbytes / (avg * 1e-3) / 1e9, "Gweights_per_s": wl.weights / (avg * 1e-3) / 1e9,
                          "frac_of_%s_hbm" % peak_kind: nbytes / (avg * 1e-3) / 1e9 / peak,
                          "frac_of_nominal_8TBps": nbytes / (avg * 1e-3) / 1e9 / 8000.0}
