@@ -390,9 +390,10 @@ __device__ __forceinline__ void walk_step_w6(uint32_t (&r)[6], uint32_t& p, int&
           "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
-// Middle phase for 5- and 6-word codes: once every r of the warp is below 2^126 the steps work
-// on four words (sign-bit compares) while still reading the 24-byte entries; an entry that
-// does not fit 126 bits is larger than any such r and fails its test.
+// Middle phase for 5- and 6-word codes: once every r of the warp and the entry it is about to
+// read are below 2^126 the steps work on four words (sign-bit compares), reading the low 16
+// bytes of the 24-byte entries.  The entries along a path never grow (N(n,k) is monotone in n
+// and k), so every later entry fits as well.
 template <typename YT, int U>
 __device__ __forceinline__ void walk_step_4of6(mp<4>& r, uint32_t& p, int& v, uint32_t& y, const int D,
                                                const Factors f) {
@@ -400,13 +401,9 @@ __device__ __forceinline__ void walk_step_4of6(mp<4>& r, uint32_t& p, int& v, ui
     asm volatile(
         "{\n\t"
         ".reg .pred pl, g1, mo, m2, ng;\n\t"
-        ".reg .u32 t0, t1, t2, t3, t4, t5, a0, a1, a2, a3, b0, b1, b2, b3, big, xh, val;\n\t"
+        ".reg .u32 t0, t1, t2, t3, a0, a1, a2, a3, b0, b1, b2, b3, xh, val;\n\t"
         "ld.shared.v2.u32 {t0, t1}, [%6+%10];\n\t"
         "ld.shared.v2.u32 {t2, t3}, [%6+%11];\n\t"
-        "ld.shared.v2.u32 {t4, t5}, [%6+%12];\n\t"
-        "or.b32 big, t4, t5;\n\t"
-        "shr.u32 xh, t3, 30;\n\t"
-        "or.b32 big, big, xh;\n\t"             // non-zero: the entry is 2^126 or more
         "sub.cc.u32 a0, %0, t0;\n\t"
         "subc.cc.u32 a1, %1, t1;\n\t"
         "subc.cc.u32 a2, %2, t2;\n\t"
@@ -417,7 +414,6 @@ __device__ __forceinline__ void walk_step_4of6(mp<4>& r, uint32_t& p, int& v, ui
         "subc.u32 b3, a3, t3;\n\t"
         "setp.gt.s32 pl, %4, 0;\n\t"
         "setp.ge.s32 g1, a3, 0;\n\t"
-        "setp.eq.and.u32 g1, big, 0, g1;\n\t"
         "selp.u32 xh, b3, a3, pl;\n\t"
         "setp.ge.and.s32 mo, xh, 0, g1;\n\t"
         "and.pred ng, g1, pl;\n\t"
@@ -491,7 +487,10 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
 #pragma unroll
             for (int w = 4; w < PW; ++w) hi |= r.w[w];
             if (next_words == 4) {
-                if constexpr (PW > 3) hi |= r.w[3] >> 30;
+                if constexpr (PW > 4) {  // r and the entry of the coming step below 2^126
+                    const mp<6> t = load_entry<6, 0>(p);
+                    hi |= (r.w[3] >> 30) | t.w[4] | t.w[5] | (t.w[3] >> 30);
+                }
             } else {
 #pragma unroll
                 for (int w = 2; w < PW && w < 4; ++w) hi |= r.w[w];
