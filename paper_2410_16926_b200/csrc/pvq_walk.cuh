@@ -390,10 +390,10 @@ __device__ __forceinline__ void walk_step_w6(uint32_t (&r)[6], uint32_t& p, int&
           "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
-// Middle phase for 5- and 6-word codes: once every r of the warp and the entry it is about to
-// read are below 2^126 the steps work on four words (sign-bit compares), reading the low 16
-// bytes of the 24-byte entries.  The entries along a path never grow (N(n,k) is monotone in n
-// and k), so every later entry fits as well.
+// Middle phases for 5- and 6-word codes: once every r of the warp and the entry it is about to
+// read are below 2^(32 M - 2) the steps work on M = 5, 4, then 3 words (sign-bit compares),
+// reading the low words of the 24-byte entries.  The entries along a path never grow (N(n,k)
+// is monotone in n and k), so every later entry fits as well.
 template <typename YT, int U>
 __device__ __forceinline__ void walk_step_4of6(mp<4>& r, uint32_t& p, int& v, uint32_t& y, const int D,
                                                const Factors f) {
@@ -439,6 +439,97 @@ __device__ __forceinline__ void walk_step_4of6(mp<4>& r, uint32_t& p, int& v, ui
           "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
+template <typename YT, int U>
+__device__ __forceinline__ void walk_step_5of6(mp<5>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                               const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, t2, t3, t4, t5, a0, a1, a2, a3, a4, b0, b1, b2, b3, b4, xh, val;\n\t"
+        "ld.shared.v2.u32 {t0, t1}, [%7+%11];\n\t"
+        "ld.shared.v2.u32 {t2, t3}, [%7+%12];\n\t"
+        "ld.shared.v2.u32 {t4, t5}, [%7+%13];\n\t"
+        "sub.cc.u32 a0, %0, t0;\n\t"
+        "subc.cc.u32 a1, %1, t1;\n\t"
+        "subc.cc.u32 a2, %2, t2;\n\t"
+        "subc.cc.u32 a3, %3, t3;\n\t"
+        "subc.u32 a4, %4, t4;\n\t"
+        "sub.cc.u32 b0, a0, t0;\n\t"
+        "subc.cc.u32 b1, a1, t1;\n\t"
+        "subc.cc.u32 b2, a2, t2;\n\t"
+        "subc.cc.u32 b3, a3, t3;\n\t"
+        "subc.u32 b4, a4, t4;\n\t"
+        "setp.gt.s32 pl, %5, 0;\n\t"
+        "setp.ge.s32 g1, a4, 0;\n\t"
+        "selp.u32 xh, b4, a4, pl;\n\t"
+        "setp.ge.and.s32 mo, xh, 0, g1;\n\t"
+        "and.pred ng, g1, pl;\n\t"
+        "and.pred m2, mo, pl;\n\t"
+        "@g1 mad.lo.u32 %0, a0, %8, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %8, 0;\n\t"
+        "@g1 mad.lo.u32 %2, a2, %8, 0;\n\t"
+        "@g1 mad.lo.u32 %3, a3, %8, 0;\n\t"
+        "@g1 mad.lo.u32 %4, a4, %8, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %8, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %8, 0;\n\t"
+        "@m2 mad.lo.u32 %2, b2, %8, 0;\n\t"
+        "@m2 mad.lo.u32 %3, b3, %8, 0;\n\t"
+        "@m2 mad.lo.u32 %4, b4, %8, 0;\n\t"
+        "mad.lo.u32 val, %5, %8, %16;\n\t"
+        "@ng mad.lo.u32 val, %5, %9, %16;\n\t"
+        "st.shared.u%15 [%6], val;\n\t"
+        "@!mo add.u32 %6, %6, %14;\n\t"
+        "@!mo add.u32 %7, %7, %10;\n\t"
+        "mad.lo.u32 %5, %5, %8, %8;\n\t"
+        "@!mo mov.u32 %5, 0;\n\t"
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(r.w[3]), "+r"(r.w[4]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 24), "n"(-U * 24 + 8), "n"(-U * 24 + 16), "n"(SZ),
+          "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+template <typename YT, int U>
+__device__ __forceinline__ void walk_step_3of6(mp<3>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                               const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, t2, t3, a0, a1, a2, b0, b1, b2, xh, val;\n\t"
+        "ld.shared.v2.u32 {t0, t1}, [%5+%9];\n\t"
+        "ld.shared.v2.u32 {t2, t3}, [%5+%10];\n\t"
+        "sub.cc.u32 a0, %0, t0;\n\t"
+        "subc.cc.u32 a1, %1, t1;\n\t"
+        "subc.u32 a2, %2, t2;\n\t"
+        "sub.cc.u32 b0, a0, t0;\n\t"
+        "subc.cc.u32 b1, a1, t1;\n\t"
+        "subc.u32 b2, a2, t2;\n\t"
+        "setp.gt.s32 pl, %3, 0;\n\t"
+        "setp.ge.s32 g1, a2, 0;\n\t"
+        "selp.u32 xh, b2, a2, pl;\n\t"
+        "setp.ge.and.s32 mo, xh, 0, g1;\n\t"
+        "and.pred ng, g1, pl;\n\t"
+        "and.pred m2, mo, pl;\n\t"
+        "@g1 mad.lo.u32 %0, a0, %6, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %6, 0;\n\t"
+        "@g1 mad.lo.u32 %2, a2, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %2, b2, %6, 0;\n\t"
+        "mad.lo.u32 val, %3, %6, %14;\n\t"
+        "@ng mad.lo.u32 val, %3, %7, %14;\n\t"
+        "st.shared.u%13 [%4], val;\n\t"
+        "@!mo add.u32 %4, %4, %12;\n\t"
+        "@!mo add.u32 %5, %5, %8;\n\t"
+        "mad.lo.u32 %3, %3, %6, %6;\n\t"
+        "@!mo mov.u32 %3, 0;\n\t"
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 24), "n"(-U * 24 + 8), "n"(-U * 24 + 16), "n"(SZ),
+          "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
 #undef PVQ_WIDE_TAIL
 
 template <int PW, int EB, bool HEADROOM, typename YT, int U>
@@ -448,8 +539,12 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
         walk_step_1<EB, YT, U>(r.w[0], p, v, y, D, f);
     else if constexpr (HEADROOM && PW == 2)
         walk_step_2<EB, YT, U>(r, p, v, y, D, f);
+    else if constexpr (HEADROOM && PW == 5 && EB == 24)
+        walk_step_5of6<YT, U>(r, p, v, y, D, f);
     else if constexpr (HEADROOM && PW == 4 && EB == 24)
         walk_step_4of6<YT, U>(r, p, v, y, D, f);
+    else if constexpr (HEADROOM && PW == 3 && EB == 24)
+        walk_step_3of6<YT, U>(r, p, v, y, D, f);
     else if constexpr (!HEADROOM && PW == 3)
         walk_step_w3<YT, U>(r, p, v, y, D, f);
     else if constexpr (!HEADROOM && PW == 4)
@@ -466,8 +561,8 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
 }
 
 // Runs steps s .. S-1 on PW-word integers with the table `tab` (entries of EB bytes),
-// leaving early, at a multiple of 8 steps, once every thread's r fits `next_words` words
-// with two bits to spare.  Returns the step reached.
+// leaving early, at a multiple of 8 steps, once every thread can go on in `next_words` words.
+// Returns the step reached.
 template <int PW, int EB, bool HEADROOM, int CW, typename YT>
 __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab, int rowlen, int K, int s,
                                           const int S, const int next_words, const Factors f) {
@@ -482,18 +577,23 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
 
     while (s + 8 <= S) {
         if (next_words > 0) {
-            // does r fit next_words (4, 2 or 1) words with the two top bits clear?
+            // can every thread go on in next_words words?  2 or 1: on a narrow table with its large
+            // values saturated, when r has the two top bits of that width clear; 3 to 5: on this
+            // table (24-byte entries), when r and the entry of the coming step have them clear
             uint32_t hi = 0;
-#pragma unroll
-            for (int w = 4; w < PW; ++w) hi |= r.w[w];
-            if (next_words == 4) {
-                if constexpr (PW > 4) {  // r and the entry of the coming step below 2^126
+            if (next_words >= 3) {
+                if constexpr (EB == 24) {
                     const mp<6> t = load_entry<6, 0>(p);
-                    hi |= (r.w[3] >> 30) | t.w[4] | t.w[5] | (t.w[3] >> 30);
+#pragma unroll
+                    for (int w = 2; w < 6; ++w) {
+                        const uint32_t rw = w < PW ? r.w[w < PW ? w : 0] : 0u;
+                        if (w >= next_words) hi |= rw | t.w[w];
+                        if (w == next_words - 1) hi |= (rw | t.w[w]) >> 30;
+                    }
                 }
             } else {
 #pragma unroll
-                for (int w = 2; w < PW && w < 4; ++w) hi |= r.w[w];
+                for (int w = 2; w < PW; ++w) hi |= r.w[w];
                 if constexpr (PW > 1) hi |= next_words == 2 ? (r.w[1] >> 30) : r.w[1];
                 if (next_words == 1) hi |= r.w[0] >> 30;
             }
@@ -569,9 +669,13 @@ __device__ __forceinline__ void walk_code(mp<W>& c, const WalkTables& t, int K, 
     st.y = st.y0 = shared_addr(yslots);
     int s = 0;
     const int narrow = t.has2 ? 2 : (t.has1 ? 1 : 0);
-    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, W > 4 ? 4 : narrow, t.f);
-    if constexpr (W > 4) {  // four-word arithmetic on the same table
-        if (s < S) s = walk_phase<4, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
+    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, W > 5 ? 5 : (W > 4 ? 4 : narrow), t.f);
+    if constexpr (W > 4) {  // fewer words on the same table as r shrinks
+        if constexpr (W > 5) {
+            if (s < S) s = walk_phase<5, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, 4, t.f);
+        }
+        if (s < S) s = walk_phase<4, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, 3, t.f);
+        if (s < S) s = walk_phase<3, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
     }
     if constexpr (W > 2) {
         if (s < S && t.has2) s = walk_phase<2, 8, true, W, YT>(c, st, t.tab2, t.rowlen, K, s, S, t.has1 ? 1 : 0, t.f);
