@@ -530,6 +530,48 @@ __device__ __forceinline__ void walk_step_3of6(mp<3>& r, uint32_t& p, int& v, ui
           "n"(SZ * 8), "n"(kSlotBias<YT>)
         : "memory");
 }
+// The same for 3- and 4-word codes (16-byte entries): three words with sign-bit compares once
+// r and the coming entry are below 2^94.
+template <typename YT, int U>
+__device__ __forceinline__ void walk_step_3of4(mp<3>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                               const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred pl, g1, mo, m2, ng;\n\t"
+        ".reg .u32 t0, t1, t2, t3, a0, a1, a2, b0, b1, b2, xh, val;\n\t"
+        "ld.shared.v4.u32 {t0, t1, t2, t3}, [%5+%9];\n\t"
+        "sub.cc.u32 a0, %0, t0;\n\t"
+        "subc.cc.u32 a1, %1, t1;\n\t"
+        "subc.u32 a2, %2, t2;\n\t"
+        "sub.cc.u32 b0, a0, t0;\n\t"
+        "subc.cc.u32 b1, a1, t1;\n\t"
+        "subc.u32 b2, a2, t2;\n\t"
+        "setp.gt.s32 pl, %3, 0;\n\t"
+        "setp.ge.s32 g1, a2, 0;\n\t"
+        "selp.u32 xh, b2, a2, pl;\n\t"
+        "setp.ge.and.s32 mo, xh, 0, g1;\n\t"
+        "and.pred ng, g1, pl;\n\t"
+        "and.pred m2, mo, pl;\n\t"
+        "@g1 mad.lo.u32 %0, a0, %6, 0;\n\t"
+        "@g1 mad.lo.u32 %1, a1, %6, 0;\n\t"
+        "@g1 mad.lo.u32 %2, a2, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %0, b0, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %1, b1, %6, 0;\n\t"
+        "@m2 mad.lo.u32 %2, b2, %6, 0;\n\t"
+        "mad.lo.u32 val, %3, %6, %14;\n\t"
+        "@ng mad.lo.u32 val, %3, %7, %14;\n\t"
+        "st.shared.u%13 [%4], val;\n\t"
+        "@!mo add.u32 %4, %4, %12;\n\t"
+        "@!mo add.u32 %5, %5, %8;\n\t"
+        "mad.lo.u32 %3, %3, %6, %6;\n\t"
+        "@!mo mov.u32 %3, 0;\n\t"
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(-U * 16), "n"(-U * 16 + 8), "n"(-U * 16 + 16), "n"(SZ),
+          "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
 #undef PVQ_WIDE_TAIL
 
 template <int PW, int EB, bool HEADROOM, typename YT, int U>
@@ -545,6 +587,8 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
         walk_step_4of6<YT, U>(r, p, v, y, D, f);
     else if constexpr (HEADROOM && PW == 3 && EB == 24)
         walk_step_3of6<YT, U>(r, p, v, y, D, f);
+    else if constexpr (HEADROOM && PW == 3 && EB == 16)
+        walk_step_3of4<YT, U>(r, p, v, y, D, f);
     else if constexpr (!HEADROOM && PW == 3)
         walk_step_w3<YT, U>(r, p, v, y, D, f);
     else if constexpr (!HEADROOM && PW == 4)
@@ -579,13 +623,13 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
         if (next_words > 0) {
             // can every thread go on in next_words words?  2 or 1: on a narrow table with its large
             // values saturated, when r has the two top bits of that width clear; 3 to 5: on this
-            // table (24-byte entries), when r and the entry of the coming step have them clear
+            // table, when r and the entry of the coming step have them clear
             uint32_t hi = 0;
             if (next_words >= 3) {
-                if constexpr (EB == 24) {
-                    const mp<6> t = load_entry<6, 0>(p);
+                if constexpr (EB == 24 || EB == 16) {
+                    const mp<EB / 4> t = load_entry<EB / 4, 0>(p);
 #pragma unroll
-                    for (int w = 2; w < 6; ++w) {
+                    for (int w = 2; w < EB / 4; ++w) {
                         const uint32_t rw = w < PW ? r.w[w < PW ? w : 0] : 0u;
                         if (w >= next_words) hi |= rw | t.w[w];
                         if (w == next_words - 1) hi |= (rw | t.w[w]) >> 30;
@@ -669,7 +713,11 @@ __device__ __forceinline__ void walk_code(mp<W>& c, const WalkTables& t, int K, 
     st.y = st.y0 = shared_addr(yslots);
     int s = 0;
     const int narrow = t.has2 ? 2 : (t.has1 ? 1 : 0);
-    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, W > 5 ? 5 : (W > 4 ? 4 : narrow), t.f);
+    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S,
+                                            W > 5 ? 5 : (W > 4 ? 4 : (W > 2 ? 3 : narrow)), t.f);
+    if constexpr (W == 3 || W == 4) {  // three words with sign-bit compares on the same table
+        if (s < S) s = walk_phase<3, 16, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
+    }
     if constexpr (W > 4) {  // fewer words on the same table as r shrinks
         if constexpr (W > 5) {
             if (s < S) s = walk_phase<5, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, 4, t.f);
