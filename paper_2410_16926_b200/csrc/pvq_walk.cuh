@@ -607,7 +607,7 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
 // Runs steps s .. S-1 on PW-word integers with the table `tab` (entries of EB bytes),
 // leaving early, at a multiple of 8 steps, once every thread can go on in `next_words` words.
 // Returns the step reached.
-template <int PW, int EB, bool HEADROOM, int CW, typename YT>
+template <int PW, int EB, bool HEADROOM, bool NEXT_SAME, int CW, typename YT>
 __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab, int rowlen, int K, int s,
                                           const int S, const int next_words, const Factors f) {
     mp<PW> r;
@@ -621,19 +621,17 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
 
     while (s + 8 <= S) {
         if (next_words > 0) {
-            // can every thread go on in next_words words?  2 or 1: on a narrow table with its large
-            // values saturated, when r has the two top bits of that width clear; 3 to 5: on this
-            // table, when r and the entry of the coming step have them clear
+            // can every thread go on in next_words words?  On a narrow table with its large values
+            // saturated: when r has the two top bits of that width clear.  NEXT_SAME, on this
+            // table with sign-bit compares: when r and the entry of the coming step have them clear.
             uint32_t hi = 0;
-            if (next_words >= 3) {
-                if constexpr (EB == 24 || EB == 16) {
-                    const mp<EB / 4> t = load_entry<EB / 4, 0>(p);
+            if constexpr (NEXT_SAME) {
+                const mp<EB / 4> t = load_entry<EB / 4, 0>(p);
 #pragma unroll
-                    for (int w = 2; w < EB / 4; ++w) {
-                        const uint32_t rw = w < PW ? r.w[w < PW ? w : 0] : 0u;
-                        if (w >= next_words) hi |= rw | t.w[w];
-                        if (w == next_words - 1) hi |= (rw | t.w[w]) >> 30;
-                    }
+                for (int w = 0; w < EB / 4; ++w) {
+                    const uint32_t rw = w < PW ? r.w[w < PW ? w : 0] : 0u;
+                    if (w >= next_words) hi |= rw | t.w[w];
+                    if (w == next_words - 1) hi |= (rw | t.w[w]) >> 30;
                 }
             } else {
 #pragma unroll
@@ -713,23 +711,31 @@ __device__ __forceinline__ void walk_code(mp<W>& c, const WalkTables& t, int K, 
     st.y = st.y0 = shared_addr(yslots);
     int s = 0;
     const int narrow = t.has2 ? 2 : (t.has1 ? 1 : 0);
-    s = walk_phase<W, TW * 4, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S,
-                                            W > 5 ? 5 : (W > 4 ? 4 : (W > 2 ? 3 : narrow)), t.f);
-    if constexpr (W == 3 || W == 4) {  // three words with sign-bit compares on the same table
-        if (s < S) s = walk_phase<3, 16, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
+    // widest phase, then fewer words (or, for two-word codes, the same two) with sign-bit
+    // compares on the same table as r shrinks
+    constexpr int kSame = W > 5 ? 5 : (W > 4 ? 4 : (W > 2 ? 3 : (W == 2 ? 2 : 0)));
+    if constexpr (kSame > 0)
+        s = walk_phase<W, TW * 4, false, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, kSame, t.f);
+    else
+        s = walk_phase<W, TW * 4, false, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
+    if constexpr (W == 2) {
+        if (s < S) s = walk_phase<2, 8, true, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
     }
-    if constexpr (W > 4) {  // fewer words on the same table as r shrinks
+    if constexpr (W == 3 || W == 4) {
+        if (s < S) s = walk_phase<3, 16, true, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
+    }
+    if constexpr (W > 4) {
         if constexpr (W > 5) {
-            if (s < S) s = walk_phase<5, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, 4, t.f);
+            if (s < S) s = walk_phase<5, 24, true, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, 4, t.f);
         }
-        if (s < S) s = walk_phase<4, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, 3, t.f);
-        if (s < S) s = walk_phase<3, 24, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
+        if (s < S) s = walk_phase<4, 24, true, true, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, 3, t.f);
+        if (s < S) s = walk_phase<3, 24, true, false, W, YT>(c, st, t.tab0, t.rowlen, K, s, S, narrow, t.f);
     }
     if constexpr (W > 2) {
-        if (s < S && t.has2) s = walk_phase<2, 8, true, W, YT>(c, st, t.tab2, t.rowlen, K, s, S, t.has1 ? 1 : 0, t.f);
+        if (s < S && t.has2) s = walk_phase<2, 8, true, false, W, YT>(c, st, t.tab2, t.rowlen, K, s, S, t.has1 ? 1 : 0, t.f);
     }
     if constexpr (W > 1) {
-        if (s < S && t.has1) s = walk_phase<1, 4, true, W, YT>(c, st, t.tab1, t.rowlen, K, s, S, 0, t.f);
+        if (s < S && t.has1) s = walk_phase<1, 4, true, false, W, YT>(c, st, t.tab1, t.rowlen, K, s, S, 0, t.f);
     }
 }
 
