@@ -17,11 +17,13 @@
 // data-dependent branch, and their table reads fall on neighbouring diagonal
 // cells, which the table layout puts in different banks.
 //
-// r only shrinks.  Once every thread of the warp has r below 2^62 (2^30) the warp
-// continues in a copy of the loop that works on two-word (one-word) integers
-// and reads a table of that width, whose larger entries are replaced by 2^62 (2^30):
-// no r of that phase reaches them, and with two spare bits the sign of a difference
-// tells the comparison.
+// r only shrinks, and so do the entries along a path (N(n,k) is monotone in n and k).
+// The warp therefore narrows its arithmetic as it goes.  First on the same table: once
+// every thread's r and the entry it is about to read leave the two top bits of a narrower
+// width free, the steps work on that many words, and with two spare bits the sign of a
+// difference tells the comparison.  Then, once every thread has r below 2^62 (2^30), in a
+// copy of the loop that works on two-word (one-word) integers and reads a table of that
+// width, whose larger entries are replaced by 2^62 (2^30): no r of that phase reaches them.
 #pragma once
 #include "mp_uint.cuh"
 #include "pvq_internal.cuh"
