@@ -91,7 +91,8 @@ def make_workload(name):
     from paper_2410_16926_b200 import inputs
     return {"c1": inputs.config1, "c2": inputs.config2, "c3": inputs.config3, "c4": inputs.config4,
             "c5": inputs.config5, "c5r": inputs.config5_unrotated, "c6": inputs.config6, "c7": inputs.config7,
-            "c8": inputs.config8, "c9": inputs.config9, "c10": inputs.config10}[name]()
+            "c8": inputs.config8, "c9": inputs.config9, "c10": inputs.config10,
+            "c10r": inputs.config10_unrotated}[name]()
 
 
 # ------------------------------------------------------------------------ clocks
@@ -434,7 +435,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5000)
     ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c5r", "c6", "c7", "c8", "c9", "c10"])
+    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c5r", "c6", "c7", "c8", "c9", "c10", "c10r"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true",

@@ -133,8 +133,7 @@ int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, f
  *              words); cols % N == 0; G >= 2.  Codes of up to 2, 3, 4, 6 words at N = 8, 16,
  *              32, 64 run on the kernels with the tables in shared memory.  Wider codes at
  *              N >= 16, and N = 128 and 256, run on slower kernels that keep the tables in
- *              global memory (the paper's grid of group sizes and direction bits, Sec. 4.1);
- *              the rotating entry points have only the former.
+ *              global memory (the paper's grid of group sizes and direction bits, Sec. 4.1).
  *   scale_bits 1..8 (quantile index), or 16 (see pvq_encode_amp).
  *   d_table    from pvq_build_count_table(N, K, ...).
  *   d_edges    2^scale_bits - 1 bin edges.
@@ -195,8 +194,8 @@ int pvq_encode_amp(const void* d_x, int dtype, int64_t rows, int64_t cols, int64
  *   block      a power of two, a multiple of N, dividing cols, at most 16384.
  * Arithmetic: fp32; the sign flip, then butterflies (a, b) -> (a + b, a - b) with strides
  * 1, 2, 4, ..., block/2, one rounding each, then one multiplication by the fp32 nearest to
- * 1/sqrt(block).  The other arguments are those of pvq_encode / pvq_roundtrip; the fused form
- * needs K <= 127. */
+ * 1/sqrt(block).  The other arguments are those of pvq_encode / pvq_roundtrip; on the kernels
+ * with the tables in shared memory the fused form needs K <= 127. */
 int pvq_rotate_encode(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t ld, int block,
                       const float* d_signs, int N, int K, int scale_bits, const uint32_t* d_table,
                       const float* d_edges, uint32_t* d_codes, uint8_t* d_scale_idx, float* d_row_norm,

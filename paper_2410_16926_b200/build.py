@@ -45,7 +45,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return cmd, r
 
     if jobs:
-        with ThreadPoolExecutor(max_workers=min(8, len(jobs))) as ex:
+        with ThreadPoolExecutor(max_workers=min(os.cpu_count() or 8, len(jobs))) as ex:
             for cmd, r in ex.map(run, jobs):
                 if verbose or r.returncode != 0:
                     sys.stderr.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)

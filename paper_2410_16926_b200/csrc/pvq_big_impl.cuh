@@ -307,6 +307,7 @@ int launch_decode_big_t(BatchArgs& a, cudaStream_t stream) {
 
 struct BigSmem {
     uint32_t es_off, ss_off, edges_off, idx_off;
+    uint32_t xs_off;  // rotation: a second column per thread for the rotated values
     int ss_floats, idx_words;
 };
 
@@ -342,17 +343,18 @@ __device__ __forceinline__ void group_values8(const void* gx, int j, float (&x)[
 // Encoder for large groups: the steps of encode_kernel with the per-thread arrays (residuals
 // to sort, the point) in shared memory columns es[i * T + t], the input re-read
 // from global memory where it is needed, and the cumulative tables read from global memory.
-template <int N, int W, bool EXACT, bool BF16, bool FUSED>
+template <int N, int W, bool EXACT, bool BF16, bool FUSED, bool ROT>
 __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_constant__ BatchArgs a,
                                                                   const __grid_constant__ BigSmem sm) {
     extern __shared__ __align__(16) uint8_t smem[];
     const int T = blockDim.x;
     const int t = threadIdx.x;
     float* es = reinterpret_cast<float*>(smem + sm.es_off) + t;         // column of this thread, stride T
+    const float* xs = nullptr;  // rotation: the column that holds this thread's rotated group
     // The point lies over the upper half of this thread's es column, two entries to a word: that
     // half is dead once the cut value has been read from the sorted residuals (the least-squares
     // tree uses the lower half).
-    auto ms = [es, T](int i) -> short& {
+    auto ms = [&es, T](int i) -> short& {
         return reinterpret_cast<short*>(es + (N / 2 + (i >> 1)) * T)[i & 1];
     };
     float* s_ss = reinterpret_cast<float*>(smem + sm.ss_off);
@@ -391,12 +393,69 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
         for (int i = t; i < rpt * idx_words; i += T) s_idx[i] = 0u;
         __syncthreads();
 
+        // Rotation in front of the encoder (Sec. 2.3 / Sec. 3.3 Step 1, as rotate_tile does it for
+        // the small groups): x <- (x * s) H_B / sqrt(B) on every block of B = N * T0 consecutive
+        // columns.  The butterflies (a, b) -> (a + b, a - b) run with strides 1, 2, 4, ...: below N
+        // inside the thread's column, from N up between the columns of threads t and t ^ d (T0
+        // divides G, so both hold groups of the same block), written to the other of two columns
+        // with a barrier between stages.  Every sum is one fp32 addition.
+        if constexpr (ROT) {
+            float* xa = reinterpret_cast<float*>(smem + sm.xs_off) + t;
+            float* xb = reinterpret_cast<float*>(smem + sm.es_off) + t;
+            const int T0 = a.rot_block / N;
+            if (active) {
+                const float* sg = a.rot_signs + (g & (T0 - 1)) * N;
+                float x[8];
+                for (int j = 0; j < N / 8; ++j) {
+                    group_values8<BF16>(gx, j, x);
+#pragma unroll
+                    for (int p = 0; p < 8; ++p) xa[(8 * j + p) * T] = __fmul_rn(x[p], __ldg(sg + 8 * j + p));
+                }
+                for (int h = 1; h < N; h <<= 1) {
+                    for (int q = 0; q < N / 2; ++q) {
+                        const int j = ((q & ~(h - 1)) << 1) | (q & (h - 1));  // the q-th index with bit h clear
+                        const float u = xa[j * T], w = xa[(j + h) * T];
+                        xa[j * T] = __fadd_rn(u, w);
+                        xa[(j + h) * T] = __fsub_rn(u, w);
+                    }
+                }
+            }
+            for (int d = 1; d < T0; d <<= 1) {
+                __syncthreads();
+                if (active) {
+                    const float sgn = (t & d) != 0 ? -1.0f : 1.0f;  // a + b on the lower thread, a - b on the upper
+                    const float* pa = xa + ((t ^ d) - t);           // the partner's column
+                    for (int i = 0; i < N; ++i) xb[i * T] = __fmaf_rn(xa[i * T], sgn, pa[i * T]);
+                }
+                float* tmp = xa;
+                xa = xb;
+                xb = tmp;
+            }
+            if (T0 > 1) __syncthreads();  // nobody reads a partner's old column any more
+            if (active) {
+                const float scale = static_cast<float>(1.0 / sqrt(static_cast<double>(a.rot_block)));
+                for (int i = 0; i < N; ++i) xa[i * T] = __fmul_rn(xa[i * T], scale);
+            }
+            xs = xa;
+            es = xb;
+        }
+        // element i / elements 8j .. 8j+7 of the group the kernel works on
+        auto value = [&](int i) -> float { return ROT ? xs[i * T] : group_value<BF16>(gx, i); };
+        auto values8 = [&](int j, float (&x)[8]) {
+            if constexpr (ROT) {
+#pragma unroll
+                for (int p = 0; p < 8; ++p) x[p] = xs[(8 * j + p) * T];
+            } else {
+                group_values8<BF16>(gx, j, x);
+            }
+        };
+
         // group norms by the balanced tree, run level by level in the es column
         float l1 = 0.0f, ss = 0.0f;
         if (active) {
             float x[8];
             for (int j = 0; j < N / 8; ++j) {
-                group_values8<BF16>(gx, j, x);
+                values8(j, x);
 #pragma unroll
                 for (int p = 0; p < 4; ++p) es[(4 * j + p) * T] = __fadd_rn(fabsf(x[2 * p]), fabsf(x[2 * p + 1]));
             }
@@ -404,7 +463,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 for (int j = 0; j < len; ++j) es[j * T] = __fadd_rn(es[2 * j * T], es[(2 * j + 1) * T]);
             l1 = es[0];
             for (int j = 0; j < N / 8; ++j) {
-                group_values8<BF16>(gx, j, x);
+                values8(j, x);
 #pragma unroll
                 for (int p = 0; p < 4; ++p)
                     es[(4 * j + p) * T] = __fadd_rn(__fmul_rn(x[2 * p], x[2 * p]), __fmul_rn(x[2 * p + 1], x[2 * p + 1]));
@@ -435,7 +494,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 float sumf = 0.0f;
                 float x[8];
                 for (int j = 0; j < N / 8; ++j) {
-                    group_values8<BF16>(gx, j, x);
+                    values8(j, x);
 #pragma unroll
                     for (int p = 0; p < 8; ++p) {
                         const float av = __fmul_rn(fabsf(x[p]), gsc);
@@ -455,7 +514,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 int cnt = 0;
                 float x[8];
                 for (int j = 0; j < N / 8; ++j) {
-                    group_values8<BF16>(gx, j, x);
+                    values8(j, x);
 #pragma unroll
                     for (int p = 0; p < 8; ++p) {
                         const float av = __fmul_rn(fabsf(x[p]), gsc);
@@ -469,7 +528,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 }
                 int excess = cnt - d;
                 for (int i = N - 1; i >= 0 && excess > 0; --i) {  // equal residuals straddle the cut
-                    const float xi = group_value<BF16>(gx, i);
+                    const float xi = value(i);
                     const float av = __fmul_rn(fabsf(xi), gsc);
                     const float tt = __fadd_rd(av, kMagic);
                     if (__fsub_rn(av, __fsub_rn(tt, kMagic)) == v) {
@@ -486,7 +545,7 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
                 int ssy = 0;  // exact; converted once (it can pass 2^24 when K > 4095)
                 float x[8];
                 for (int j8 = 0; j8 < N / 8; ++j8) {
-                    group_values8<BF16>(gx, j8, x);
+                    values8(j8, x);
 #pragma unroll
                     for (int p = 0; p < 4; ++p) {
                         const int j = 4 * j8 + p;
@@ -588,17 +647,18 @@ __global__ void __launch_bounds__(kBigThreads) encode_big_kernel(const __grid_co
     }
 }
 
-template <int N, int W, bool EXACT, bool BF16, bool FUSED>
+template <int N, int W, bool EXACT, bool BF16, bool FUSED, bool ROT>
 int launch_encode_big_t(BatchArgs& a, cudaStream_t stream) {
     DeviceInfo di;
     int st = device_info(&di);
     if (st != PVQ_OK) return st;
     // a block covers whole rows: the fewest wasted thread slots among multiples of 32 whose
-    // columns fit in shared memory
+    // columns (one per thread, two when rotating) fit in shared memory
+    const unsigned columns = ROT ? 2u : 1u;
     int best = 0;
     long long best_cost = -1;
     for (int threads = 32; threads <= kBigThreads; threads += 32) {
-        if (static_cast<size_t>(threads) * N * 4u + 8192u > static_cast<size_t>(di.smem_max)) break;
+        if (static_cast<size_t>(threads) * N * 4u * columns + 8192u > static_cast<size_t>(di.smem_max)) break;
         long long cost = 0;
         bool ok = true;
         for (int i = 0; i < a.count && ok; ++i) {
@@ -627,14 +687,15 @@ int launch_encode_big_t(BatchArgs& a, cudaStream_t stream) {
     a.total_tiles = tiles;
     BigSmem sm;
     sm.es_off = 0;
-    sm.ss_off = static_cast<uint32_t>(threads) * N * 4u;
+    sm.xs_off = static_cast<uint32_t>(threads) * N * 4u;
+    sm.ss_off = sm.xs_off * columns;
     sm.edges_off = sm.ss_off + ss_floats * 4u;
     sm.idx_off = sm.edges_off + 256u * 4u;
     sm.ss_floats = ss_floats;
     sm.idx_words = idx_words;
     const size_t smem = sm.idx_off + idx_words * 4u;
     if (smem > static_cast<size_t>(di.smem_max)) return PVQ_ERR_UNSUPPORTED;
-    auto kern = encode_big_kernel<N, W, EXACT, BF16, FUSED>;
+    auto kern = encode_big_kernel<N, W, EXACT, BF16, FUSED, ROT>;
     int per_sm = 0;
     if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
@@ -649,11 +710,19 @@ int launch_big_w(BatchArgs& a, int dtype, bool decode, cudaStream_t s) {
     if (decode)
         return a.K <= 127 ? launch_decode_big_t<N, W, EXACT, int8_t>(a, s)
                           : launch_decode_big_t<N, W, EXACT, int16_t>(a, s);
+    const bool bf16 = dtype == PVQ_DTYPE_BF16;
+    if (a.rot_block != 0) {
+        if (a.fused)
+            return bf16 ? launch_encode_big_t<N, W, EXACT, true, true, true>(a, s)
+                        : launch_encode_big_t<N, W, EXACT, false, true, true>(a, s);
+        return bf16 ? launch_encode_big_t<N, W, EXACT, true, false, true>(a, s)
+                    : launch_encode_big_t<N, W, EXACT, false, false, true>(a, s);
+    }
     if (a.fused)
-        return dtype == PVQ_DTYPE_BF16 ? launch_encode_big_t<N, W, EXACT, true, true>(a, s)
-                                       : launch_encode_big_t<N, W, EXACT, false, true>(a, s);
-    return dtype == PVQ_DTYPE_BF16 ? launch_encode_big_t<N, W, EXACT, true, false>(a, s)
-                                   : launch_encode_big_t<N, W, EXACT, false, false>(a, s);
+        return bf16 ? launch_encode_big_t<N, W, EXACT, true, true, false>(a, s)
+                    : launch_encode_big_t<N, W, EXACT, false, true, false>(a, s);
+    return bf16 ? launch_encode_big_t<N, W, EXACT, true, false, false>(a, s)
+                : launch_encode_big_t<N, W, EXACT, false, false, false>(a, s);
 }
 
 }  // namespace

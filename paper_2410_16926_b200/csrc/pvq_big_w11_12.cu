@@ -1,0 +1,15 @@
+// Group size 128, codes of 11 to 12 words: kernels that compute in exactly the code's width
+// (one of the translation units the instantiations are spread over, to build in parallel).
+#include "pvq_big_impl.cuh"
+
+namespace pvq {
+
+int launch_big_128_w11_12(BatchArgs& a, int dtype, int W, bool decode, cudaStream_t s) {
+    switch (W) {
+        case 11: return launch_big_w<128, 11, true>(a, dtype, decode, s);
+        case 12: return launch_big_w<128, 12, true>(a, dtype, decode, s);
+        default: return PVQ_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace pvq

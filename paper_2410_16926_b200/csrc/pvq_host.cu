@@ -325,8 +325,7 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // codes the shared-memory kernels are built for, by group size
     const int fast_words = c.N == 8 ? 2 : (c.N == 16 ? 3 : (c.N == 32 ? 4 : (c.N == 64 ? 6 : 0)));
-    if (c.W > fast_words) {  // large groups, wide codes: no rotation in front of the encoder
-        if (rot_block != 0) return PVQ_ERR_UNSUPPORTED;
+    if (c.W > fast_words) {  // large groups, wide codes
         a.fused = kind == 2 ? 1 : 0;
         return launch_big(a, dtype, c.N, c.W, kind == 1, s);
     }

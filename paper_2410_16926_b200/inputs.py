@@ -200,3 +200,11 @@ def config10(tokens=16384, hidden=4096) -> Workload:
     K = 386) and 16-bit amplitudes; fused encode -> decode."""
     wl = config5(tokens, hidden)
     return Workload("c10_bf16_activations_group128", 128, 512, 16, "roundtrip", wl.matrices)
+
+
+def config10_unrotated(tokens=16384, hidden=4096) -> Workload:
+    """config10 from the activations before their rotation (config5_unrotated's input and signs):
+    rotate -> encode -> decode in one kernel at group size 128."""
+    wl = config5_unrotated(tokens, hidden)
+    return Workload("c10r_bf16_activations_group128_rotated_on_the_fly", 128, 512, 16, "rotate_roundtrip",
+                    wl.matrices, rot_block=wl.rot_block, signs=wl.signs)

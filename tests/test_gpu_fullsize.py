@@ -152,6 +152,26 @@ def test_c10_activations_group_128_fused_sampled_rows():
     check_rows(wl, items, K, W, nrows=96, what=("out",))
 
 
+def test_c10r_activations_group_128_rotated_on_the_fly_sampled_rows():
+    wl = inputs.config10_unrotated()
+    K = pvq.max_pulses(wl.N, wl.index_bits)
+    W = pvq.code_words(wl.N, K)
+    table = pvq.build_count_table(wl.N, K)
+    items = workload_items(wl, K, W)
+    it = items[0]
+    signs = torch.from_numpy(wl.signs).to(DEV)
+    pvq.rotate_roundtrip(it["x"], wl.rot_block, signs, wl.N, K, wl.scale_bits, table, it["edges"], it["levels"],
+                         out=it["out"])
+    torch.cuda.synchronize()
+    m = wl.matrices[0]
+    rows = sample_rows(m.rows, 64, seed=77)
+    xr = po.rotate(np.ascontiguousarray(m.data[rows]), wl.rot_block, wl.signs)
+    enc = po.encode(xr, wl.N, K, wl.scale_bits, it["e_np"], W=W)
+    o_out, st = po.decode(*enc, wl.N, K, wl.scale_bits, it["l_np"])
+    r = torch.from_numpy(rows).to(DEV)
+    assert st == 0 and np.array_equal(bf16_bits(it["out"][r].contiguous()), o_out)
+
+
 def test_c9_group_16_sampled_rows():
     wl = inputs.config9()
     K = pvq.max_pulses(wl.N, wl.index_bits)

@@ -383,6 +383,13 @@ def test_library_codebook_end_to_end():
     (32, 64, 21, 512, 32, 8, "f32"),         # block = group: in-thread stages only
     (16, 40, 11, 192, 64, 4, "f32"),         # G = 12, three blocks per row
     (64, 192, 5, 3584, 512, 6, "bf16"),      # N = 64
+    # the kernels with the tables in global memory
+    (128, 512, 5, 4096, 4096, 8, "bf16"),    # activations at group size 128: a block spans 32 threads
+    (128, 384, 3, 1024, 128, 8, "f32"),      # block = group
+    (128, 256, 4, 2048, 512, 6, "bf16"),     # four threads per block
+    (64, 256, 6, 1024, 256, 8, "f32"),       # wide codes at N = 64
+    (256, 768, 2, 2048, 1024, 8, "bf16"),    # N = 256
+    (128, 384, 2, 16384, 16384, 4, "bf16"),  # a block of 128 threads
 ])
 def test_rotate_encode_and_roundtrip_parity(N, bits, rows, cols, block, b, kind):
     rng = np.random.default_rng(block + rows)
@@ -401,7 +408,8 @@ def test_rotate_encode_and_roundtrip_parity(N, bits, rows, cols, block, b, kind)
     assert np.array_equal(rnorm.cpu().numpy().view(np.uint32), o_rnorm.view(np.uint32)), "row norms"
     assert np.array_equal(sidx.cpu().numpy(), o_sidx), "amplitude indices"
     assert np.array_equal(as_u32(codes), o_codes), "codes"
-    if cd.K <= 127:
+    global_tables = cd.W > {8: 2, 16: 3, 32: 4, 64: 6}.get(N, 0)
+    if cd.K <= 127 or global_tables:
         out = pvq.rotate_roundtrip(x_dev, block, s_dev, cd.N, cd.K, cd.b, cd.table, cd.edges, cd.levels)
         torch.cuda.synchronize()
         assert np.array_equal(bf16_bits(out), o_out), "fused round trip"
