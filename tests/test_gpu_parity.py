@@ -323,10 +323,13 @@ def test_fused_roundtrip_global_table_kernels(N, bits, rows, cols, b, kind):
     assert np.array_equal(bf16_bits(out), o_out)
 
 
-def test_batched_calls_match_single_calls():
+@pytest.mark.parametrize("N,bits", [(32, 96), (128, 384), (64, 320)])
+def test_batched_calls_match_single_calls(N, bits):
+    """All matrices of a decoder layer in one launch, on the shared-memory kernels and (group size
+    128; wide codes) on the global-table kernels, whose blocks then cover rows of different lengths."""
     wl = inputs.config3(scale_div=256)       # the seven matrices of a layer, 1/256 of the rows
-    N, b = wl.N, wl.scale_bits
-    K = pvq.max_pulses(N, wl.index_bits)
+    b = wl.scale_bits
+    K = pvq.max_pulses(N, bits)
     W = pvq.code_words(N, K)
     table = pvq.build_count_table(N, K)
     items, refs = [], []
