@@ -250,11 +250,13 @@ def test_non_finite_inputs_give_valid_codes(N, bits, b):
     assert np.array_equal(bf16_bits(out[f].contiguous()), o_out)
 
 
-def test_leading_dimensions():
-    N, rows, cols, ld, ldo = 32, 10, 256, 320, 288
+@pytest.mark.parametrize("N,bits,cols,ld,ldo", [(32, 96, 256, 320, 288), (128, 384, 1024, 1280, 1032),
+                                               (64, 256, 512, 520, 640)])
+def test_leading_dimensions(N, bits, cols, ld, ldo):
+    rows = 10
     rng = np.random.default_rng(8)
     x = inputs.f32_to_bf16_bits((rng.standard_normal((rows, cols))).astype(np.float32))
-    cd = Codec(N, 96, cols // N, 4)
+    cd = Codec(N, bits, cols // N, 4)
     big = torch.zeros((rows, ld), dtype=torch.bfloat16, device=DEV)
     big[:, :cols] = to_device(x, "bf16")
     enc_dev, enc_np = check_encode(cd, x, "bf16", x_dev=big[:, :cols])
@@ -266,21 +268,24 @@ def test_leading_dimensions():
     assert torch.all(out_big[:, cols:] == 7.0)       # nothing written past cols
 
 
-def test_invalid_codes_set_status_and_decode_to_zero():
-    cd = Codec(32, 64, 8, 8)
+@pytest.mark.parametrize("N,bits", [(32, 64), (128, 380), (64, 300)])
+def test_invalid_codes_set_status_and_decode_to_zero(N, bits):
+    cd = Codec(N, bits, 8, 8)
+    W = cd.W
     rng = np.random.default_rng(5)
-    x = rng.standard_normal((4, 256)).astype(np.float32)
+    x = rng.standard_normal((4, 8 * N)).astype(np.float32)
     enc_dev, enc_np = check_encode(cd, x, "f32")
     codes = enc_np[0].copy()
-    codes[1, 3, :] = 0xFFFFFFFF                      # >= N(32,22)
-    total = po.code_to_int(po.count_table(32, cd.K, 3)[32, cd.K])
-    codes[2, 0, :] = po.int_to_code(total, 2)         # the first invalid value
-    codes[2, 1, :] = po.int_to_code(total - 1, 2)     # the last valid one
+    codes[1, 3, :] = 0xFFFFFFFF                      # >= N(N,K)
+    total = po.code_to_int(po.count_table(N, cd.K, W + 1)[N, cd.K])
+    assert total < 1 << (32 * W)
+    codes[2, 0, :] = po.int_to_code(total, W)         # the first invalid value
+    codes[2, 1, :] = po.int_to_code(total - 1, W)     # the last valid one
     enc_np2 = (codes, enc_np[1], enc_np[2])
     enc_dev2 = (torch.from_numpy(codes.view(np.int32)).to(DEV), enc_dev[1], enc_dev[2])
     out = check_decode(cd, enc_dev2, enc_np2)
-    assert torch.all(out[1, 96:128] == 0) and torch.all(out[2, :32] == 0)
-    assert torch.any(out[2, 32:64] != 0)
+    assert torch.all(out[1, 3 * N:4 * N] == 0) and torch.all(out[2, :N] == 0)
+    assert torch.any(out[2, N:2 * N] != 0)
 
 
 def test_fused_roundtrip_equals_encode_then_decode():
