@@ -576,6 +576,313 @@ __device__ __forceinline__ void walk_step_3of4(mp<3>& r, uint32_t& p, int& v, ui
 }
 #undef PVQ_WIDE_TAIL
 
+// Eight consecutive steps in one asm statement, for the sign-bit forms.  Whether a pulse has
+// already been placed at the current position (v > 0) is, from the second step on, the previous
+// step's "one more pulse" predicate, so only the first step tests v.  Step u reads the entry
+// u entries to the left of p; the caller moves p left by eight entries afterwards.
+#define PVQ_STEP_1(OFF, PL, MO) \
+    "ld.shared.u32 t, [%3+" #OFF "];\n\t"     \
+    "mad.lo.u32 d2, t, %5, %0;\n\t"           \
+    "mad.lo.u32 d1, t, %5, d2;\n\t"           \
+    "setp.ge.s32 g1, d2, 0;\n\t"              \
+    "selp.u32 x, d1, d2, " #PL ";\n\t"        \
+    "setp.ge.s32 " #MO ", x, 0;\n\t"          \
+    "and.pred ng, g1, " #PL ";\n\t"           \
+    "@g1 mad.lo.u32 %0, d2, %4, 0;\n\t"       \
+    "@" #MO " mad.lo.u32 %0, x, %4, 0;\n\t"   \
+    "mad.lo.u32 val, %1, %4, %9;\n\t"         \
+    "@ng mad.lo.u32 val, %1, %5, %9;\n\t"     \
+    "st.shared.u%8 [%2], val;\n\t"            \
+    "@!" #MO " add.u32 %2, %2, %7;\n\t"       \
+    "@!" #MO " add.u32 %3, %3, %6;\n\t"       \
+    "mad.lo.u32 %1, %1, %4, %4;\n\t"          \
+    "@!" #MO " mov.u32 %1, 0;\n\t"
+template <typename YT>
+__device__ __forceinline__ void walk_block8_1(uint32_t& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                                const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred g1, m2, ng, pl0, mo0, mo1, mo2, mo3, mo4, mo5, mo6, mo7;\n\t"
+        ".reg .u32 t, d2, d1, x, val;\n\t"
+        "setp.gt.s32 pl0, %1, 0;\n\t"
+        PVQ_STEP_1(0, pl0, mo0)
+        PVQ_STEP_1(-4, mo0, mo1)
+        PVQ_STEP_1(-8, mo1, mo2)
+        PVQ_STEP_1(-12, mo2, mo3)
+        PVQ_STEP_1(-16, mo3, mo4)
+        PVQ_STEP_1(-20, mo4, mo5)
+        PVQ_STEP_1(-24, mo5, mo6)
+        PVQ_STEP_1(-28, mo6, mo7)
+        "}"
+        : "+r"(r), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+#undef PVQ_STEP_1
+
+#define PVQ_STEP_2(OFF, PL, MO) \
+    "ld.shared.v2.u32 {t0, t1}, [%4+" #OFF "];\n\t"   \
+    "sub.cc.u32 a0, %0, t0;\n\t"                      \
+    "subc.u32 a1, %1, t1;\n\t"                        \
+    "sub.cc.u32 b0, a0, t0;\n\t"                      \
+    "subc.u32 b1, a1, t1;\n\t"                        \
+    "setp.ge.s32 g1, a1, 0;\n\t"                      \
+    "selp.u32 xh, b1, a1, " #PL ";\n\t"               \
+    "setp.ge.and.s32 " #MO ", xh, 0, g1;\n\t"         \
+    "and.pred ng, g1, " #PL ";\n\t"                   \
+    "and.pred m2, " #MO ", " #PL ";\n\t"              \
+    "@g1 mad.lo.u32 %0, a0, %5, 0;\n\t"               \
+    "@g1 mad.lo.u32 %1, a1, %5, 0;\n\t"               \
+    "@m2 mad.lo.u32 %0, b0, %5, 0;\n\t"               \
+    "@m2 mad.lo.u32 %1, b1, %5, 0;\n\t"               \
+    "mad.lo.u32 val, %2, %5, %10;\n\t"                \
+    "@ng mad.lo.u32 val, %2, %6, %10;\n\t"            \
+    "st.shared.u%9 [%3], val;\n\t"                    \
+    "@!" #MO " add.u32 %3, %3, %8;\n\t"               \
+    "@!" #MO " add.u32 %4, %4, %7;\n\t"               \
+    "mad.lo.u32 %2, %2, %5, %5;\n\t"                  \
+    "@!" #MO " mov.u32 %2, 0;\n\t"
+template <typename YT>
+__device__ __forceinline__ void walk_block8_2(mp<2>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                                const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred g1, m2, ng, pl0, mo0, mo1, mo2, mo3, mo4, mo5, mo6, mo7;\n\t"
+        ".reg .u32 t0, t1, a0, a1, b0, b1, xh, val;\n\t"
+        "setp.gt.s32 pl0, %2, 0;\n\t"
+        PVQ_STEP_2(0, pl0, mo0)
+        PVQ_STEP_2(-8, mo0, mo1)
+        PVQ_STEP_2(-16, mo1, mo2)
+        PVQ_STEP_2(-24, mo2, mo3)
+        PVQ_STEP_2(-32, mo3, mo4)
+        PVQ_STEP_2(-40, mo4, mo5)
+        PVQ_STEP_2(-48, mo5, mo6)
+        PVQ_STEP_2(-56, mo6, mo7)
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+#undef PVQ_STEP_2
+
+#define PVQ_STEP_3OF4(OFF, PL, MO) \
+    "ld.shared.v4.u32 {t0, t1, t2, t3}, [%5+" #OFF "];\n\t"   \
+    "sub.cc.u32 a0, %0, t0;\n\t"                              \
+    "subc.cc.u32 a1, %1, t1;\n\t"                             \
+    "subc.u32 a2, %2, t2;\n\t"                                \
+    "sub.cc.u32 b0, a0, t0;\n\t"                              \
+    "subc.cc.u32 b1, a1, t1;\n\t"                             \
+    "subc.u32 b2, a2, t2;\n\t"                                \
+    "setp.ge.s32 g1, a2, 0;\n\t"                              \
+    "selp.u32 xh, b2, a2, " #PL ";\n\t"                       \
+    "setp.ge.and.s32 " #MO ", xh, 0, g1;\n\t"                 \
+    "and.pred ng, g1, " #PL ";\n\t"                           \
+    "and.pred m2, " #MO ", " #PL ";\n\t"                      \
+    "@g1 mad.lo.u32 %0, a0, %6, 0;\n\t"                       \
+    "@g1 mad.lo.u32 %1, a1, %6, 0;\n\t"                       \
+    "@g1 mad.lo.u32 %2, a2, %6, 0;\n\t"                       \
+    "@m2 mad.lo.u32 %0, b0, %6, 0;\n\t"                       \
+    "@m2 mad.lo.u32 %1, b1, %6, 0;\n\t"                       \
+    "@m2 mad.lo.u32 %2, b2, %6, 0;\n\t"                       \
+    "mad.lo.u32 val, %3, %6, %11;\n\t"                        \
+    "@ng mad.lo.u32 val, %3, %7, %11;\n\t"                    \
+    "st.shared.u%10 [%4], val;\n\t"                           \
+    "@!" #MO " add.u32 %4, %4, %9;\n\t"                       \
+    "@!" #MO " add.u32 %5, %5, %8;\n\t"                       \
+    "mad.lo.u32 %3, %3, %6, %6;\n\t"                          \
+    "@!" #MO " mov.u32 %3, 0;\n\t"
+template <typename YT>
+__device__ __forceinline__ void walk_block8_3of4(mp<3>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                                const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred g1, m2, ng, pl0, mo0, mo1, mo2, mo3, mo4, mo5, mo6, mo7;\n\t"
+        ".reg .u32 t0, t1, t2, t3, a0, a1, a2, b0, b1, b2, xh, val;\n\t"
+        "setp.gt.s32 pl0, %3, 0;\n\t"
+        PVQ_STEP_3OF4(0, pl0, mo0)
+        PVQ_STEP_3OF4(-16, mo0, mo1)
+        PVQ_STEP_3OF4(-32, mo1, mo2)
+        PVQ_STEP_3OF4(-48, mo2, mo3)
+        PVQ_STEP_3OF4(-64, mo3, mo4)
+        PVQ_STEP_3OF4(-80, mo4, mo5)
+        PVQ_STEP_3OF4(-96, mo5, mo6)
+        PVQ_STEP_3OF4(-112, mo6, mo7)
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+#undef PVQ_STEP_3OF4
+
+#define PVQ_STEP_3OF6(OFF, OFF8, OFF16, PL, MO) \
+    "ld.shared.v2.u32 {t0, t1}, [%5+" #OFF "];\n\t"    \
+    "ld.shared.v2.u32 {t2, t3}, [%5+" #OFF8 "];\n\t"   \
+    "sub.cc.u32 a0, %0, t0;\n\t"                       \
+    "subc.cc.u32 a1, %1, t1;\n\t"                      \
+    "subc.u32 a2, %2, t2;\n\t"                         \
+    "sub.cc.u32 b0, a0, t0;\n\t"                       \
+    "subc.cc.u32 b1, a1, t1;\n\t"                      \
+    "subc.u32 b2, a2, t2;\n\t"                         \
+    "setp.ge.s32 g1, a2, 0;\n\t"                       \
+    "selp.u32 xh, b2, a2, " #PL ";\n\t"                \
+    "setp.ge.and.s32 " #MO ", xh, 0, g1;\n\t"          \
+    "and.pred ng, g1, " #PL ";\n\t"                    \
+    "and.pred m2, " #MO ", " #PL ";\n\t"               \
+    "@g1 mad.lo.u32 %0, a0, %6, 0;\n\t"                \
+    "@g1 mad.lo.u32 %1, a1, %6, 0;\n\t"                \
+    "@g1 mad.lo.u32 %2, a2, %6, 0;\n\t"                \
+    "@m2 mad.lo.u32 %0, b0, %6, 0;\n\t"                \
+    "@m2 mad.lo.u32 %1, b1, %6, 0;\n\t"                \
+    "@m2 mad.lo.u32 %2, b2, %6, 0;\n\t"                \
+    "mad.lo.u32 val, %3, %6, %11;\n\t"                 \
+    "@ng mad.lo.u32 val, %3, %7, %11;\n\t"             \
+    "st.shared.u%10 [%4], val;\n\t"                    \
+    "@!" #MO " add.u32 %4, %4, %9;\n\t"                \
+    "@!" #MO " add.u32 %5, %5, %8;\n\t"                \
+    "mad.lo.u32 %3, %3, %6, %6;\n\t"                   \
+    "@!" #MO " mov.u32 %3, 0;\n\t"
+template <typename YT>
+__device__ __forceinline__ void walk_block8_3of6(mp<3>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                                const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred g1, m2, ng, pl0, mo0, mo1, mo2, mo3, mo4, mo5, mo6, mo7;\n\t"
+        ".reg .u32 t0, t1, t2, t3, t4, t5, a0, a1, a2, b0, b1, b2, xh, val;\n\t"
+        "setp.gt.s32 pl0, %3, 0;\n\t"
+        PVQ_STEP_3OF6(0, 8, 16, pl0, mo0)
+        PVQ_STEP_3OF6(-24, -16, -8, mo0, mo1)
+        PVQ_STEP_3OF6(-48, -40, -32, mo1, mo2)
+        PVQ_STEP_3OF6(-72, -64, -56, mo2, mo3)
+        PVQ_STEP_3OF6(-96, -88, -80, mo3, mo4)
+        PVQ_STEP_3OF6(-120, -112, -104, mo4, mo5)
+        PVQ_STEP_3OF6(-144, -136, -128, mo5, mo6)
+        PVQ_STEP_3OF6(-168, -160, -152, mo6, mo7)
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+#undef PVQ_STEP_3OF6
+
+#define PVQ_STEP_4OF6(OFF, OFF8, OFF16, PL, MO) \
+    "ld.shared.v2.u32 {t0, t1}, [%6+" #OFF "];\n\t"    \
+    "ld.shared.v2.u32 {t2, t3}, [%6+" #OFF8 "];\n\t"   \
+    "sub.cc.u32 a0, %0, t0;\n\t"                       \
+    "subc.cc.u32 a1, %1, t1;\n\t"                      \
+    "subc.cc.u32 a2, %2, t2;\n\t"                      \
+    "subc.u32 a3, %3, t3;\n\t"                         \
+    "sub.cc.u32 b0, a0, t0;\n\t"                       \
+    "subc.cc.u32 b1, a1, t1;\n\t"                      \
+    "subc.cc.u32 b2, a2, t2;\n\t"                      \
+    "subc.u32 b3, a3, t3;\n\t"                         \
+    "setp.ge.s32 g1, a3, 0;\n\t"                       \
+    "selp.u32 xh, b3, a3, " #PL ";\n\t"                \
+    "setp.ge.and.s32 " #MO ", xh, 0, g1;\n\t"          \
+    "and.pred ng, g1, " #PL ";\n\t"                    \
+    "and.pred m2, " #MO ", " #PL ";\n\t"               \
+    "@g1 mad.lo.u32 %0, a0, %7, 0;\n\t"                \
+    "@g1 mad.lo.u32 %1, a1, %7, 0;\n\t"                \
+    "@g1 mad.lo.u32 %2, a2, %7, 0;\n\t"                \
+    "@g1 mad.lo.u32 %3, a3, %7, 0;\n\t"                \
+    "@m2 mad.lo.u32 %0, b0, %7, 0;\n\t"                \
+    "@m2 mad.lo.u32 %1, b1, %7, 0;\n\t"                \
+    "@m2 mad.lo.u32 %2, b2, %7, 0;\n\t"                \
+    "@m2 mad.lo.u32 %3, b3, %7, 0;\n\t"                \
+    "mad.lo.u32 val, %4, %7, %12;\n\t"                 \
+    "@ng mad.lo.u32 val, %4, %8, %12;\n\t"             \
+    "st.shared.u%11 [%5], val;\n\t"                    \
+    "@!" #MO " add.u32 %5, %5, %10;\n\t"               \
+    "@!" #MO " add.u32 %6, %6, %9;\n\t"                \
+    "mad.lo.u32 %4, %4, %7, %7;\n\t"                   \
+    "@!" #MO " mov.u32 %4, 0;\n\t"
+template <typename YT>
+__device__ __forceinline__ void walk_block8_4of6(mp<4>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                                const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred g1, m2, ng, pl0, mo0, mo1, mo2, mo3, mo4, mo5, mo6, mo7;\n\t"
+        ".reg .u32 t0, t1, t2, t3, t4, t5, a0, a1, a2, a3, b0, b1, b2, b3, xh, val;\n\t"
+        "setp.gt.s32 pl0, %4, 0;\n\t"
+        PVQ_STEP_4OF6(0, 8, 16, pl0, mo0)
+        PVQ_STEP_4OF6(-24, -16, -8, mo0, mo1)
+        PVQ_STEP_4OF6(-48, -40, -32, mo1, mo2)
+        PVQ_STEP_4OF6(-72, -64, -56, mo2, mo3)
+        PVQ_STEP_4OF6(-96, -88, -80, mo3, mo4)
+        PVQ_STEP_4OF6(-120, -112, -104, mo4, mo5)
+        PVQ_STEP_4OF6(-144, -136, -128, mo5, mo6)
+        PVQ_STEP_4OF6(-168, -160, -152, mo6, mo7)
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(r.w[3]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+#undef PVQ_STEP_4OF6
+
+#define PVQ_STEP_5OF6(OFF, OFF8, OFF16, PL, MO) \
+    "ld.shared.v2.u32 {t0, t1}, [%7+" #OFF "];\n\t"     \
+    "ld.shared.v2.u32 {t2, t3}, [%7+" #OFF8 "];\n\t"    \
+    "ld.shared.v2.u32 {t4, t5}, [%7+" #OFF16 "];\n\t"   \
+    "sub.cc.u32 a0, %0, t0;\n\t"                        \
+    "subc.cc.u32 a1, %1, t1;\n\t"                       \
+    "subc.cc.u32 a2, %2, t2;\n\t"                       \
+    "subc.cc.u32 a3, %3, t3;\n\t"                       \
+    "subc.u32 a4, %4, t4;\n\t"                          \
+    "sub.cc.u32 b0, a0, t0;\n\t"                        \
+    "subc.cc.u32 b1, a1, t1;\n\t"                       \
+    "subc.cc.u32 b2, a2, t2;\n\t"                       \
+    "subc.cc.u32 b3, a3, t3;\n\t"                       \
+    "subc.u32 b4, a4, t4;\n\t"                          \
+    "setp.ge.s32 g1, a4, 0;\n\t"                        \
+    "selp.u32 xh, b4, a4, " #PL ";\n\t"                 \
+    "setp.ge.and.s32 " #MO ", xh, 0, g1;\n\t"           \
+    "and.pred ng, g1, " #PL ";\n\t"                     \
+    "and.pred m2, " #MO ", " #PL ";\n\t"                \
+    "@g1 mad.lo.u32 %0, a0, %8, 0;\n\t"                 \
+    "@g1 mad.lo.u32 %1, a1, %8, 0;\n\t"                 \
+    "@g1 mad.lo.u32 %2, a2, %8, 0;\n\t"                 \
+    "@g1 mad.lo.u32 %3, a3, %8, 0;\n\t"                 \
+    "@g1 mad.lo.u32 %4, a4, %8, 0;\n\t"                 \
+    "@m2 mad.lo.u32 %0, b0, %8, 0;\n\t"                 \
+    "@m2 mad.lo.u32 %1, b1, %8, 0;\n\t"                 \
+    "@m2 mad.lo.u32 %2, b2, %8, 0;\n\t"                 \
+    "@m2 mad.lo.u32 %3, b3, %8, 0;\n\t"                 \
+    "@m2 mad.lo.u32 %4, b4, %8, 0;\n\t"                 \
+    "mad.lo.u32 val, %5, %8, %13;\n\t"                  \
+    "@ng mad.lo.u32 val, %5, %9, %13;\n\t"              \
+    "st.shared.u%12 [%6], val;\n\t"                     \
+    "@!" #MO " add.u32 %6, %6, %11;\n\t"                \
+    "@!" #MO " add.u32 %7, %7, %10;\n\t"                \
+    "mad.lo.u32 %5, %5, %8, %8;\n\t"                    \
+    "@!" #MO " mov.u32 %5, 0;\n\t"
+template <typename YT>
+__device__ __forceinline__ void walk_block8_5of6(mp<5>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                                const Factors f) {
+    constexpr int SZ = static_cast<int>(sizeof(YT));
+    asm volatile(
+        "{\n\t"
+        ".reg .pred g1, m2, ng, pl0, mo0, mo1, mo2, mo3, mo4, mo5, mo6, mo7;\n\t"
+        ".reg .u32 t0, t1, t2, t3, t4, t5, a0, a1, a2, a3, a4, b0, b1, b2, b3, b4, xh, val;\n\t"
+        "setp.gt.s32 pl0, %5, 0;\n\t"
+        PVQ_STEP_5OF6(0, 8, 16, pl0, mo0)
+        PVQ_STEP_5OF6(-24, -16, -8, mo0, mo1)
+        PVQ_STEP_5OF6(-48, -40, -32, mo1, mo2)
+        PVQ_STEP_5OF6(-72, -64, -56, mo2, mo3)
+        PVQ_STEP_5OF6(-96, -88, -80, mo3, mo4)
+        PVQ_STEP_5OF6(-120, -112, -104, mo4, mo5)
+        PVQ_STEP_5OF6(-144, -136, -128, mo5, mo6)
+        PVQ_STEP_5OF6(-168, -160, -152, mo6, mo7)
+        "}"
+        : "+r"(r.w[0]), "+r"(r.w[1]), "+r"(r.w[2]), "+r"(r.w[3]), "+r"(r.w[4]), "+r"(v), "+r"(y), "+r"(p)
+        : "r"(f.one), "r"(f.minus_one), "r"(D), "n"(SZ), "n"(SZ * 8), "n"(kSlotBias<YT>)
+        : "memory");
+}
+#undef PVQ_STEP_5OF6
+
 template <int PW, int EB, bool HEADROOM, typename YT, int U>
 __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32_t& y, const int D,
                                           const Factors f) {
@@ -604,6 +911,34 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
         for (int w = 0; w < 5; ++w) r.w[w] = r6[w];
     } else
         walk_step_wide<PW, EB, YT, U>(r, p, v, y, D);
+}
+
+// Eight steps: one block where the form has one, else eight single steps.
+template <int PW, int EB, bool HEADROOM, typename YT>
+__device__ __forceinline__ void walk_block8(mp<PW>& r, uint32_t& p, int& v, uint32_t& y, const int D,
+                                            const Factors f) {
+    if constexpr (HEADROOM && PW == 1) {
+        walk_block8_1<YT>(r.w[0], p, v, y, D, f);
+    } else if constexpr (HEADROOM && PW == 2 && EB == 8) {
+        walk_block8_2<YT>(r, p, v, y, D, f);
+    } else if constexpr (HEADROOM && PW == 3 && EB == 16) {
+        walk_block8_3of4<YT>(r, p, v, y, D, f);
+    } else if constexpr (HEADROOM && PW == 3 && EB == 24) {
+        walk_block8_3of6<YT>(r, p, v, y, D, f);
+    } else if constexpr (HEADROOM && PW == 4 && EB == 24) {
+        walk_block8_4of6<YT>(r, p, v, y, D, f);
+    } else if constexpr (HEADROOM && PW == 5 && EB == 24) {
+        walk_block8_5of6<YT>(r, p, v, y, D, f);
+    } else {
+        walk_step<PW, EB, HEADROOM, YT, 0>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 1>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 2>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 3>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 4>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 5>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 6>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 7>(r, p, v, y, D, f);
+    }
 }
 
 // Runs steps s .. S-1 on PW-word integers with the table `tab` (entries of EB bytes),
@@ -643,14 +978,7 @@ __device__ __forceinline__ int walk_phase(mp<CW>& rfull, Walk& st, uint32_t tab,
             }
             if (__all_sync(kFull, hi == 0u)) break;
         }
-        walk_step<PW, EB, HEADROOM, YT, 0>(r, p, v, y, D, f);
-        walk_step<PW, EB, HEADROOM, YT, 1>(r, p, v, y, D, f);
-        walk_step<PW, EB, HEADROOM, YT, 2>(r, p, v, y, D, f);
-        walk_step<PW, EB, HEADROOM, YT, 3>(r, p, v, y, D, f);
-        walk_step<PW, EB, HEADROOM, YT, 4>(r, p, v, y, D, f);
-        walk_step<PW, EB, HEADROOM, YT, 5>(r, p, v, y, D, f);
-        walk_step<PW, EB, HEADROOM, YT, 6>(r, p, v, y, D, f);
-        walk_step<PW, EB, HEADROOM, YT, 7>(r, p, v, y, D, f);
+        walk_block8<PW, EB, HEADROOM, YT>(r, p, v, y, D, f);
         p -= 8 * EB;
         s += 8;
     }
