@@ -38,11 +38,11 @@ FALLBACK_HBM_GBS = 6650.0
 # workload and launch configuration as this bench): DRAM bytes read + written, and warp
 # instructions executed.  Set an entry to None when its kernel changes until it is re-captured.
 NCU_COUNTERS = {
-    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_970_176 + 256, "warp_inst": 32_479_472},
-    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_659_328 + 409_088, "warp_inst": 38_781_692},
-    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_489_088 + 89_635_072, "warp_inst": 217_046_280},
-    ("c6_bf16_q_proj_group128", "encode"): {"dram_bytes": 34_220_032 + 16_128, "warp_inst": 89_047_985},
-    ("c6_bf16_q_proj_group128", "decode"): {"dram_bytes": 7_024_896 + 164_608, "warp_inst": 81_724_198},
+    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_969_920 + 1_792, "warp_inst": 32_479_472},
+    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_658_816 + 473_600, "warp_inst": 37_778_508},
+    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_471_936 + 88_764_672, "warp_inst": 214_752_520},
+    ("c6_bf16_q_proj_group128", "encode"): {"dram_bytes": 34_222_592 + 5_632, "warp_inst": 89_047_985},
+    ("c6_bf16_q_proj_group128", "decode"): {"dram_bytes": 7_047_936 + 222_720, "warp_inst": 81_724_198},
 }
 SMS, SCHEDULERS_PER_SM = 148, 4      # issue slots per cycle on the part = SMS * SCHEDULERS_PER_SM
 
