@@ -217,6 +217,27 @@ def test_missing_update_breaks_only_points_with_a_negative_before_the_end():
     assert exposed > 0 and broken > exposed // 2
 
 
+@pytest.mark.parametrize("N,K,W", [(128, 187, 12), (128, 386, 16), (256, 369, 24), (64, 3359, 16), (128, 6378, 32)])
+def test_wide_codes_against_python_integers(N, K, W):
+    """The C oracle's 32-limb integers at the group sizes and bit rates of the paper's grid
+    (Sec. 4.1) against Python's: the enumeration of quantised Gaussian groups, and back."""
+    rng = np.random.default_rng(N + K)
+    total = pr.count_table(N, K)[N][K]
+    assert (total.bit_length() + 31) // 32 <= W and total > 1 << (32 * (W - 1))
+    for _ in range(6):
+        x = rng.standard_normal(N).astype(np.float32)
+        y = po.quantize_group(x, K)
+        assert np.abs(y).sum() == K
+        cw = po.enumerate_point(y, K, W)
+        c = po.code_to_int(cw)
+        assert c == pr.enumerate_point(y.tolist(), K) and 0 <= c < total
+        y2, ok = po.deenumerate_code(cw, N, K)
+        assert ok and np.array_equal(y, y2)
+    for c in (0, total - 1):
+        y, ok = po.deenumerate_code(po.int_to_code(c, W), N, K)
+        assert ok and np.abs(y).sum() == K
+
+
 def test_random_points_round_trip_at_config_sizes():
     rng = np.random.default_rng(7)
     for (N, K, W) in [(32, 22, 2), (32, 50, 3), (64, 96, 6)]:
