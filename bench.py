@@ -98,52 +98,91 @@ def make_workload(name):
 # ------------------------------------------------------------------------ clocks
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """SM clock and throttle reasons of one GPU, polled through NVML from a thread while the
+    bench runs (a few hundred samples per second, each with its host time), so that even a
+    timed region of some milliseconds holds samples of its own.  `nvidia-smi -lms` serves
+    when NVML cannot be loaded."""
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
+               ("sw_power_cap", 0x4))
 
     def __init__(self, index):
-        self.index, self.proc, self.lines = index, None, []
+        self.index, self.samples, self.thread, self.proc = index, [], None, None
+        self.stop_flag = threading.Event()
+        self.sm_max = None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+            import pynvml
+            pynvml.nvmlInit()
+            h = pynvml.nvmlDeviceGetHandleByIndex(self._physical_index())
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+
+            def poll():
+                while not self.stop_flag.is_set():
+                    try:
+                        mhz = pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)
+                        why = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                        self.samples.append((time.perf_counter(), float(mhz), int(why)))
+                    except Exception:
+                        pass
+                    time.sleep(0.002)
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+        except Exception:
+            self._start_smi()
+
+    def _physical_index(self):
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+        if vis:
+            ids = [v for v in vis.split(",") if v.strip() != ""]
+            if self.index < len(ids) and ids[self.index].strip().isdigit():
+                return int(ids[self.index])
+        return self.index
+
+    def _start_smi(self):
+        q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self._physical_index()), "--query-gpu=" + q,
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+
+            def read():
+                for line in self.proc.stdout:
+                    f = [x.strip() for x in line.split(",")]
+                    try:
+                        why = sum(bit for (_, bit), v in zip(self.REASONS, f[2:6]) if v.lower().startswith("active"))
+                        self.samples.append((time.perf_counter(), float(f[0]), why))
+                        self.sm_max = float(f[1])
+                    except (ValueError, IndexError):
+                        pass
+            self.thread = threading.Thread(target=read, daemon=True)
             self.thread.start()
         except Exception:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
-
     def stop(self):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            f = [s.strip() for s in ln.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0]))
-                mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self.stop_flag.set()
+        if self.proc:
+            self.proc.terminate()
+        if self.thread:
+            self.thread.join(timeout=5)
+
+    def summary(self, t0, t1):
+        """Median SM clock and the throttle reasons seen between host times t0 and t1 (the timed
+        region); `samples_under_load` counts everything from warm-up on, whose median is given
+        too, since a short region may hold few samples of its own."""
+        inside = [x for x in self.samples if t0 <= x[0] <= t1]
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "samples": 0, "reasons": ["no clock samples"]}
+        use = inside if inside else self.samples
+        why = 0
+        for x in use:
+            why |= x[2]
+        return {"sm_mhz": statistics.median(x[1] for x in use), "sm_max_mhz": self.sm_max,
+                "samples": len(inside), "samples_under_load": len(self.samples),
+                "sm_mhz_under_load": statistics.median(x[1] for x in self.samples),
+                "reasons": sorted(n for n, bit in self.REASONS if why & bit)}
 
 
 # --------------------------------------------------------------------- GPU runner
@@ -434,12 +473,89 @@ def whole_job_value(step_bytes, steps, world, total_ms):
 
 # --------------------------------------------------------------------------- main
 
+CONFIGS = ["c1", "c2", "c3", "c4", "c5", "c5r", "c6", "c7", "c8", "c9", "c10", "c10r"]
+MODE_DIRS = {"encode+decode": ["encode", "decode"], "decode": ["decode"], "roundtrip": ["roundtrip"],
+             "rotate_roundtrip": ["rotate_roundtrip"]}
+
+
+def kernel_source_sha():
+    """Hash of the CUDA sources: the ncu counters typed in above hold only for the sources they
+    were captured from."""
+    import hashlib
+    d = os.path.join(ROOT, "paper_2410_16926_b200", "csrc")
+    h = hashlib.sha256()
+    for f in sorted(os.listdir(d)):
+        if f.endswith((".cu", ".cuh")):
+            h.update(open(os.path.join(d, f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def config_of(wl, K, W):
+    step_bytes = sum(algorithmic_bytes(wl, d) for d in MODE_DIRS[wl.mode])
+    per_set = algorithmic_bytes(wl, "encode") + algorithmic_bytes(wl, "decode")
+    nsets = max(1, min(16, -(-3 * L2_BYTES // per_set)))
+    return {"workload": wl.name, "matrices": [[m.name, m.rows, m.cols, m.dtype] for m in wl.matrices],
+            "N": wl.N, "index_bits": wl.index_bits, "scale_bits": wl.scale_bits, "mode": wl.mode,
+            "weights": wl.weights, "algorithmic_bytes_per_step": step_bytes, "buffer_sets": nsets,
+            "l2": ("%d buffer set(s), %.0f MB in total, larger than the 126 MB L2" % (nsets, nsets * step_bytes / 1e6)
+                   if nsets * step_bytes > L2_BYTES else
+                   "%d buffer sets, %.1f MB: fits the L2 (launch-bound workload)" % (nsets, nsets * step_bytes / 1e6)),
+            "K": K, "W": W}
+
+
+def kernel_table(wl, per, peak, peak_kind):
+    kernels = {}
+    for name, ms_list in per.items():
+        avg = sum(ms_list) / len(ms_list)
+        nbytes = algorithmic_bytes(wl, name)
+        kernels[name] = {"avg_ms": avg, "median_ms": sorted(ms_list)[len(ms_list) // 2], "min_ms": min(ms_list),
+                         "algorithmic_bytes": nbytes,
+                         "GBps": nbytes / (avg * 1e-3) / 1e9, "Gweights_per_s": wl.weights / (avg * 1e-3) / 1e9,
+                         "frac_of_%s_hbm" % peak_kind: nbytes / (avg * 1e-3) / 1e9 / peak,
+                         "frac_of_nominal_8TBps": nbytes / (avg * 1e-3) / 1e9 / 8000.0}
+    return kernels
+
+
+def timed_run(run, steps, warmup, sampler, barrier, min_warm_seconds=0.3):
+    """W warm-up steps (repeated until the GPU has been busy for min_warm_seconds, so that its
+    clocks have settled and the sampler has something to show), then exactly `steps` steps
+    between two barriers.  Returns (total_ms, per-kernel ms lists, clock summary)."""
+    import torch
+    t_w = time.perf_counter()
+    run.run(1, warmup)
+    while time.perf_counter() - t_w < min_warm_seconds:
+        run.run(1, warmup)
+    barrier()
+    t0 = time.perf_counter()
+    total_ms, per = run.run(steps, 0)
+    barrier()
+    t1 = time.perf_counter()
+    return total_ms, per, sampler.summary(t0, t1)
+
+
+def spawn_ranks(n, argv):
+    """`bench.py --gpus N` started without a launcher: start the N ranks, one per GPU."""
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + argv
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5000)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--config", default="c2", choices=["c1", "c2", "c3", "c4", "c5", "c5r", "c6", "c7", "c8", "c9", "c10", "c10r"])
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="c3", choices=CONFIGS,
+                    help="the workload of the JSON line; c3 (the full decoder layer) is the largest that "
+                         "runs both directions")
+    ap.add_argument("--others", default=None,
+                    help="comma list of further workloads timed briefly and reported under `other_workloads` "
+                         "(default: c2,c4,c5 beside c3 on one GPU; `none` to skip)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--graph", action="store_true",
@@ -447,22 +563,22 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     warmup = max(args.warmup, 3)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
 
     wl = make_workload(args.config)
     metric = "pvq_%s_throughput" % wl.mode.replace("+", "_")
-    dirs = {"encode+decode": ["encode", "decode"], "decode": ["decode"], "roundtrip": ["roundtrip"],
-            "rotate_roundtrip": ["rotate_roundtrip"]}[wl.mode]
-    step_bytes = sum(algorithmic_bytes(wl, d) for d in dirs)
-    config = {"workload": wl.name, "matrices": [[m.name, m.rows, m.cols, m.dtype] for m in wl.matrices],
-              "N": wl.N, "index_bits": wl.index_bits, "scale_bits": wl.scale_bits, "mode": wl.mode,
-              "weights": wl.weights, "algorithmic_bytes_per_step": step_bytes}
+    step_bytes = sum(algorithmic_bytes(wl, d) for d in MODE_DIRS[wl.mode])
 
     if args.impl == "reference":
         if rank != 0:
             return
+        from oracle import pvq_oracle as po
+        K = po.max_pulses(wl.N, wl.index_bits)
+        config = config_of(wl, K, po.words_for_bits(wl.index_bits))
         gbs, threads, sample, nb, t, gbs1 = oracle_sample(wl, target_seconds=max(2.0, min(20.0, 0.05 * args.steps)))
         line = {"impl": "reference", "metric": metric, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
                 "steps": args.steps, "warmup": warmup, "ms_per_step": step_bytes / (gbs * 1e9) * 1e3,
@@ -483,23 +599,19 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
 
-    run = DeviceRun(wl, device)
-    config["buffer_sets"] = run.nsets
-    config["l2"] = "rotating %d buffer sets, %.0f MB in total, larger than the 126 MB L2" % (
-        run.nsets, run.nsets * step_bytes / 1e6)
-    config["K"], config["W"] = run.K, run.W
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
     sampler = ClockSampler(local_rank)
-    barrier()
     sampler.start()
-    total_ms, per = run.run(args.steps, warmup)
+    run = DeviceRun(wl, device)
+    config = config_of(wl, run.K, run.W)
+    assert config["buffer_sets"] == run.nsets
+
     barrier()
-    clocks = sampler.stop()
+    total_ms, per, clocks = timed_run(run, args.steps, warmup, sampler, barrier)
     total_ms = max_over_ranks(total_ms, world, device)
     value = whole_job_value(step_bytes, args.steps, world, total_ms)
 
@@ -513,39 +625,63 @@ def main():
         e2e = {"value": whole_job_value(step_bytes, 1, world, ms), "unit": "GB/s", "ms_per_step": ms,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
+    peak, peak_kind = measured_peak()
+    sha = kernel_source_sha()
+
+    # the other workloads of the metric, each timed briefly on its own (one GPU only)
+    others = args.others if args.others is not None else ("c2,c4,c5" if args.config == "c3" and world == 1 else "none")
+    other_lines = {}
+    if others != "none":
+        del run
+        torch.cuda.empty_cache()
+        for name in [o for o in others.split(",") if o and o != args.config]:
+            wl2 = make_workload(name)
+            run2 = DeviceRun(wl2, device)
+            o_steps = max(10, min(args.steps, 50))
+            ms2, per2, clk2 = timed_run(run2, o_steps, warmup, sampler, barrier)
+            sb2 = sum(algorithmic_bytes(wl2, d) for d in MODE_DIRS[wl2.mode])
+            other_lines[wl2.name] = {"steps": o_steps, "ms_per_step": ms2 / o_steps,
+                                     "value": sb2 * o_steps / (ms2 * 1e-3) / 1e9, "unit": "GB/s",
+                                     "config": config_of(wl2, run2.K, run2.W),
+                                     "kernels": kernel_table(wl2, per2, peak, peak_kind), "clocks": clk2}
+            del run2
+            torch.cuda.empty_cache()
+    sampler.stop()
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = measured_peak()
-    kernels = {}
-    for name, ms_list in per.items():
-        avg = sum(ms_list) / len(ms_list)
-        nbytes = algorithmic_bytes(wl, name)
-        kernels[name] = {"avg_ms": avg, "median_ms": sorted(ms_list)[len(ms_list) // 2], "min_ms": min(ms_list),
-                         "algorithmic_bytes": nbytes,
-                         "GBps": nbytes / (avg * 1e-3) / 1e9, "Gweights_per_s": wl.weights / (avg * 1e-3) / 1e9,
-                         "frac_of_%s_hbm" % peak_kind: nbytes / (avg * 1e-3) / 1e9 / peak,
-                         "frac_of_nominal_8TBps": nbytes / (avg * 1e-3) / 1e9 / 8000.0}
+    kernels = kernel_table(wl, per, peak, peak_kind)
     dom = max(kernels, key=lambda k: kernels[k]["avg_ms"])
     ncu = NCU_COUNTERS.get((wl.name, dom))
+    if ncu and ncu.get("kernel_sha") != sha:
+        ncu = None                      # the kernels have changed since the counters were taken
     roofline = {"kernel": "pvq %s_kernel" % dom, "bound": "hbm", "achieved": kernels[dom]["GBps"], "peak": peak,
                 "peak_source": "%s (MEASURED_PEAKS.json hbm_gbs)" % peak_kind if peak_kind == "measured"
                 else "fallback", "unit": "GB/s", "frac": kernels[dom]["GBps"] / peak,
-                "traffic": ncu["dram_bytes"] if ncu else None}
+                "traffic": ncu["dram_bytes"] if ncu else None,
+                "traffic_source": "ncu capture summarised under profiles/ (not this run)" if ncu else None}
     # The limit that binds in practice: instruction issue (every kernel here is integer work
-    # on a table walk).  achieved = ncu's warp instructions per launch / measured time,
+    # on a table walk).  achieved = warp instructions per launch (from the ncu capture under
+    # profiles/, valid while the sources are unchanged) / the time measured in this run;
     # peak = issue slots per second at the SM clock sampled during the run.
     issue = {}
+    mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz")
     for name in kernels:
         c = NCU_COUNTERS.get((wl.name, name))
-        mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz")
-        if c and mhz:
+        pk = SMS * SCHEDULERS_PER_SM * mhz * 1e6 if mhz else None
+        entry = {"bound": "alu", "peak": pk / 1e9 if pk else None, "unit": "Gwarp-inst/s",
+                 "peak_source": "148 SMs x 4 schedulers x sampled SM clock"}
+        if c and c.get("kernel_sha") == sha and pk:
             ach = c["warp_inst"] / (kernels[name]["avg_ms"] * 1e-3)
-            pk = SMS * SCHEDULERS_PER_SM * mhz * 1e6
-            issue[name] = {"bound": "alu", "achieved": ach / 1e9, "peak": pk / 1e9, "unit": "Gwarp-inst/s",
-                           "frac": ach / pk, "warp_inst_per_weight": c["warp_inst"] / wl.weights}
+            entry.update({"achieved": ach / 1e9, "frac": ach / pk, "warp_inst_per_weight": c["warp_inst"] / wl.weights,
+                          "warp_inst_source": "ncu capture summarised under profiles/ (not this run)"})
+        else:
+            entry.update({"achieved": None, "frac": None, "warp_inst_per_weight": None,
+                          "warp_inst_source": "no capture of the current sources"})
+        issue[name] = entry
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -558,7 +694,9 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "u32+f32", "data": "synthetic",
             "config": config, "Gweights_per_s": wl.weights * args.steps * world / (total_ms * 1e-3) / 1e9,
             "kernels": kernels, "roofline": roofline, "issue": issue, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
-            "gpu_launches": len(per) * args.steps}
+            "gpu_launches": len(per) * args.steps, "kernel_source_sha": sha}
+    if other_lines:
+        line["other_workloads"] = other_lines
     if graph_ms is not None:
         line["graph_replay"] = {"ms_per_step": graph_ms, "GBps": step_bytes / (graph_ms * 1e-3) / 1e9}
     print(json.dumps(line))

@@ -22,7 +22,10 @@
  *     that point.  The device current at the call must own all pointers.
  *   - Every function returns a pvq_status; nothing is thrown across the ABI and
  *     no argument error reaches a kernel.
- *   - Inputs must be finite.  NaN or Inf gives unspecified codes but never an
+ *   - Inputs must be finite, and so must the fp32 sums taken over them: the l1 norm and
+ *     the energy of every group, the energy of every row, and K divided by a group's l1
+ *     norm.  NaN or Inf in the input, or a sum that overflows fp32, gives unspecified
+ *     codes (the group is then usually treated as having no direction) but never an
  *     out-of-bounds access.
  *
  * Storage formats (also the persistent format of an encoded matrix)
@@ -239,21 +242,25 @@ int pvq_decode_batched(const pvq_matrix_desc* descs, int count, int N, int K, in
  * an engine that has already planned all of its memory, a control loop whose allocator is
  * frozen, a process whose memory budget is enforced by refusing cudaMalloc - the table
  * N(n,k) is kept in a fixed array inside the library (PVQ_STATIC_TABLE_BYTES per GPU that
- * loads the library, held until the process exits).  This call allocates and frees
- * nothing, on the device or through any allocating library routine; codes, amplitude
- * indices, row norms, levels and the output are still the caller's buffers, with the
- * meaning and alignment they have in pvq_decode.
+ * loads the library, held until the process exits).  This call allocates and frees no
+ * device memory; codes, amplitude indices, row norms, levels and the output are still the
+ * caller's buffers, with the meaning and alignment they have in pvq_decode.  The first
+ * call for an (N,K) in a process also fills small host-side caches (the code width, the
+ * kernel's launch geometry), so make it during set-up.
  *
  *   - (N,K) whose table needs more than PVQ_STATIC_TABLE_BYTES (pvq_count_table_bytes
  *     tells) is refused with PVQ_ERR_TABLE_TOO_SMALL.
- *   - The first call on a device looks up the array's device address and fills the table
- *     on `stream`; so does any later call whose (N,K) differs from the previous call's on
- *     that device.  Make that first call before any stream capture begins.
+ *   - The first call on a device looks up the array's device address, creates one event
+ *     and fills the table on `stream`; so does (the fill) any later call whose (N,K)
+ *     differs from the previous call's on that device.  Make that first call before any
+ *     stream capture begins.
  *   - All calls on a device share the one array, which keeps what the last call put
  *     there.  Nothing in it has to start at zero (the fill overwrites every word decode
- *     reads).  Two calls with different (N,K) whose work overlaps on the GPU - different
- *     streams, no dependency between them - race on the array; calls with the same (N,K)
- *     only read it and may overlap freely once the first has been enqueued. */
+ *     reads).  A call with the same (N,K) as the previous one only reads the array; if
+ *     the fill is still in flight on another stream, the call first makes its stream wait
+ *     for it, so such calls may overlap freely.  Two calls with different (N,K) whose
+ *     work overlaps on the GPU - different streams, no dependency between them - race on
+ *     the array: the second call's fill overwrites what the first call's decode reads. */
 int pvq_decode_static_table(const uint32_t* d_codes, const uint8_t* d_scale_idx, const float* d_row_norm,
                             int64_t rows, int64_t cols, int N, int K, int scale_bits,
                             const float* d_levels, void* d_out, int64_t ld_out, uint32_t* d_status,

@@ -190,7 +190,9 @@ int pvqo_index_bits(int N, int K) {
 }
 
 /* Sec. 3.3 Step 2: the largest K with N(N,K) <= 2^index_bits, tested on the
- * integers themselves.  0 when not even K = 1 fits; -1 on bad arguments. */
+ * integers themselves.  0 when not even K = 1 fits; -1 on bad arguments.
+ * The search stops at 8191 pulses (N(1,K) = 2 for every K would never end it,
+ * and no caller stores more: a coordinate is kept in 16 bits). */
 int pvqo_max_pulses(int N, int index_bits) {
     if (N < 1 || index_bits < 1 || index_bits > 32 * (PVQO_MAXW - 1)) return -1;
     int K = 0;
@@ -198,7 +200,7 @@ int pvqo_max_pulses(int N, int index_bits) {
         int b = pvqo_index_bits(N, K + 1);
         if (b < 0 || b > index_bits) break;
         ++K;
-        if (K > 4096) break;
+        if (K >= 8191) break;
     }
     return K;
 }

@@ -27,8 +27,9 @@ static __device__ __align__(256) uint32_t g_static_table[kStaticTableBytes / siz
 namespace {
 
 struct DeviceSlot {
-    uint32_t* ptr = nullptr;  // device address of g_static_table on this device
-    int N = 0, K = 0;         // the table it was last filled for (0: never)
+    uint32_t* ptr = nullptr;      // device address of g_static_table on this device
+    cudaEvent_t filled = nullptr; // recorded behind the last fill, on the stream that ran it
+    int N = 0, K = 0;             // the table it was last filled for (0: never)
 };
 
 std::mutex g_mu;
@@ -59,16 +60,29 @@ extern "C" int pvq_decode_static_table(const uint32_t* d_codes, const uint8_t* d
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_static_table);
         if (e != cudaSuccess) return set_cuda_error(e);
+        cudaEvent_t ev = nullptr;
+        e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e != cudaSuccess) return set_cuda_error(e);
         slot.ptr = static_cast<uint32_t*>(p);
+        slot.filled = ev;
     }
+    const cudaStream_t cs = static_cast<cudaStream_t>(stream);
     if (slot.N != N || slot.K != K) {
         // Every word the decode kernel reads for (N,K) is written by the builder, so the
         // array needs no clearing between different (N,K).
         slot.N = slot.K = 0;
         const int st = pvq_build_count_table(N, K, slot.ptr, kStaticTableBytes, stream);
         if (st != PVQ_OK) return st;
+        e = cudaEventRecord(slot.filled, cs);
+        if (e != cudaSuccess) return set_cuda_error(e);
         slot.N = N;
         slot.K = K;
+    } else if (cudaEventQuery(slot.filled) != cudaSuccess) {
+        // Same (N,K), but the fill may still be in flight on another stream: order this call's
+        // decode behind it.  Once the fill has completed no wait is enqueued any more.
+        (void)cudaGetLastError();  // cudaErrorNotReady from the query is not an error
+        e = cudaStreamWaitEvent(cs, slot.filled, 0);
+        if (e != cudaSuccess) return set_cuda_error(e);
     }
     return pvq_decode(d_codes, d_scale_idx, d_row_norm, rows, cols, N, K, scale_bits, slot.ptr, d_levels,
                       d_out, ld_out, d_status, stream);

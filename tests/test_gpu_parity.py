@@ -288,6 +288,50 @@ def test_invalid_codes_set_status_and_decode_to_zero(N, bits):
     assert torch.any(out[2, N:2 * N] != 0)
 
 
+def _random_codes(rng, total, shape, W):
+    """Codes drawn uniformly from [0, total) with Python integers, as (..., W) uint32 words."""
+    n = int(np.prod(shape))
+    nbytes = (total.bit_length() + 7) // 8 + 8              # 64 spare bits: the modulo bias is below 2^-64
+    raw = rng.integers(0, 256, size=(n, nbytes), dtype=np.uint8)
+    out = np.empty((n, W), dtype=np.uint32)
+    for j in range(n):
+        out[j] = po.int_to_code(int.from_bytes(raw[j].tobytes(), "little") % total, W)
+    return out.reshape(*shape, W)
+
+
+@pytest.mark.parametrize("N,K", [(32, 22), (32, 50), (64, 96), (128, 187), (64, 199), (16, 27), (8, 40)])
+def test_decode_of_codes_the_encoder_did_not_make(N, K):
+    # Algorithm 3 on codes that come from no encoder: uniform over [0, N(N,K)), where the
+    # remainder shrinks at a different pace than on encoded Gaussian data, and batches built so
+    # that one thread of a warp keeps a wide remainder while the other 31 go narrow at once
+    # (and the reverse), which is what decides when a warp may switch to narrower arithmetic.
+    rows, G, b = 6, 64, 8
+    cd = Codec(N, 0, G, b, K=K)
+    W = cd.W
+    total = po.code_to_int(po.count_table(N, K, W + 1)[N, K])
+    rng = np.random.default_rng(1000 * N + K)
+    codes = _random_codes(rng, total, (rows, G), W)
+    big = po.int_to_code(total - 1, W)
+    small = _random_codes(rng, min(total, 1 << 20), (rows, G), W)
+    flat = codes.reshape(-1, W)
+    sflat = small.reshape(-1, W)
+    n = flat.shape[0]
+    third = n // 3 // 32 * 32
+    # second third: lane 0 of every warp holds N(N,K) - 1, the rest hold small codes
+    flat[third:2 * third] = sflat[third:2 * third]
+    flat[third:2 * third:32] = big
+    # last third: lane 0 holds a small code, the rest hold large random ones (as drawn)
+    flat[2 * third::32] = sflat[2 * third::32]
+    flat[-1] = big
+    flat[0] = 0
+    sidx = rng.integers(0, 256, size=(rows, int(pvq.scale_row_stride(G, b))), dtype=np.uint8)
+    rnorm = (rng.random(rows).astype(np.float32) + 0.5)
+    enc_np = (codes, sidx, rnorm)
+    enc_dev = (torch.from_numpy(codes.view(np.int32)).to(DEV), torch.from_numpy(sidx).to(DEV),
+               torch.from_numpy(rnorm).to(DEV))
+    check_decode(cd, enc_dev, enc_np)
+
+
 def test_fused_roundtrip_equals_encode_then_decode():
     for (N, bits, rows, cols, b, kind) in [(32, 64, 40, 4096, 8, "bf16"), (16, 40, 9, 208, 4, "f32"),
                                            (64, 192, 5, 3584, 6, "bf16")]:

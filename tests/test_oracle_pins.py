@@ -131,6 +131,14 @@ def test_max_pulses_is_largest_that_fits(N, bits):
     assert po.index_bits(N, K) == (binomial_count(N, K) - 1).bit_length() <= bits
 
 
+def test_max_pulses_beyond_4096():
+    # Step 2 with closed forms for tiny N: N(2,K) = 4K and N(3,K) = 4K^2 + 2, so the largest K
+    # with N(3,K) <= 2^27 is floor(sqrt((2^27 - 2) / 4)) = 5792, and N(2,K) <= 2^14 gives 4096.
+    assert po.max_pulses(3, 27) == math.isqrt(((1 << 27) - 2) // 4) == 5792
+    assert po.max_pulses(2, 14) == 4096
+    assert binomial_count(3, 5792) == 4 * 5792 ** 2 + 2 <= 1 << 27 < binomial_count(3, 5793)
+
+
 def test_bits_per_weight_examples():
     # Sec. 4.1: group size 16 with a 40-bit direction code is 2.5 bits per weight; the
     # tables' 3.125 = 3 + 16/128, 3.25 = 3 + 4/16, 3.5 = 2.5 + 16/16, 3.88 ~ 3.5 + 6/16
@@ -378,6 +386,29 @@ def test_edges_are_the_quantiles(N, G, b):
         cdf = mpmath.betainc(a, bb, 0, mpmath.mpf(float(e[j - 1])), regularized=True)
         assert abs(float(cdf) - j / L) < 1e-9
     assert np.all(np.diff(bc.edges_f32(N, G, b)) > 0)
+
+
+@pytest.mark.parametrize("N,G,b", [(32, 16, 8), (32, 128, 4), (32, 448, 8), (64, 448, 6)])
+def test_levels_are_the_probability_midpoints(N, G, b):
+    # Sec. 3.4: dequantize(q) = PPF((q + 1/2) / 2^b), i.e. CDF(level_q) = (q + 1/2) / 2^b with
+    # mpmath's regularised incomplete beta.  A midpoint of the two edges in the u domain, or
+    # PPF(q / 2^b), lands in the same bin but misses this value by far more than the bound.
+    lev = bc.levels_f64(N, G, b)
+    mpmath.mp.dps = 40
+    a, bb = bc.beta_params(N, G)
+    L = 1 << b
+    for q in (0, L // 4, L // 2, L - 1):
+        cdf = mpmath.betainc(a, bb, 0, mpmath.mpf(float(lev[q])), regularized=True)
+        assert abs(float(cdf) - (q + 0.5) / L) < 1e-9
+    # the plausible mistakes, shown to fail the same check
+    e = np.concatenate(([0.0], bc.edges_f64(N, G, b), [1.0]))
+    for q in (L // 4, L // 2):
+        for wrong in (0.5 * (e[q] + e[q + 1]), e[q]):
+            cdf = mpmath.betainc(a, bb, 0, mpmath.mpf(float(wrong)), regularized=True)
+            assert abs(float(cdf) - (q + 0.5) / L) > 1e-7  # a hundred times the bound above
+    # the amplitude table is the square root of it, rounded once
+    amp = bc.levels_amp_f32(N, G, b)
+    assert np.array_equal(amp, np.sqrt(lev).astype(np.float32))
 
 
 def test_uniform_and_power_special_cases():

@@ -12,6 +12,7 @@ import pytest
 import torch
 
 from oracle import beta_codebook as bc
+from oracle import pvq_oracle as po
 from paper_2410_16926_b200 import pvq
 
 pytestmark = pytest.mark.gpu
@@ -31,6 +32,14 @@ def _encoded(N, bits, rows, cols, b, seed):
     return K, table, levels, enc
 
 
+def _oracle_bits(enc, N, K, b, G):
+    """Algorithm 3 + Sec. 3.4 by the CPU oracle on the same codes: bf16 bit patterns."""
+    codes, sidx, rnorm = (t.cpu().numpy() for t in enc)
+    out, status = po.decode(codes.view(np.uint32), sidx, rnorm, N, K, b, bc.levels_amp_f32(N, G, b))
+    assert status == 0
+    return torch.from_numpy(out.view(np.int16)).to(DEV)
+
+
 def _same_bits(a, b):
     return torch.equal(a.view(torch.int16), b.view(torch.int16))
 
@@ -47,6 +56,7 @@ def test_static_table_decode_equals_decode_on_consecutive_calls():
     torch.cuda.synchronize()
     assert int(st.item()) == 0
     assert _same_bits(out1, ref) and _same_bits(out2, ref)
+    assert torch.equal(out1.view(torch.int16), _oracle_bits(enc, 32, K, 4, 4096 // 32))
 
     # a different (N, K) refills the shared array; going back refills it again
     K2, table2, levels2, enc2 = _encoded(32, 64, 19, 512, 8, seed=12)
@@ -55,6 +65,42 @@ def test_static_table_decode_equals_decode_on_consecutive_calls():
     out4 = pvq.decode_static_table(*enc, 32, K, 4, levels, out=torch.empty_like(ref))
     torch.cuda.synchronize()
     assert _same_bits(out3, ref2) and _same_bits(out4, ref)
+    assert torch.equal(out3.view(torch.int16), _oracle_bits(enc2, 32, K2, 8, 512 // 32))
+
+
+def test_static_table_same_parameters_on_two_streams():
+    # The first call fills the shared array on its own stream; a second call with the same
+    # (N, K) on another stream, with no dependency of the caller's making, must still read the
+    # finished table: the library orders it behind the fill.
+    K, table, levels, enc = _encoded(32, 96, 23, 2048, 4, seed=21)
+    K0, _, levels0, enc0 = _encoded(16, 40, 5, 256, 4, seed=22)
+    ref = pvq.decode(*enc, 32, K, 4, table, levels)
+    pvq.decode_static_table(*enc0, 16, K0, 4, levels0)      # leave another (N, K) in the array
+    torch.cuda.synchronize()
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    out1, out2 = torch.empty_like(ref), torch.empty_like(ref)
+    with torch.cuda.stream(s1):
+        pvq.decode_static_table(*enc, 32, K, 4, levels, out=out1)
+    with torch.cuda.stream(s2):
+        pvq.decode_static_table(*enc, 32, K, 4, levels, out=out2)
+    torch.cuda.synchronize()
+    assert _same_bits(out1, ref) and _same_bits(out2, ref)
+
+
+def test_static_table_calls_leave_device_memory_alone():
+    # once set-up is over (first call made, output preallocated) repeated calls neither take
+    # nor give back device memory: the driver's free-byte count and torch's allocator agree
+    K, table, levels, enc = _encoded(32, 96, 8, 1024, 4, seed=31)
+    out = torch.empty((8, 1024), dtype=torch.bfloat16, device=DEV)
+    pvq.decode_static_table(*enc, 32, K, 4, levels, out=out)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    alloc0 = torch.cuda.memory_allocated()
+    for _ in range(5):
+        pvq.decode_static_table(*enc, 32, K, 4, levels, out=out)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and torch.cuda.memory_allocated() == alloc0
 
 
 def test_static_table_rejects_what_does_not_fit():
