@@ -1,8 +1,8 @@
 // Encode kernels for group size 64, 5-word codes.
-#include "pvq_encode_impl.cuh"
+#include "pvq_encode_fast.cuh"
 
 namespace pvq {
 int launch_encode_n64_w5(BatchArgs& a, int dtype, bool fused, cudaStream_t s) {
-    return launch_encode_nw<64, 5>(a, dtype, fused, s);
+    return launch_encode_any<64, 5>(a, dtype, fused, s);
 }
 }  // namespace pvq

@@ -1,8 +1,8 @@
 // Encode kernels for group size 8, 2-word codes.
-#include "pvq_encode_impl.cuh"
+#include "pvq_encode_fast.cuh"
 
 namespace pvq {
 int launch_encode_n8_w2(BatchArgs& a, int dtype, bool fused, cudaStream_t s) {
-    return launch_encode_nw<8, 2>(a, dtype, fused, s);
+    return launch_encode_any<8, 2>(a, dtype, fused, s);
 }
 }  // namespace pvq

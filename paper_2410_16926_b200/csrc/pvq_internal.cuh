@@ -29,6 +29,7 @@ struct MatrixArgs {
     int G;                // groups per row
     int sstride;          // bytes per row of scale_idx
     int rows_per_tile;    // encode: rows one thread block covers
+    int chunks;           // encode: pieces a row longer than the block is taken in (else 1)
     unsigned tile_begin;  // first tile of this matrix in the launch
 };
 
@@ -76,6 +77,24 @@ struct BatchArgs {
 //                 enc[0]  U(n,col) = V(n,col) + V(n,col-1)
 //                 enc[1]  2 V(n,col)
 //                 enc[2]  V(n,col)
+//
+// For the kernels that keep their tables in shared memory (N <= 64, W <= 6) three more
+// sections follow:
+//
+//   walkd       the walk table as doubles (8 bytes an entry, same rows and row length as
+//               walk[0]), values from 2^53 up replaced by 2^53: the last stretch of the walk,
+//               once every remainder is below 2^53, runs in fp64
+//   start       U(N-1, K) as `top_words` words (16 bytes reserved): where the encoder's sum starts
+//   cenc[0..1]  the encoder's tables in telescoped form (present for codes of up to 4 words and
+//               up to 127 pulses when both fit 160 KB), rows by position i, `crow` entries of
+//               `top_words` words for k = 0..K (zeros beyond K), crow = 32, 64 or 128, the
+//               first that holds K+1; cenc[1] follows cenc[0] directly.  Modulo 2^(32 W):
+//                 cenc[0]  U(n-1,k) - U(n,k)      for y_i <= 0
+//                 cenc[1]  U(n-1,k) - 2 V(n,k)    for y_i > 0
+//               with n = N-1-i and U(-1, .) = 0.  The contribution of position i to the code,
+//               U(n,k_i) - U(n,k_{i+1}) or U(n,k_i) - 2 V(n,k_{i+1}) (k_i pulses before it,
+//               k_{i+1} after it), then costs one table read: the U(n,k_i) of position i is
+//               carried by the entry of position i-1, that of position 0 is `start`.
 // words per entry of the widest tables for W-word codes
 __host__ __device__ constexpr int top_words_of(int W) {
     return W <= 2 ? W : (W <= 4 ? 4 : (W <= 6 ? 6 : (W <= 8 ? 8 : (W <= 12 ? 12 : ((W + 3) & ~3)))));
@@ -92,8 +111,15 @@ struct TableLayout {
     uint32_t walk_bytes[3];
     uint32_t enc_off[3];
     uint32_t enc_bytes;  // of each of the three
+    uint32_t walkd_off, walkd_bytes;  // 0 bytes: absent
+    uint32_t start_off;
+    uint32_t cenc_off[2];
+    uint32_t cenc_bytes;  // of each of the two; 0: absent
+    int crow;             // entries per row of cenc
     uint32_t total;
 };
+
+constexpr uint32_t kCencLimit = 160u * 1024u;  // both telescoped encoder tables have to fit this
 
 __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
     TableLayout L;
@@ -103,6 +129,8 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
         L.bound_off = 0;
         for (int p = 0; p < 3; ++p) L.walk_off[p] = L.walk_bytes[p] = L.enc_off[p] = 0;
         L.enc_bytes = 0;
+        L.walkd_off = L.walkd_bytes = L.start_off = L.cenc_off[0] = L.cenc_off[1] = L.cenc_bytes = 0;
+        L.crow = 0;
         L.total = static_cast<uint32_t>(N) * (K + 1) * W * 4u;
         return L;
     }
@@ -123,6 +151,25 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
     for (int p = 0; p < 3; ++p) {
         L.enc_off[p] = off;
         off += (L.enc_bytes + 127u) & ~127u;
+    }
+    L.walkd_off = L.walkd_bytes = L.start_off = L.cenc_off[0] = L.cenc_off[1] = L.cenc_bytes = 0;
+    L.crow = 0;
+    if (N <= 64 && W <= 6) {
+        L.walkd_off = off;
+        L.walkd_bytes = entries * 8u;
+        off += (L.walkd_bytes + 127u) & ~127u;
+        L.start_off = off;
+        off += 128u;
+        const int crow = K + 1 <= 32 ? 32 : (K + 1 <= 64 ? 64 : 128);
+        const uint32_t cb = static_cast<uint32_t>(N) * crow * L.top_words * 4u;
+        if (W <= 4 && K + 1 <= 128 && 2u * cb <= kCencLimit) {
+            L.crow = crow;
+            L.cenc_bytes = cb;
+            for (int p = 0; p < 2; ++p) {
+                L.cenc_off[p] = off;
+                off += cb;  // a multiple of 128
+            }
+        }
     }
     L.total = off;
     return L;

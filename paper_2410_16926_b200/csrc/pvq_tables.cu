@@ -224,6 +224,56 @@ __global__ void derive_tables_kernel(int N, int K, int Wc, uint32_t* __restrict_
     }
 }
 
+// The sections for the shared-memory kernels (see TableLayout): the walk table as doubles,
+// and the encoder's telescoped tables with the value the sum starts from.  Runs after
+// derive_tables_kernel: it reads the walk table and the cumulative tables U and 2V.
+__global__ void derive_fast_tables_kernel(int N, int K, int Wc, uint32_t* __restrict__ blob) {
+    const TableLayout L = table_layout(N, K, Wc);
+    if (L.walkd_bytes == 0) return;
+    const int TW = L.top_words;
+    const int entries = N * L.rowlen;
+    const int tid = blockIdx.x * blockDim.x + threadIdx.x, nthr = gridDim.x * blockDim.x;
+    double* wd = reinterpret_cast<double*>(blob + L.walkd_off / 4);
+    for (int e = tid; e < entries; e += nthr) {
+        const uint32_t* t = blob + L.walk_off[0] / 4 + static_cast<size_t>(e) * TW;
+        uint32_t hi = 0;
+        for (int w = 2; w < TW; ++w) hi |= t[w];
+        const uint32_t t1 = TW > 1 ? t[1] : 0u;
+        const bool big = hi != 0u || (t1 >> 21) != 0u;  // 2^53 and up (the row padding too)
+        const unsigned long long v = static_cast<unsigned long long>(t[0]) | (static_cast<unsigned long long>(t1) << 32);
+        wd[e] = big ? 9007199254740992.0 : static_cast<double>(v);  // exact: below 2^53
+    }
+    const uint32_t* U = blob + L.enc_off[0] / 4;  // (i, col + 1), K + 2 entries a row
+    const uint32_t* V2 = blob + L.enc_off[1] / 4;
+    if (tid < TW) blob[L.start_off / 4 + tid] = U[static_cast<size_t>(K + 1) * TW + tid];  // U(N-1, K): position 0
+    if (L.cenc_bytes == 0) return;
+    const int centries = N * L.crow;
+    for (int e = tid; e < centries; e += nthr) {
+        const int i = e / L.crow;
+        const int k = e - i * L.crow;
+        uint32_t* c0 = blob + L.cenc_off[0] / 4 + static_cast<size_t>(e) * TW;
+        uint32_t* c1 = blob + L.cenc_off[1] / 4 + static_cast<size_t>(e) * TW;
+        if (k > K) {  // the rest of the row
+            for (int w = 0; w < TW; ++w) c0[w] = c1[w] = 0u;
+            continue;
+        }
+        const uint32_t* un = U + (static_cast<size_t>(i + 1) * (K + 2) + k + 1) * TW;  // U(n-1, k): next position
+        const uint32_t* u = U + (static_cast<size_t>(i) * (K + 2) + k + 1) * TW;
+        const uint32_t* v2 = V2 + (static_cast<size_t>(i) * (K + 2) + k + 1) * TW;
+        long long b0 = 0, b1 = 0;  // borrows
+        for (int w = 0; w < TW; ++w) {
+            const long long a = (i + 1 < N && w < Wc) ? static_cast<long long>(un[w]) : 0;
+            const long long d0 = a - static_cast<long long>(u[w]) + b0;
+            const long long d1 = a - static_cast<long long>(v2[w]) + b1;
+            b0 = d0 >> 32;  // 0 or -1
+            b1 = d1 >> 32;
+            const bool in = w < Wc;  // modulo 2^(32 Wc): the words above stay zero
+            c0[w] = in ? static_cast<uint32_t>(d0) : 0u;
+            c1[w] = in ? static_cast<uint32_t>(d1) : 0u;
+        }
+    }
+}
+
 template <int W>
 static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStream_t s) {
     const int threads = ((K + 1 + 31) / 32) * 32;
@@ -242,6 +292,8 @@ static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStrea
     if (e != cudaSuccess) return set_cuda_error(e);
     if (table_layout(N, K, Wc).rowlen != 0) {
         derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table);
+        if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
+        derive_fast_tables_kernel<<<16, 256, 0, s>>>(N, K, Wc, d_table);
         e = cudaGetLastError();
     }
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
@@ -259,6 +311,8 @@ static int launch_count_table_chunked(int N, int K, int Wc, uint32_t* d_table, c
     if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
     if (table_layout(N, K, Wc).rowlen != 0) {
         derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table);
+        if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
+        derive_fast_tables_kernel<<<16, 256, 0, s>>>(N, K, Wc, d_table);
         e = cudaGetLastError();
     }
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);

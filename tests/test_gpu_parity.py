@@ -94,6 +94,17 @@ def _blob_layout(N, K, W):
     for name in ("enc_u", "enc_2v", "enc_v"):
         lay[name] = off
         off += up(N * (K + 2) * top * 4)
+    lay["walkd"] = lay["start"] = lay["cenc0"] = lay["cenc1"] = None
+    if N <= 64 and W <= 6:            # the sections of the shared-memory kernels
+        lay["walkd"] = off
+        off += up(N * rowlen * 8)
+        lay["start"] = off
+        off += 128
+        crow = 32 if K + 1 <= 32 else (64 if K + 1 <= 64 else 128)
+        cb = N * crow * top * 4
+        if W <= 4 and K + 1 <= 128 and 2 * cb <= 160 * 1024:
+            lay["cenc0"], lay["cenc1"], lay["crow"] = off, off + cb, crow
+            off += 2 * cb
     lay["total"] = off
     return lay
 
@@ -136,6 +147,26 @@ def test_table_blob_sections(N, K):
                 prev = V[c1 - 1] if c1 > 0 else 0
                 want = {"enc_u": V[c1] + prev, "enc_2v": 2 * V[c1], "enc_v": V[c1]}[name] & mask
                 assert list(sec[i, c1]) == words(want, top), (name, i, c1)
+    if lay["walkd"] is not None:
+        # the walk table as doubles, saturated at 2^53
+        sec = blob[lay["walkd"] // 4: lay["walkd"] // 4 + N * rowlen * 2].view(np.float64).reshape(N, rowlen)
+        for i in range(N):
+            for col in range(K + 1):
+                assert sec[i, col] == float(min(val[N - 1 - i][col], 1 << 53)), ("walkd", i, col)
+        # U(n,k) = V(n,k) + V(n,k-1) with V(n,k) = sum_{j<=k} N(n,j) (App. C.2); U(-1, .) = 0
+        def U(n, k):
+            return 0 if n < 0 else 2 * sum(val[n][:k + 1]) - val[n][k]
+        assert list(blob[lay["start"] // 4: lay["start"] // 4 + top]) == words(U(N - 1, K) & mask, top)
+    if lay["cenc0"] is not None:
+        for name, off in (("cenc0", lay["cenc0"]), ("cenc1", lay["cenc1"])):
+            crow = lay["crow"]
+            sec = blob[off // 4: off // 4 + N * crow * top].reshape(N, crow, top)
+            assert not sec[:, K + 1:].any()
+            for i in range(N):
+                n = N - 1 - i
+                for k in range(K + 1):
+                    sub = U(n, k) if name == "cenc0" else 2 * sum(val[n][:k + 1])
+                    assert list(sec[i, k]) == words((U(n - 1, k) - sub) & mask, top), (name, i, k)
 
 
 @pytest.mark.parametrize("N,G,b", [(32, 16, 8), (32, 128, 4), (32, 448, 8), (64, 448, 6), (32, 128, 8),

@@ -120,6 +120,30 @@ def test_cumulative_identity():
                 assert sum(t[d][k - j] for j in range(1, m)) == V[d][k - 1] - V[d][k - m]
 
 
+def test_telescoped_enumeration_identity():
+    # Algorithm 2 rewritten with the cumulative counts of App. C.2, as the CUDA encoder uses it:
+    # with U(n,k) = V(n,k) + V(n,k-1), V(n,k) = sum_{j<=k} N(n,j), the term of position i is
+    # U(n,k_i) - U(n,k_{i+1}) for y_i <= 0 and U(n,k_i) - 2 V(n,k_{i+1}) for y_i > 0, so the code is
+    # U(N-1,K) + sum_i [ U(n_i - 1, k_{i+1}) - (U or 2V)(n_i, k_{i+1}) ] with U(-1, .) = 0.
+    rng = np.random.default_rng(3)
+    for (N, K) in [(2, 7), (3, 4), (6, 4), (8, 11), (16, 18), (32, 50)]:
+        t = pr.count_table(N, K)
+        V = [[sum(row[:k + 1]) for k in range(K + 1)] for row in t]
+        U = lambda n, k: 0 if n < 0 else V[n][k] + (V[n][k - 1] if k > 0 else 0)
+        pts = pyramid_points(N, K) if N <= 3 else []
+        for _ in range(200):
+            cuts = np.sort(rng.integers(0, K + 1, size=N - 1))
+            mags = np.diff(np.concatenate(([0], cuts, [K])))
+            pts.append(tuple(int(m) * int(sg) for m, sg in zip(mags, rng.choice([-1, 1], size=N))))
+        for y in pts:
+            code, k = U(N - 1, K), K
+            for i, yi in enumerate(y):
+                n = N - 1 - i
+                k -= abs(yi)
+                code += U(n - 1, k) - (2 * V[n][k] if yi > 0 else U(n, k))
+            assert k == 0 and code == pr.enumerate_point(list(y), K)
+
+
 # -------------------------------------------------------------------- pulses K
 
 @pytest.mark.parametrize("N,bits", [(32, 64), (32, 96), (64, 192), (16, 40), (8, 24), (128, 384)])
