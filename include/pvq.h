@@ -133,10 +133,18 @@ int pvq_build_scale_codebook(int N, int64_t G, int scale_bits, float* d_edges, f
  *   d_x        rows x cols values of `dtype`, leading dimension ld (elements); 16-byte
  *              aligned, ld a multiple of 8 (bf16) or 4 (fp32) elements.
  *   N, K       group size (power of two, 8..256) and pulses (up to 8191, codes of up to 32
- *              words); cols % N == 0; G >= 2.  Codes of up to 2, 3, 4, 6 words at N = 8, 16,
- *              32, 64 run on the kernels with the tables in shared memory.  Wider codes at
- *              N >= 16, and N = 128 and 256, run on slower kernels that keep the tables in
- *              global memory (the paper's grid of group sizes and direction bits, Sec. 4.1).
+ *              words); cols % N == 0; 2 <= G <= 4096.  Codes of up to 2, 3, 4, 6 words at
+ *              N = 8, 16, 32, 64 run on the kernels with the tables in shared memory.  Wider
+ *              codes at N >= 16, and N = 128 and 256, run on slower kernels that keep the
+ *              tables in global memory (the paper's grid of group sizes and direction bits,
+ *              Sec. 4.1).
+ *              Rows of up to 4096 groups are taken by pvq_encode proper (amplitude ||x_g||,
+ *              no rotation) for codes of up to 4 words and K <= 127.  Everything else on the
+ *              encode side - pvq_roundtrip, pvq_encode_amp with amp_mode 1, the rotating
+ *              calls, 5- and 6-word codes, K > 127, the global-table kernels - keeps a whole
+ *              row in one thread block and returns PVQ_ERR_UNSUPPORTED for G > 512 (fewer on
+ *              the global-table kernels, where a row also has to fit shared memory: about
+ *              G <= 256 at N = 128, 192 at N = 256).  Decoding has no such limit.
  *   scale_bits 1..8 (quantile index), or 16 (see pvq_encode_amp).
  *   d_table    from pvq_build_count_table(N, K, ...).
  *   d_edges    2^scale_bits - 1 bin edges.

@@ -36,6 +36,9 @@ struct FastSmem {
     uint32_t ss_off;                // 2 x ss_floats: group energies of a tile
     uint32_t edges_off, idx_off;    // 2 x 256 floats; 2 x idx_words
     int ss_floats, idx_words;
+    // round trip: the decoder's walk tables, 2 x 256 levels, one output slot per thread
+    uint32_t walk_off, walk_bytes, levels_off, wbuf_off;
+    int walk_phases;
 };
 
 // 1.0f where the comparison holds, else 0.0f (one instruction; the flags are then summed or
@@ -137,18 +140,16 @@ __device__ __forceinline__ void index_step(float avs, float t, float one, uint32
 }
 
 // Positions I, I-1, ..., 0 of the index sum.
-template <int N, int W, int TW, int CROW, bool TIES, int I>
+template <int N, int W, int TW, int CROW, int I>
 __device__ __forceinline__ void index_steps(Scaled<N>& s, int K, float v, float& excess, uint32_t& A, mp<W>& c) {
     touch(s.avs[I]);
     const float aa = fabsf(s.avs[I]);
     float t = __fadd_rd(aa, kMagic);
     const float e = __fsub_rn(aa, __fsub_rn(t, kMagic));  // exact
     float one = flag_ge(e, v);
-    if constexpr (TIES) {
-        const float drop = fminf(flag_eq(e, v), excess);  // 1 while pulses are left to take back
-        excess = __fsub_rn(excess, drop);
-        one = __fsub_rn(one, drop);
-    }
+    const float drop = fminf(flag_eq(e, v), excess);  // 1 while pulses are left to take back
+    excess = __fsub_rn(excess, drop);
+    one = __fsub_rn(one, drop);
     float av = s.avs[I];
     if (I == 0 && !s.has_dir) {  // (K, 0, ..., 0)
         t = __int_as_float(kMagicBits + K);
@@ -156,7 +157,7 @@ __device__ __forceinline__ void index_steps(Scaled<N>& s, int K, float v, float&
         av = 1.0f;
     }
     index_step<N, W, TW, CROW, I>(av, t, one, A, c);
-    if constexpr (I > 0) index_steps<N, W, TW, CROW, TIES, I - 1>(s, K, v, excess, A, c);
+    if constexpr (I > 0) index_steps<N, W, TW, CROW, I - 1>(s, K, v, excess, A, c);
 }
 
 // The cut of the greedy fix-up: the d largest residuals e_i = a_i - floor(a_i) get one more
@@ -186,16 +187,13 @@ __device__ __forceinline__ void direction_cut(const Scaled<N>& s, float& v, floa
 template <int N, int W, int TW, int CROW>
 __device__ __forceinline__ mp<W> direction_index(Scaled<N>& s, int K, float v, float excess, uint32_t tab0,
                                                  const mp<W>& start) {
-    // Some thread of the warp may have residuals equal to its cut on both sides of it: coming
-    // from the back, the first `excess` of them give their pulse back (a loop of its own, so
-    // that warps without such ties do not pay for the countdown).
-    const bool ties = __any_sync(kFull, excess > 0.0f);
+    // A thread may have residuals equal to its cut on both sides of it: coming from the back,
+    // the first `excess` of them give their pulse back.  (One loop for all warps: a second,
+    // countdown-free copy for warps without such ties cost more in instruction fetch than the
+    // four instructions per position it saved.)
     mp<W> c = start;
     uint32_t A = tab0;
-    if (!ties)
-        index_steps<N, W, TW, CROW, false, N - 1>(s, K, v, excess, A, c);
-    else
-        index_steps<N, W, TW, CROW, true, N - 1>(s, K, v, excess, A, c);
+    index_steps<N, W, TW, CROW, N - 1>(s, K, v, excess, A, c);
     return c;
 }
 
@@ -240,12 +238,15 @@ __device__ __forceinline__ float warp_tree_sum(const float* p, int gp, int lane)
     return v;
 }
 
-template <int N, int W, bool BF16, int CROW>
+// FUSED: the round trip of pvq_roundtrip.  The code is not stored; once the row energy is known
+// the thread walks it back to its point (pvq_walk.cuh) and writes the bf16 values.
+template <int N, int W, bool BF16, int CROW, bool FUSED, typename YT>
 __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const __grid_constant__ BatchArgs a,
                                                                           const __grid_constant__ FastSmem sm) {
     extern __shared__ __align__(16) uint8_t smem[];
     constexpr int TW = W <= 2 ? W : 4;
     constexpr int RW = BF16 ? N / 2 : N;
+    constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
     const int K = a.K;
     const int b = a.scale_bits;
     const int nedges = b <= 8 ? (1 << b) - 1 : 0;  // 16 bits: the amplitude itself, no codebook
@@ -261,8 +262,18 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
     __shared__ uint64_t stage_bar;
     const BulkStage stage = bulk_stage_begin(&stage_bar);
     if (tid == 0) {
-        bulk_stage_expect(stage, 2u * L.cenc_bytes);
+        bulk_stage_expect(stage, 2u * L.cenc_bytes + (FUSED ? sm.walk_bytes : 0u));
         bulk_stage_copy(stage, smem, reinterpret_cast<const uint8_t*>(a.table) + L.cenc_off[0], 2u * L.cenc_bytes);
+        if constexpr (FUSED)
+            bulk_stage_copy(stage, smem + sm.walk_off, reinterpret_cast<const uint8_t*>(a.table) + L.walk_off[0], sm.walk_bytes);
+    }
+    WalkTables wt;
+    YT* yslots = nullptr;
+    float* s_levels2 = nullptr;
+    if constexpr (FUSED) {
+        wt = walk_tables(L, shared_addr(smem) + sm.walk_off, sm.walk_phases, a);
+        yslots = reinterpret_cast<YT*>(smem + sm.wbuf_off + tid * YS);
+        s_levels2 = reinterpret_cast<float*>(smem + sm.levels_off);
     }
     for (int i = tid; i < 2 * sm.idx_words; i += T) s_idx2[i] = 0u;
     const uint32_t tab0 = shared_addr(smem);
@@ -336,6 +347,8 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
         const bool have_next = next_tile < a.total_tiles;
         const int cur_mi = mi, cur_G = G, cur_gp = gp, cur_rl = rl, cur_g0 = g0, cur_chunks = chunks, cur_rpt = rpt;
         const int cur_idx_words = idx_words;
+        mp<W> kept;  // round trip: this thread's code (one chunk per tile there)
+        mp_zero(kept);
 
         for (int ch = 0; ch < cur_chunks; ++ch) {
             const int g = cur_g0 + ch * T;
@@ -378,7 +391,9 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
                 fetch_first(next_tile, pre);
             }
             const mp<W> c = direction_index<N, W, TW, CROW>(sc, K, v, excess, tab0, start);
-            if (active) {
+            if constexpr (FUSED) {
+                if (active) kept = c;
+            } else if (active) {
                 uint32_t* cp = m.codes + (static_cast<size_t>(row0 + cur_rl) * cur_G + g) * W;
 #pragma unroll
                 for (int w = 0; w < W; ++w) cp[w] = c.w[w];
@@ -390,6 +405,8 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
                 if ((j & (cur_gp - 1)) >= cur_G) s_ss[j] = 0.0f;
         if (nedges != 0 && (buf ? edges1 : edges0) != m.edges) {  // uniform across the block
             for (int i = tid; i < nedges; i += T) s_edges[i] = m.edges[i];
+            if constexpr (FUSED)
+                for (int i = tid; i <= nedges; i += T) s_levels2[buf * 256 + i] = m.levels[i];
             if (buf)
                 edges1 = m.edges;
             else
@@ -397,7 +414,8 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
         }
         __syncthreads();  // this tile's energies (and edges) are in place; the previous tile's index words are complete
 
-        if (!first_tile) flush_idx(prev_mi, tile - gridDim.x, s_idx2 + (buf ^ 1) * sm.idx_words);
+        if constexpr (!FUSED)
+            if (!first_tile) flush_idx(prev_mi, tile - gridDim.x, s_idx2 + (buf ^ 1) * sm.idx_words);
 
         // Row energies: every warp sums the rows its threads sit in (for a row of 32 k groups that
         // is one row; the same sum is then made by several warps, which costs less than a barrier).
@@ -408,6 +426,7 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
             const float sum = warp_tree_sum(s_ss + r * cur_gp, cur_gp, lane);
             if (r == cur_rl) ss_row = sum;
         }
+        float fused_amp = 0.0f;
         for (int ch = 0; ch < cur_chunks; ++ch) {
             const int g = cur_g0 + ch * T;
             if (!(row_ok && g < cur_G)) continue;
@@ -421,6 +440,11 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
                 for (int step = 1 << (b - 1); step >= 1; step >>= 1)
                     if (s_edges[q + step - 1] <= u) q += step;
             }
+            if constexpr (FUSED) {  // the dequantised amplitude, then the walk below
+                fused_amp = b == 16 ? __half2float(__ushort_as_half(static_cast<unsigned short>(q)))
+                                    : __fmul_rn(__fsqrt_rn(ss_row), s_levels2[buf * 256 + q]);
+                continue;
+            }
             if (g == 0) m.row_norm[row0 + cur_rl] = __fsqrt_rn(ss_row);
             const unsigned bit = static_cast<unsigned>(g) * b;
             const unsigned sh = bit & 31u;
@@ -428,18 +452,29 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
             if (sh + b > 32u)
                 atomicOr(&s_idx[cur_rl * cur_idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));
         }
+        if constexpr (FUSED) {
+            // decode the code just made (every thread of the warp walks, in lockstep; a thread
+            // without a group walks code 0)
+            const bool active = row_ok && cur_g0 < cur_G;
+            walk_code<N, W, YT>(kept, wt, K, yslots);
+            if (active)
+                emit_group<N, YT>(m, yslots, fused_amp, static_cast<unsigned>(row0 + cur_rl), static_cast<unsigned>(cur_g0));
+        }
         prev_mi = cur_mi;
         if (!have_next) break;
         tile = next_tile;
     }
-    __syncthreads();  // the last tile's index words are complete
-    flush_idx(prev_mi, tile, s_idx2 + buf * sm.idx_words);
+    if constexpr (!FUSED) {
+        __syncthreads();  // the last tile's index words are complete
+        flush_idx(prev_mi, tile, s_idx2 + buf * sm.idx_words);
+    }
 }
 
 // Geometry and launch.  Returns PVQ_ERR_UNSUPPORTED when the case is not this kernel's (the
 // caller then takes the general kernel).
-template <int N, int W, bool BF16, int CROW>
+template <int N, int W, bool BF16, int CROW, bool FUSED, typename YT>
 static int launch_encode_fast_c(BatchArgs& a, cudaStream_t stream) {
+    constexpr int YS = N * static_cast<int>(sizeof(YT)) + 4;
     constexpr int TW = W <= 2 ? W : 4;
     constexpr int EB = TW * 4;
     DeviceInfo di;
@@ -473,6 +508,7 @@ static int launch_encode_fast_c(BatchArgs& a, cudaStream_t stream) {
     for (int i = 0; i < a.count; ++i) {
         MatrixArgs& m = a.m[i];
         if (m.G > kFastMaxGroups) return PVQ_ERR_UNSUPPORTED;
+        if (FUSED && m.G > threads) return PVQ_ERR_UNSUPPORTED;  // the round trip keeps one code per thread
         m.chunks = m.G <= threads ? 1 : (m.G + threads - 1) / threads;
         m.rows_per_tile = m.G <= threads ? threads / m.G : 1;
         m.tile_begin = tiles;
@@ -493,10 +529,23 @@ static int launch_encode_fast_c(BatchArgs& a, cudaStream_t stream) {
     sm.edges_off = sm.ss_off + 2u * static_cast<uint32_t>(ss_floats) * 4u;
     sm.idx_off = sm.edges_off + 2u * 256u * 4u;
     sm.idx_words = max_idx_words;
-    const size_t smem = sm.idx_off + 2u * static_cast<size_t>(max_idx_words) * 4u;
+    size_t smem = sm.idx_off + 2u * static_cast<size_t>(max_idx_words) * 4u;
+    sm.walk_off = sm.walk_bytes = sm.levels_off = sm.wbuf_off = 0;
+    sm.walk_phases = 0;
+    if (FUSED) {
+        const TableLayout L = table_layout(N, a.K, W);
+        sm.levels_off = static_cast<uint32_t>((smem + 15u) & ~size_t(15));
+        sm.wbuf_off = sm.levels_off + 2u * 256u * 4u;
+        sm.walk_off = (sm.wbuf_off + static_cast<uint32_t>(threads) * YS + 15u) & ~15u;
+        if (sm.walk_off >= static_cast<size_t>(di.smem_max)) return PVQ_ERR_UNSUPPORTED;
+        sm.walk_phases = walk_phases_that_fit(L, static_cast<size_t>(di.smem_max) - sm.walk_off);
+        if (sm.walk_phases == 0) return PVQ_ERR_UNSUPPORTED;
+        sm.walk_bytes = (walk_tables_bytes(L, sm.walk_phases) + 15u) & ~15u;
+        smem = sm.walk_off + sm.walk_bytes;
+    }
     if (smem > static_cast<size_t>(di.smem_max)) return PVQ_ERR_UNSUPPORTED;
 
-    auto kern = encode_fast_kernel<N, W, BF16, CROW>;
+    auto kern = encode_fast_kernel<N, W, BF16, CROW, FUSED, YT>;
     int per_sm = 0;
     if ((st = prepare_kernel(reinterpret_cast<const void*>(kern), threads, smem, &per_sm)) != PVQ_OK) return st;
     if (per_sm < 1) return PVQ_ERR_UNSUPPORTED;
@@ -506,28 +555,32 @@ static int launch_encode_fast_c(BatchArgs& a, cudaStream_t stream) {
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 
-template <int N, int W, bool BF16>
+template <int N, int W, bool BF16, bool FUSED, typename YT>
 static int launch_encode_fast_t(BatchArgs& a, cudaStream_t stream) {
     if constexpr (W > 4) {
         return PVQ_ERR_UNSUPPORTED;  // entries of 24 bytes: the general kernel
     } else {
         const TableLayout L = table_layout(N, a.K, W);
         if (L.cenc_bytes == 0) return PVQ_ERR_UNSUPPORTED;
-        if (L.crow == 32) return launch_encode_fast_c<N, W, BF16, 32>(a, stream);
-        if (L.crow == 64) return launch_encode_fast_c<N, W, BF16, 64>(a, stream);
-        if (L.crow == 128) return launch_encode_fast_c<N, W, BF16, 128>(a, stream);
+        if (L.crow == 32) return launch_encode_fast_c<N, W, BF16, 32, FUSED, YT>(a, stream);
+        if (L.crow == 64) return launch_encode_fast_c<N, W, BF16, 64, FUSED, YT>(a, stream);
+        if (L.crow == 128) return launch_encode_fast_c<N, W, BF16, 128, FUSED, YT>(a, stream);
         return PVQ_ERR_UNSUPPORTED;
     }
 }
 
-// Entry of the per-(N, W) translation units: the plain encode goes to the kernel above when its
-// tables fit, everything else (round trip, rotation, least-squares amplitude) to the general one.
+// Entry of the per-(N, W) translation units: the plain encode and the round trip go to the
+// kernel above when its tables fit (K <= 127 there, so a byte per coordinate), everything else
+// (rotation, least-squares amplitude, larger tables) to the general one.
 template <int N, int W>
 static int launch_encode_any(BatchArgs& a, int dtype, bool fused, cudaStream_t s) {
-    if (!fused && a.rot_block == 0 && a.amp_mode == 0) {
+    if (a.rot_block == 0 && a.amp_mode == 0) {
         BatchArgs b = a;
-        const int st = dtype == PVQ_DTYPE_BF16 ? launch_encode_fast_t<N, W, true>(b, s)
-                                               : launch_encode_fast_t<N, W, false>(b, s);
+        int st;
+        if (dtype == PVQ_DTYPE_BF16)
+            st = fused ? launch_encode_fast_t<N, W, true, true, int8_t>(b, s) : launch_encode_fast_t<N, W, true, false, int8_t>(b, s);
+        else
+            st = fused ? launch_encode_fast_t<N, W, false, true, int8_t>(b, s) : launch_encode_fast_t<N, W, false, false, int8_t>(b, s);
         if (st != PVQ_ERR_UNSUPPORTED) return st;
     }
     return launch_encode_nw<N, W>(a, dtype, fused, s);

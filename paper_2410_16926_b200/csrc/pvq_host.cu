@@ -253,7 +253,7 @@ int fill_matrix(const pvq_matrix_desc& d, int need, int dtype, const Common& c, 
     if (d.rows < 1 || d.cols < 1 || d.cols % c.N != 0) return PVQ_ERR_INVALID_ARG;
     const int64_t G = d.cols / c.N;
     if (G < 2) return PVQ_ERR_UNSUPPORTED;  // the quantile codebook needs two groups (beta > 0)
-    if (G > 1024) return PVQ_ERR_UNSUPPORTED;
+    if (G > 4096) return PVQ_ERR_UNSUPPORTED;  // groups per row (the encoders' row trees; see pvq.h)
     if (d.rows * G >= (int64_t(1) << 31)) return PVQ_ERR_UNSUPPORTED;
     if (need & NEED_X) {
         if (!d.d_x || d.ld < d.cols) return PVQ_ERR_INVALID_ARG;

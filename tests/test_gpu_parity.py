@@ -196,6 +196,10 @@ SMALL = [
     (32, 128, 12, 1024, 6, "bf16"),  # 4-word codes
     (64, 192, 11, 3584, 6, "bf16"),  # N = 64, 6-word codes, G = 56
     (64, 64, 6, 640, 2, "f32"),      # few pulses per position
+    (16, 48, 5, 14336, 4, "bf16"),   # G = 896: the paper's group size 16 on a 14336-column matrix (Sec. 4.1)
+    (32, 96, 3, 28672, 8, "bf16"),   # G = 896 at group size 32: rows longer than a thread block
+    (8, 24, 3, 32768, 4, "f32"),     # G = 4096: the longest row taken
+    (32, 64, 5, 4800, 6, "f32"),     # G = 150: neither a power of two nor a multiple of 32
 ]
 
 
