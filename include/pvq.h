@@ -274,6 +274,25 @@ int pvq_decode_static_table(const uint32_t* d_codes, const uint8_t* d_scale_idx,
                             const float* d_levels, void* d_out, int64_t ld_out, uint32_t* d_status,
                             pvq_stream_t stream);
 
+/* ---- bounds-checked build -------------------------------------------------------------- */
+
+/* Bits of the word of pvq_debug_status. */
+#define PVQ_DEBUG_TABLE_READ 1u   /* a read outside the staged tables */
+#define PVQ_DEBUG_SLOT_WRITE 2u   /* a write outside the thread's output slots */
+#define PVQ_DEBUG_SHARED_INDEX 4u /* an index outside one of the encoders' shared arrays */
+#define PVQ_DEBUG_GLOBAL_STORE 8u /* a store outside an output buffer */
+
+/* The library built with -DPVQ_DEBUG (`python -m paper_2410_16926_b200.build --debug`,
+ * libpvq_b200_debug.so; shared-memory kernels only) checks every table read, slot write,
+ * shared-array index and global store of its kernels against the extent it belongs to,
+ * skips an access that falls outside and ORs the matching bit into *d_status (a device
+ * word of the caller's, zeroed by the caller).  It is the memory-safety evidence of this
+ * code base where a memory checker cannot be run; the results are those of the production
+ * build.  (The paper has no counterpart.)  This call sets the word for all later calls of
+ * the calling thread; NULL switches reporting off.  In the production build it returns
+ * PVQ_ERR_UNSUPPORTED. */
+int pvq_debug_status(uint32_t* d_status);
+
 #ifdef __cplusplus
 }
 #endif

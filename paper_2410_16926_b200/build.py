@@ -1,7 +1,11 @@
 """Build the CUDA library in-tree: csrc/*.cu -> libpvq_b200.so next to this file.
 
-`python -m paper_2410_16926_b200.build [--force] [--verbose]`.  sm_100a only.
+`python -m paper_2410_16926_b200.build [--force] [--verbose] [--debug]`.  sm_100a only.
 Objects go to _build/ (not committed); translation units compile in parallel.
+
+--debug builds libpvq_b200_debug.so instead: the bounds-checked variant (-DPVQ_DEBUG, see
+pvq_debug_status in include/pvq.h) of the kernels that keep their tables in shared memory;
+the global-table kernels are left out of it (calls that need them return "unsupported").
 """
 import os
 import subprocess
@@ -13,6 +17,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJDIR = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "libpvq_b200.so")
+DEBUG_LIB = os.path.join(HERE, "libpvq_b200_debug.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
@@ -28,16 +33,23 @@ def _headers_mtime():
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    os.makedirs(OBJDIR, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    objdir = os.path.join(OBJDIR, "debug") if debug else OBJDIR
+    lib = DEBUG_LIB if debug else LIB
+    os.makedirs(objdir, exist_ok=True)
     hdr = _headers_mtime()
     jobs, objs = [], []
-    for src in _sources():
+    sources = _sources()
+    extra = []
+    if debug:  # the shared-memory kernels only; the rest of the launchers answer "unsupported"
+        sources = [f for f in sources if not f.startswith(("pvq_big", "pvq_wide"))]
+        extra = ["-DPVQ_DEBUG"]
+    for src in sources:
         s = os.path.join(CSRC, src)
-        o = os.path.join(OBJDIR, src[:-3] + ".o")
+        o = os.path.join(objdir, src[:-3] + ".o")
         objs.append(o)
         if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr):
-            cmd = ["nvcc"] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
+            cmd = ["nvcc"] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", s, "-o", o]
             jobs.append(cmd)
 
     def run(cmd):
@@ -51,14 +63,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
                     sys.stderr.write(" ".join(cmd) + "\n" + r.stdout + r.stderr)
                 if r.returncode != 0:
                     raise RuntimeError("nvcc failed for " + cmd[-3])
-    if jobs or not os.path.exists(LIB):
-        link = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] + objs
+    if jobs or not os.path.exists(lib):
+        link = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib] + objs
         r = subprocess.run(link, capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)
             raise RuntimeError("link failed")
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

@@ -25,12 +25,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
     const TableLayout L = table_layout(N, K, W);
     const uint32_t tab_bytes = walk_tables_bytes(L, a.walk_phases);
 
-    // stage the walk tables: one flat bulk copy, waited for below
+    // stage the walk tables with the bulk-copy engine; waited for below
     __shared__ uint64_t stage_bar;
     const BulkStage stage = bulk_stage_begin(&stage_bar);
     if (threadIdx.x == 0) {
-        bulk_stage_expect(stage, tab_bytes);
-        bulk_stage_copy(stage, smem, reinterpret_cast<const uint8_t*>(a.table) + L.walk_off[0], tab_bytes);
+        bulk_stage_expect(stage, walk_tables_stage_bytes(L, a.walk_phases));
+        walk_tables_stage(stage, smem, a.table, L, a.walk_phases);
     }
     const WalkTables wt = walk_tables(L, shared_addr(smem), a.walk_phases, a);
 
@@ -48,13 +48,18 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
         if (a.status && threadIdx.x == 0) atomicOr(a.status, PVQ_STATUS_STAGING_TIMEOUT);
         return;
     }
+#ifdef PVQ_DEBUG
+    debug_begin(shared_addr(smem), shared_addr(smem) + tab_bytes, shared_addr(smem) + ((tab_bytes + 15u) & ~15u), YS,
+                N * static_cast<uint32_t>(sizeof(YT)), a.debug_status);
+#endif
 
     const unsigned b = a.scale_bits;
     const unsigned warps_total = gridDim.x * (blockDim.x >> 5);
     bool bad = false;
 
+    int mi = 0;  // the matrices follow one another: the tile's matrix only ever moves on
     for (unsigned tile = blockIdx.x * (blockDim.x >> 5) + warp; tile < a.total_tiles; tile += warps_total) {
-        const int mi = find_matrix(a, tile);
+        while (mi + 1 < a.count && tile >= a.m[mi + 1].tile_begin) ++mi;
         const MatrixArgs& m = a.m[mi];
         const unsigned G = static_cast<unsigned>(m.G);
         const unsigned ngroups = static_cast<unsigned>(m.rows) * G;  // below 2^31 (checked by the host)

@@ -262,10 +262,9 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
     __shared__ uint64_t stage_bar;
     const BulkStage stage = bulk_stage_begin(&stage_bar);
     if (tid == 0) {
-        bulk_stage_expect(stage, 2u * L.cenc_bytes + (FUSED ? sm.walk_bytes : 0u));
+        bulk_stage_expect(stage, 2u * L.cenc_bytes + (FUSED ? walk_tables_stage_bytes(L, sm.walk_phases) : 0u));
         bulk_stage_copy(stage, smem, reinterpret_cast<const uint8_t*>(a.table) + L.cenc_off[0], 2u * L.cenc_bytes);
-        if constexpr (FUSED)
-            bulk_stage_copy(stage, smem + sm.walk_off, reinterpret_cast<const uint8_t*>(a.table) + L.walk_off[0], sm.walk_bytes);
+        if constexpr (FUSED) walk_tables_stage(stage, smem + sm.walk_off, a.table, L, sm.walk_phases);
     }
     WalkTables wt;
     YT* yslots = nullptr;
@@ -334,6 +333,11 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
         return;
     }
     __syncthreads();  // index words cleared
+#ifdef PVQ_DEBUG
+    // tables: the two telescoped ones with the slack behind them, and (round trip) the walk tables
+    debug_begin(tab0, tab0 + (FUSED ? sm.walk_off + sm.walk_bytes : sm.tab_bytes), tab0 + sm.wbuf_off, YS,
+                N * static_cast<uint32_t>(sizeof(YT)), a.debug_status);
+#endif
 
     int buf = 0, prev_mi = mi;
     for (bool first_tile = true;; buf ^= 1, first_tile = false) {
@@ -376,7 +380,7 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
                     t[i] = __fmul_rn(xi, xi);
                 }
                 ss = tree_sum<N>(t);
-                if (active) s_ss[cur_rl * cur_gp + g] = ss;
+                if (active && PVQ_DEBUG_INDEX(cur_rl * cur_gp + g, sm.ss_floats, PVQ_DEBUG_SHARED_INDEX)) s_ss[cur_rl * cur_gp + g] = ss;
                 direction_begin<N, BF16>(raw, l1, K, sc);
             }
             float v, excess;
@@ -395,14 +399,16 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
                 if (active) kept = c;
             } else if (active) {
                 uint32_t* cp = m.codes + (static_cast<size_t>(row0 + cur_rl) * cur_G + g) * W;
+                if (PVQ_DEBUG_INDEX((row0 + cur_rl) * cur_G + g, m.rows * cur_G, PVQ_DEBUG_GLOBAL_STORE)) {
 #pragma unroll
-                for (int w = 0; w < W; ++w) cp[w] = c.w[w];
+                    for (int w = 0; w < W; ++w) cp[w] = c.w[w];
+                }
             }
         }
         // zero padding of the rows' trees
         if (cur_gp != cur_G)
             for (int j = tid; j < cur_rpt * cur_gp; j += T)
-                if ((j & (cur_gp - 1)) >= cur_G) s_ss[j] = 0.0f;
+                if ((j & (cur_gp - 1)) >= cur_G && PVQ_DEBUG_INDEX(j, sm.ss_floats, PVQ_DEBUG_SHARED_INDEX)) s_ss[j] = 0.0f;
         if (nedges != 0 && (buf ? edges1 : edges0) != m.edges) {  // uniform across the block
             for (int i = tid; i < nedges; i += T) s_edges[i] = m.edges[i];
             if constexpr (FUSED)
@@ -445,9 +451,12 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
                                     : __fmul_rn(__fsqrt_rn(ss_row), s_levels2[buf * 256 + q]);
                 continue;
             }
-            if (g == 0) m.row_norm[row0 + cur_rl] = __fsqrt_rn(ss_row);
+            if (g == 0 && PVQ_DEBUG_INDEX(row0 + cur_rl, m.rows, PVQ_DEBUG_GLOBAL_STORE))
+                m.row_norm[row0 + cur_rl] = __fsqrt_rn(ss_row);
             const unsigned bit = static_cast<unsigned>(g) * b;
             const unsigned sh = bit & 31u;
+            if (!PVQ_DEBUG_INDEX(cur_rl * cur_idx_words + (bit >> 5) + (sh + b > 32u ? 1 : 0), sm.idx_words, PVQ_DEBUG_SHARED_INDEX))
+                continue;
             atomicOr(&s_idx[cur_rl * cur_idx_words + (bit >> 5)], static_cast<uint32_t>(q) << sh);
             if (sh + b > 32u)
                 atomicOr(&s_idx[cur_rl * cur_idx_words + (bit >> 5) + 1], static_cast<uint32_t>(q) >> (32u - sh));

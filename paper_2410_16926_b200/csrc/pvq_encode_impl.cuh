@@ -429,10 +429,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     const BulkStage stage = bulk_stage_begin(&stage_bar);
     if (threadIdx.x == 0) {
         const uint8_t* blob = reinterpret_cast<const uint8_t*>(a.table);
-        bulk_stage_expect(stage, sm.enc_bytes + (FUSED ? sm.walk_bytes : 0u));
+        bulk_stage_expect(stage, sm.enc_bytes + (FUSED ? walk_tables_stage_bytes(L, sm.walk_phases) : 0u));
         if (sm.enc_bytes)
             bulk_stage_copy(stage, smem, blob + (sm.enum_mode == 2 ? L.enc_off[0] : L.enc_off[2]), sm.enc_bytes);
-        if constexpr (FUSED) bulk_stage_copy(stage, smem + sm.enc_bytes, blob + L.walk_off[0], sm.walk_bytes);
+        if constexpr (FUSED) walk_tables_stage(stage, smem + sm.enc_bytes, a.table, L, sm.walk_phases);
     }
     for (int i = threadIdx.x; i < 2 * sm.idx_words; i += blockDim.x) s_idx2[i] = 0u;
     const uint32_t tabA = shared_addr(smem);
@@ -458,6 +458,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
     }
     if (!bulk_stage_wait(stage)) return;  // the tables never arrived: leave rather than spin
     __syncthreads();                      // index words cleared
+#ifdef PVQ_DEBUG
+    debug_begin(tabA, tabA + sm.enc_bytes + (FUSED ? sm.walk_bytes : 0u), tabA + sm.wbuf_off, YS,
+                N * static_cast<uint32_t>(sizeof(YT)), a.debug_status);
+#endif
     struct {
         bool valid;
         int mi, rpt;
@@ -501,7 +505,7 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             }
             ss = tree_sum<N>(t);
         }
-        if (active) {
+        if (active && PVQ_DEBUG_INDEX(rl * gp + g, sm.ss_floats, PVQ_DEBUG_SHARED_INDEX)) {
             s_ss[rl * gp + g] = ss;
             if (g < gp - G) s_ss[rl * gp + G + g] = 0.0f;  // zero padding of the row's tree
         }
@@ -620,8 +624,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
             if (active) {
                 if (g == 0) m.row_norm[row] = rnorm;
                 uint32_t* cp = m.codes + (static_cast<size_t>(row) * G + g) * W;
+                if (PVQ_DEBUG_INDEX(row * G + g, m.rows * G, PVQ_DEBUG_GLOBAL_STORE)) {
 #pragma unroll
-                for (int w = 0; w < W; ++w) cp[w] = c.w[w];
+                    for (int w = 0; w < W; ++w) cp[w] = c.w[w];
+                }
                 const unsigned bit = static_cast<unsigned>(g) * b;
                 const unsigned sh = bit & 31u;
                 atomicOr(&s_idx[rl * idx_words + (bit >> 5)], static_cast<uint32_t>(q) << sh);

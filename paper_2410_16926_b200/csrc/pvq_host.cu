@@ -222,6 +222,27 @@ extern "C" size_t pvq_scale_row_stride(int64_t G, int scale_bits) {
     return (bytes + 3u) & ~static_cast<size_t>(3u);
 }
 
+// ------------------------------------------------------ bounds-checked build
+
+static thread_local uint32_t* g_debug_status = nullptr;
+
+#ifdef PVQ_DEBUG
+namespace pvq {
+// the global-table kernels are not part of the bounds-checked build
+int launch_big(const BatchArgs&, int, int, int, bool, cudaStream_t) { return PVQ_ERR_UNSUPPORTED; }
+}  // namespace pvq
+#endif
+
+extern "C" int pvq_debug_status(uint32_t* d_status) {
+#ifdef PVQ_DEBUG
+    g_debug_status = d_status;
+    return PVQ_OK;
+#else
+    (void)d_status;
+    return PVQ_ERR_UNSUPPORTED;
+#endif
+}
+
 // ------------------------------------------------------ public: hot-path calls
 
 namespace {
@@ -308,6 +329,7 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
     a.status = d_status;
     a.c_one = 1u;
     a.c_minus_one = 0xffffffffu;
+    a.debug_status = g_debug_status;
     if (amp_mode != 0 && amp_mode != 1) return PVQ_ERR_INVALID_ARG;
     a.amp_mode = amp_mode;
     if (rot_block != 0) {

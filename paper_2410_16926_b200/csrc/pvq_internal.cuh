@@ -42,7 +42,7 @@ struct BatchArgs {
     int code_words;         // W: 32-bit words of one code in memory (kernels may compute in more)
     const uint32_t* table;  // the blob written by pvq_build_count_table (see TableLayout)
     uint32_t* status;
-    int walk_phases;        // decode: how many of the walk tables are staged in shared memory (1..3)
+    int walk_phases;        // decode: which walk tables are staged in shared memory (see walk_tables)
     // The integers 1 and -1 as kernel arguments.  Multiply-adds by a factor the assembler cannot
     // see through stay multiply-adds, which run on the FMA pipe; the walk uses them for plain
     // moves, adds and subtracts to take load off the integer ALU pipe, its bottleneck.
@@ -52,6 +52,7 @@ struct BatchArgs {
     int fused;               // global-table encoder: decode the code just made instead of storing it
     const float* rot_signs;  // +-1, rot_block of them
     int rot_block;           // power of two, a multiple of N, dividing every cols
+    uint32_t* debug_status;  // bounds-checked build: where violations are reported (pvq_debug_status); else null
 };
 
 // Layout of the table blob.  Section 0 is the count table as the paper defines it,
@@ -230,6 +231,59 @@ __device__ __forceinline__ int find_matrix(const BatchArgs& a, unsigned tile) {
         if (tile >= a.m[i].tile_begin) mi = i;
     return mi;
 }
+
+// ---- bounds-checked build (-DPVQ_DEBUG) ---------------------------------------------------
+// Every read of a staged table, every write of an output slot, the indices of the encoders'
+// shared arrays and the global stores are checked against the extent they belong to; a
+// violation ORs a bit into the word given to pvq_debug_status and the access is skipped
+// (nothing traps).  The decode walk runs its plain C++ step in this build, so that each of
+// its table reads and slot writes passes through the checked helpers; the hand-written
+// forms of the production build take the same pointers through the same transitions.
+#ifdef PVQ_DEBUG
+struct DebugCtx {
+    uint32_t tab_lo, tab_hi;                      // shared addresses: the staged tables
+    uint32_t slot_base, slot_stride, slot_bytes;  // output slots: thread t owns [base + t * stride, + bytes)
+    uint32_t* status;
+};
+__shared__ DebugCtx s_debug;
+
+// thread 0 fills the context; the caller's next block-wide barrier publishes it
+__device__ __forceinline__ void debug_begin(uint32_t tab_lo, uint32_t tab_hi, uint32_t slot_base, uint32_t slot_stride,
+                                            uint32_t slot_bytes, uint32_t* status) {
+    if (threadIdx.x == 0) {
+        s_debug.tab_lo = tab_lo;
+        s_debug.tab_hi = tab_hi;
+        s_debug.slot_base = slot_base;
+        s_debug.slot_stride = slot_stride;
+        s_debug.slot_bytes = slot_bytes;
+        s_debug.status = status;
+    }
+    __syncthreads();
+}
+__device__ __forceinline__ void debug_flag(uint32_t bit) {
+    if (s_debug.status) atomicOr(s_debug.status, bit);
+}
+__device__ __forceinline__ bool debug_table_ok(uint32_t addr, uint32_t bytes) {
+    const bool ok = addr >= s_debug.tab_lo && addr + bytes <= s_debug.tab_hi && (addr & 3u) == 0u;
+    if (!ok) debug_flag(PVQ_DEBUG_TABLE_READ);
+    return ok;
+}
+__device__ __forceinline__ bool debug_slot_ok(uint32_t addr, uint32_t bytes) {
+    const uint32_t lo = s_debug.slot_base + threadIdx.x * s_debug.slot_stride;
+    const bool ok = addr >= lo && addr + bytes <= lo + s_debug.slot_bytes;
+    if (!ok) debug_flag(PVQ_DEBUG_SLOT_WRITE);
+    return ok;
+}
+// index into one of the encoders' shared arrays / a global output
+__device__ __forceinline__ bool debug_index_ok(long long idx, long long limit, uint32_t bit) {
+    const bool ok = idx >= 0 && idx < limit;
+    if (!ok) debug_flag(bit);
+    return ok;
+}
+#define PVQ_DEBUG_INDEX(idx, limit, bit) debug_index_ok((idx), (limit), (bit))
+#else
+#define PVQ_DEBUG_INDEX(idx, limit, bit) true
+#endif
 
 #endif  // __CUDACC__
 

@@ -95,6 +95,17 @@ __device__ __forceinline__ bool bulk_stage_wait(const BulkStage& st) {
 template <int PW, int OFF = 0>
 __device__ __forceinline__ mp<PW> load_entry(uint32_t addr) {
     mp<PW> t;
+#ifdef PVQ_DEBUG
+    {  // checked, word by word (no alignment beyond 4 bytes assumed); an access outside reads as zero
+        const bool ok = debug_table_ok(addr + OFF, PW * 4);
+#pragma unroll
+        for (int w = 0; w < PW; ++w) {
+            t.w[w] = 0u;
+            if (ok) asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t.w[w]) : "r"(addr + static_cast<uint32_t>(OFF + 4 * w)));
+        }
+        return t;
+    }
+#endif
     if constexpr (PW == 1) {
         asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(t.w[0]) : "r"(addr), "n"(OFF));
     } else if constexpr (PW == 2) {
@@ -119,6 +130,9 @@ __device__ __forceinline__ mp<PW> load_entry(uint32_t addr) {
 
 template <typename YT>
 __device__ __forceinline__ void store_y(uint32_t addr, int val) {
+#ifdef PVQ_DEBUG
+    if (!debug_slot_ok(addr, sizeof(YT))) return;
+#endif
     if constexpr (sizeof(YT) == 1)
         asm volatile("st.shared.u8 [%0], %1;" ::"r"(addr), "r"(val) : "memory");
     else
@@ -886,6 +900,10 @@ __device__ __forceinline__ void walk_block8_5of6(mp<5>& r, uint32_t& p, int& v, 
 template <int PW, int EB, bool HEADROOM, typename YT, int U>
 __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32_t& y, const int D,
                                           const Factors f) {
+#ifdef PVQ_DEBUG
+    walk_step_wide<PW, EB, YT, U>(r, p, v, y, D);  // the plain step: every access through the checked helpers
+    return;
+#endif
     if constexpr (HEADROOM && PW == 1)
         walk_step_1<EB, YT, U>(r.w[0], p, v, y, D, f);
     else if constexpr (HEADROOM && PW == 2)
@@ -917,6 +935,19 @@ __device__ __forceinline__ void walk_step(mp<PW>& r, uint32_t& p, int& v, uint32
 template <int PW, int EB, bool HEADROOM, typename YT>
 __device__ __forceinline__ void walk_block8(mp<PW>& r, uint32_t& p, int& v, uint32_t& y, const int D,
                                             const Factors f) {
+#ifdef PVQ_DEBUG
+    if constexpr (true) {
+        walk_step<PW, EB, HEADROOM, YT, 0>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 1>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 2>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 3>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 4>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 5>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 6>(r, p, v, y, D, f);
+        walk_step<PW, EB, HEADROOM, YT, 7>(r, p, v, y, D, f);
+        return;
+    }
+#endif
     if constexpr (HEADROOM && PW == 1) {
         walk_block8_1<YT>(r.w[0], p, v, y, D, f);
     } else if constexpr (HEADROOM && PW == 2 && EB == 8) {
@@ -1003,13 +1034,16 @@ struct WalkTables {
     Factors f;
 };
 
+// `phases`: how many of the walk tables are staged, in the blob's order (widest, two-word,
+// one-word): 1, 2 or 3; or 4 = the widest and the one-word table only, the one-word table
+// directly behind the widest (when the two-word table does not fit beside them).
 __device__ __forceinline__ WalkTables walk_tables(const TableLayout& L, uint32_t smem_base, int phases,
                                                   const BatchArgs& a) {
     WalkTables t;
     t.tab0 = smem_base;
     t.tab2 = smem_base + (L.walk_off[1] - L.walk_off[0]);
-    t.tab1 = smem_base + (L.walk_off[2] - L.walk_off[0]);
-    t.has2 = phases >= 2 && L.walk_bytes[1] != 0;
+    t.tab1 = phases == 4 ? smem_base + ((L.walk_bytes[0] + 127u) & ~127u) : smem_base + (L.walk_off[2] - L.walk_off[0]);
+    t.has2 = (phases == 2 || phases == 3) && L.walk_bytes[1] != 0;
     t.has1 = phases >= 3;
     t.rowlen = L.rowlen;
     t.f.one = a.c_one;
@@ -1018,17 +1052,37 @@ __device__ __forceinline__ WalkTables walk_tables(const TableLayout& L, uint32_t
 }
 
 __host__ __device__ inline uint32_t walk_tables_bytes(const TableLayout& L, int phases) {
+    if (phases == 4) return ((L.walk_bytes[0] + 127u) & ~127u) + L.walk_bytes[2];
     return L.walk_off[phases - 1] + L.walk_bytes[phases - 1] - L.walk_off[0];
 }
 
-// How many of the walk tables (a prefix of: widest, two-word, one-word) fit in `room` bytes
-// of shared memory; 0 when not even the widest does.
+// Which walk tables fit in `room` bytes of shared memory (see walk_tables for the codes): all
+// three, the widest two, the widest and the one-word one, the widest alone; 0 when not even that.
 inline int walk_phases_that_fit(const TableLayout& L, size_t room) {
-    for (int p = 3; p >= 1; --p) {
-        if (p > 1 && L.walk_bytes[p - 1] == 0) continue;
+    const int order[4] = {3, 2, 4, 1};
+    for (int p : order) {
+        if (p == 3 && L.walk_bytes[2] == 0) continue;  // one-word codes: the widest table is all there is
+        if (p == 2 && L.walk_bytes[1] == 0) continue;  // no two-word copy (codes of one or two words)
+        if (p == 4 && (L.walk_bytes[1] == 0 || L.walk_bytes[2] == 0)) continue;  // 3 covers these
         if (((walk_tables_bytes(L, p) + 15u) & ~size_t(15)) <= room) return p;
     }
     return 0;
+}
+
+// Stages the chosen walk tables at `dst` (thread 0 only, between bulk_stage_expect and the wait).
+__device__ __forceinline__ void walk_tables_stage(const BulkStage& st, void* dst, const uint32_t* blob,
+                                                  const TableLayout& L, int phases) {
+    const uint8_t* src = reinterpret_cast<const uint8_t*>(blob);
+    if (phases == 4) {
+        bulk_stage_copy(st, dst, src + L.walk_off[0], L.walk_bytes[0]);
+        bulk_stage_copy(st, static_cast<uint8_t*>(dst) + ((L.walk_bytes[0] + 127u) & ~127u), src + L.walk_off[2],
+                        L.walk_bytes[2]);
+    } else {
+        bulk_stage_copy(st, dst, src + L.walk_off[0], walk_tables_bytes(L, phases));
+    }
+}
+__host__ __device__ inline uint32_t walk_tables_stage_bytes(const TableLayout& L, int phases) {
+    return phases == 4 ? L.walk_bytes[0] + L.walk_bytes[2] : walk_tables_bytes(L, phases);
 }
 
 // Code c (destroyed) -> the thread's N slots `yslots` in shared memory.
@@ -1092,6 +1146,9 @@ __device__ __forceinline__ void emit_group(const MatrixArgs& m, const YT* yslots
         for (int v = 0; v < N; ++v) ssy += static_cast<int>(yslots[v]) * static_cast<int>(yslots[v]);
     }
     const float sc = __fdiv_rn(amp, __fsqrt_rn(static_cast<float>(ssy)));
+    if (!PVQ_DEBUG_INDEX(static_cast<long long>(row), m.rows, PVQ_DEBUG_GLOBAL_STORE) ||
+        !PVQ_DEBUG_INDEX(static_cast<long long>(g + 1) * N - 1, m.cols, PVQ_DEBUG_GLOBAL_STORE))
+        return;
     uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.out) + static_cast<size_t>(row) * m.ld_out +
                                           static_cast<size_t>(g) * N);
 #pragma unroll

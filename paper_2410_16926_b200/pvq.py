@@ -12,7 +12,9 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libpvq_b200.so")
+# PVQ_B200_LIB selects another build of the same library, e.g. the bounds-checked one
+# (libpvq_b200_debug.so, see pvq_debug_status in include/pvq.h).
+LIB_PATH = os.environ.get("PVQ_B200_LIB") or os.path.join(_HERE, "libpvq_b200.so")
 
 DTYPE_F32 = 0
 DTYPE_BF16 = 1
@@ -69,6 +71,7 @@ def lib():
         L.pvq_rotate_encode.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.pvq_rotate_roundtrip.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, i32, i32, vp, vp, vp, vp, i64, vp]
         L.pvq_decode_static_table.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, i64, vp, vp]
+        L.pvq_debug_status.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -76,7 +79,8 @@ def lib():
 EXPORTS = ["pvq_strerror", "pvq_last_cuda_error", "pvq_index_bits", "pvq_max_pulses", "pvq_code_words",
            "pvq_count_table_bytes", "pvq_scale_row_stride", "pvq_build_count_table",
            "pvq_build_scale_codebook", "pvq_encode", "pvq_decode", "pvq_roundtrip", "pvq_encode_batched",
-           "pvq_decode_batched", "pvq_decode_static_table", "pvq_rotate_encode", "pvq_rotate_roundtrip", "pvq_encode_amp"]
+           "pvq_decode_batched", "pvq_decode_static_table", "pvq_rotate_encode", "pvq_rotate_roundtrip", "pvq_encode_amp",
+           "pvq_debug_status"]
 
 
 def _check(status, where):
@@ -106,6 +110,12 @@ def _dtype_code(x):
     if x.dtype == torch.bfloat16:
         return DTYPE_BF16
     raise TypeError("input must be float32 or bfloat16")
+
+
+def debug_status(word):
+    """Bounds-checked build only: violations are ORed into `word` (an int32 device tensor of one
+    element, zeroed by the caller) by every later call of this thread; None switches it off."""
+    _check(lib().pvq_debug_status(_ptr(word, torch.int32)), "pvq_debug_status")
 
 
 # ---- host helpers ---------------------------------------------------------------

@@ -24,3 +24,38 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _bounds_checked_build_reports_nothing(request):
+    """When the suite runs on the bounds-checked library (PVQ_B200_LIB points at
+    libpvq_b200_debug.so and PVQ_B200_DEBUG_STATUS is set; tests/test_gpu_bounds_checked.py
+    starts such a run), every GPU test hands the library a zeroed status word and must
+    find it zero afterwards: no table read, slot write, shared-array index or global
+    store of any kernel left its extent."""
+    if not os.environ.get("PVQ_B200_DEBUG_STATUS") or "gpu" not in request.keywords:
+        yield
+        return
+    import torch
+    from paper_2410_16926_b200 import pvq
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    pvq.debug_status(word)
+    yield
+    torch.cuda.synchronize()
+    pvq.debug_status(None)
+    assert int(word.item()) == 0, "bounds-checked build reported violation bits %#x" % int(word.item())
+
+
+@pytest.hookimpl(hookwrapper=True)
+def pytest_runtest_call(item):
+    """On the bounds-checked build the global-table kernels are absent: a case that needs
+    them (the library answers PVQ_ERR_UNSUPPORTED) counts as skipped there, not failed."""
+    outcome = yield
+    if not os.environ.get("PVQ_B200_DEBUG_STATUS") or outcome.excinfo is None:
+        return
+    exc = outcome.excinfo[1]
+    if type(exc).__name__ == "PvqError" and getattr(exc, "status", None) == 2:
+        try:
+            pytest.skip("not part of the bounds-checked build")
+        except BaseException:
+            outcome.force_exception(sys.exc_info()[1])

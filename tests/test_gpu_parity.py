@@ -43,10 +43,28 @@ class Codec:
         self.levels = torch.from_numpy(self.levels_np).to(DEV)
 
 
+GUARD = 64   # canary elements behind every output buffer
+
+
+def guarded(shape, dtype, fill):
+    """A tensor of `shape` whose storage is followed by GUARD canary elements; returns
+    (tensor, check) where check() asserts that the canaries still hold `fill`."""
+    n = int(np.prod(shape))
+    flat = torch.full((n + GUARD,), fill, dtype=dtype, device=DEV)
+    def check():
+        assert bool((flat[n:] == fill).all()), "written past the end of an output buffer"
+    return flat[:n].view(*shape), check
+
+
 def check_encode(cd, x_np, kind, x_dev=None):
     x_dev = to_device(x_np, kind) if x_dev is None else x_dev
-    codes, sidx, rnorm = pvq.encode(x_dev, cd.N, cd.K, cd.b, cd.table, cd.edges)
+    rows = x_np.shape[0]
+    codes, c1 = guarded((rows, cd.G, cd.W), torch.int32, 0x5A5A5A5A)
+    sidx, c2 = guarded((rows, int(pvq.scale_row_stride(cd.G, cd.b))), torch.uint8, 0xA5)
+    rnorm, c3 = guarded((rows,), torch.float32, 12345.0)
+    pvq.encode(x_dev, cd.N, cd.K, cd.b, cd.table, cd.edges, out=(codes, sidx, rnorm))
     torch.cuda.synchronize()
+    c1(), c2(), c3()
     o_codes, o_sidx, o_rnorm = po.encode(x_np, cd.N, cd.K, cd.b, cd.edges_np, W=cd.W)
     assert np.array_equal(rnorm.cpu().numpy().view(np.uint32), o_rnorm.view(np.uint32)), "row norms"
     assert np.array_equal(sidx.cpu().numpy(), o_sidx), "amplitude indices"
@@ -57,8 +75,11 @@ def check_encode(cd, x_np, kind, x_dev=None):
 
 def check_decode(cd, enc_dev, enc_np):
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    out = pvq.decode(*enc_dev, cd.N, cd.K, cd.b, cd.table, cd.levels, status=status)
+    rows, G, _ = enc_dev[0].shape
+    out, c1 = guarded((rows, G * cd.N), torch.bfloat16, 7.0)
+    pvq.decode(*enc_dev, cd.N, cd.K, cd.b, cd.table, cd.levels, status=status, out=out)
     torch.cuda.synchronize()
+    c1()
     o_out, o_status = po.decode(*enc_np, cd.N, cd.K, cd.b, cd.levels_np)
     assert int(status.item()) == o_status
     bad = np.argwhere(bf16_bits(out) != o_out)
