@@ -36,14 +36,26 @@ FALLBACK_HBM_GBS = 6650.0
 
 # Per-launch counters of the kernels from the ncu captures summarised under profiles/ (same
 # workload and launch configuration as this bench): DRAM bytes read + written, and warp
-# instructions executed.  Set an entry to None when its kernel changes until it is re-captured.
+# instructions executed.  They hold for the CUDA sources they were captured from, whose hash
+# is recorded with them; with any other sources the line reports them as null.
+NCU_SOURCES = "419c039013919f73"
 NCU_COUNTERS = {
-    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_969_920 + 1_792, "warp_inst": 32_479_472},
-    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_658_816 + 473_600, "warp_inst": 37_778_508},
-    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_471_936 + 88_764_672, "warp_inst": 214_752_520},
-    ("c6_bf16_q_proj_group128", "encode"): {"dram_bytes": 34_222_592 + 5_632, "warp_inst": 89_047_985},
-    ("c6_bf16_q_proj_group128", "decode"): {"dram_bytes": 7_047_936 + 222_720, "warp_inst": 81_724_198},
+    ("c3_llama3_8b_layer", "encode"): {"dram_bytes": 436_335_360 + 74_592_256, "warp_inst": 401_893_184,
+                                       "kernel": "encode_fast_kernel<32,3,bf16>", "profile": "profiles/encode_fast_kernel_c3.md"},
+    ("c3_llama3_8b_layer", "decode"): {"dram_bytes": 88_886_016 + 391_325_952, "warp_inst": 487_979_342,
+                                       "kernel": "decode_kernel<32,3,int8>", "profile": "profiles/decode_kernel_c3.md"},
+    ("c2_bf16_q_proj", "encode"): {"dram_bytes": 33_673_728 + 0, "warp_inst": 30_391_824,
+                                   "kernel": "encode_fast_kernel<32,3,bf16>", "profile": "profiles/encode_fast_kernel_c2.md"},
+    ("c2_bf16_q_proj", "decode"): {"dram_bytes": 6_662_400 + 1_076_992, "warp_inst": 38_158_702,
+                                   "kernel": "decode_kernel<32,3,int8>", "profile": "profiles/decode_kernel_c2.md"},
+    ("c4_bf16_down_proj_70b", "decode"): {"dram_bytes": 91_125_248 + 422_567_168, "warp_inst": 649_471_394,
+                                          "kernel": "decode_kernel<64,6,int8>", "profile": "profiles/decode_kernel_c4.md"},
+    ("c5_bf16_activations", "roundtrip"): {"dram_bytes": 134_318_848 + 91_176_960, "warp_inst": 208_252_664,
+                                           "kernel": "encode_fast_kernel<32,2,bf16,FUSED>",
+                                           "profile": "profiles/roundtrip_kernel_c5.md"},
 }
+for _c in NCU_COUNTERS.values():
+    _c["kernel_sha"] = NCU_SOURCES
 SMS, SCHEDULERS_PER_SM = 148, 4      # issue slots per cycle on the part = SMS * SCHEDULERS_PER_SM
 
 
@@ -438,6 +450,9 @@ def oracle_sample(wl, target_seconds=12.0):
     nb, t = run(probe)
     frac = min(1.0, probe * target_seconds / max(t, 1e-4))
     nb, t = run(frac)
+    if frac < 1.0 and t < target_seconds / 2:        # the probe overestimated the cost per row: scale once more
+        frac = min(1.0, frac * target_seconds / max(t, 1e-4))
+        nb, t = run(frac)
     reps = 1
     if frac >= 1.0 and t < target_seconds / 4:       # the whole workload is quick: repeat it for a steadier figure
         reps = int(min(20, max(1, target_seconds / 4 / max(t, 1e-4))))
@@ -514,6 +529,29 @@ def kernel_table(wl, per, peak, peak_kind):
                          "frac_of_%s_hbm" % peak_kind: nbytes / (avg * 1e-3) / 1e9 / peak,
                          "frac_of_nominal_8TBps": nbytes / (avg * 1e-3) / 1e9 / 8000.0}
     return kernels
+
+
+def issue_table(wl, kernels, clocks, sha):
+    """The limit that binds in practice: instruction issue (every kernel here is integer work on
+    a table walk or a sorting network).  achieved = warp instructions per launch (from the ncu
+    capture under profiles/, valid while the sources are unchanged) / the time measured in this
+    run; peak = issue slots per second at the SM clock sampled during the run."""
+    issue = {}
+    mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz")
+    for name in kernels:
+        c = NCU_COUNTERS.get((wl.name, name))
+        pk = SMS * SCHEDULERS_PER_SM * mhz * 1e6 if mhz else None
+        entry = {"bound": "alu", "peak": pk / 1e9 if pk else None, "unit": "Gwarp-inst/s",
+                 "peak_source": "148 SMs x 4 schedulers x sampled SM clock"}
+        if c and c.get("kernel_sha") == sha and pk:
+            ach = c["warp_inst"] / (kernels[name]["avg_ms"] * 1e-3)
+            entry.update({"achieved": ach / 1e9, "frac": ach / pk, "warp_inst_per_weight": c["warp_inst"] / wl.weights,
+                          "warp_inst_source": "ncu capture %s (not this run)" % c["profile"]})
+        else:
+            entry.update({"achieved": None, "frac": None, "warp_inst_per_weight": None,
+                          "warp_inst_source": "no capture of the current sources"})
+        issue[name] = entry
+    return issue
 
 
 def timed_run(run, steps, warmup, sampler, barrier, min_warm_seconds=0.3):
@@ -644,6 +682,7 @@ def main():
                                      "value": sb2 * o_steps / (ms2 * 1e-3) / 1e9, "unit": "GB/s",
                                      "config": config_of(wl2, run2.K, run2.W),
                                      "kernels": kernel_table(wl2, per2, peak, peak_kind), "clocks": clk2}
+            other_lines[wl2.name]["issue"] = issue_table(wl2, other_lines[wl2.name]["kernels"], clk2, sha)
             del run2
             torch.cuda.empty_cache()
     sampler.stop()
@@ -658,30 +697,12 @@ def main():
     ncu = NCU_COUNTERS.get((wl.name, dom))
     if ncu and ncu.get("kernel_sha") != sha:
         ncu = None                      # the kernels have changed since the counters were taken
-    roofline = {"kernel": "pvq %s_kernel" % dom, "bound": "hbm", "achieved": kernels[dom]["GBps"], "peak": peak,
+    roofline = {"kernel": ncu["kernel"] if ncu else "pvq %s kernel" % dom, "bound": "hbm", "achieved": kernels[dom]["GBps"], "peak": peak,
                 "peak_source": "%s (MEASURED_PEAKS.json hbm_gbs)" % peak_kind if peak_kind == "measured"
                 else "fallback", "unit": "GB/s", "frac": kernels[dom]["GBps"] / peak,
                 "traffic": ncu["dram_bytes"] if ncu else None,
-                "traffic_source": "ncu capture summarised under profiles/ (not this run)" if ncu else None}
-    # The limit that binds in practice: instruction issue (every kernel here is integer work
-    # on a table walk).  achieved = warp instructions per launch (from the ncu capture under
-    # profiles/, valid while the sources are unchanged) / the time measured in this run;
-    # peak = issue slots per second at the SM clock sampled during the run.
-    issue = {}
-    mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz")
-    for name in kernels:
-        c = NCU_COUNTERS.get((wl.name, name))
-        pk = SMS * SCHEDULERS_PER_SM * mhz * 1e6 if mhz else None
-        entry = {"bound": "alu", "peak": pk / 1e9 if pk else None, "unit": "Gwarp-inst/s",
-                 "peak_source": "148 SMs x 4 schedulers x sampled SM clock"}
-        if c and c.get("kernel_sha") == sha and pk:
-            ach = c["warp_inst"] / (kernels[name]["avg_ms"] * 1e-3)
-            entry.update({"achieved": ach / 1e9, "frac": ach / pk, "warp_inst_per_weight": c["warp_inst"] / wl.weights,
-                          "warp_inst_source": "ncu capture summarised under profiles/ (not this run)"})
-        else:
-            entry.update({"achieved": None, "frac": None, "warp_inst_per_weight": None,
-                          "warp_inst_source": "no capture of the current sources"})
-        issue[name] = entry
+                "traffic_source": "ncu capture %s (not this run)" % ncu["profile"] if ncu else None}
+    issue = issue_table(wl, kernels, clocks, sha)
 
     cpu = None
     if not args.no_cpu_baseline:

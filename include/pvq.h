@@ -81,7 +81,8 @@ typedef enum {
 /* bit 0 of the decode status word: some code was >= N(N,K) */
 #define PVQ_STATUS_INVALID_CODE 1u
 /* bit 1: a thread block gave up waiting for its tables to arrive in shared memory and wrote
- * nothing (a bounded wait; not expected to happen) */
+ * nothing (a bounded wait; not expected to happen).  Decoding reports it in its d_status, the
+ * encode-side calls in the word of pvq_encode_status. */
 #define PVQ_STATUS_STAGING_TIMEOUT 2u
 
 typedef void* pvq_stream_t; /* a cudaStream_t */
@@ -237,6 +238,13 @@ int pvq_encode_batched(const pvq_matrix_desc* descs, int count, int dtype, int N
                        int scale_bits, const uint32_t* d_table, pvq_stream_t stream);
 int pvq_decode_batched(const pvq_matrix_desc* descs, int count, int N, int K, int scale_bits,
                        const uint32_t* d_table, uint32_t* d_status, pvq_stream_t stream);
+
+/* Status word of the encode-side calls (pvq_encode, pvq_encode_amp, pvq_roundtrip, the rotating
+ * calls, pvq_encode_batched), which take no status argument: a device word of the caller's into
+ * which PVQ_STATUS_STAGING_TIMEOUT is OR-ed when a thread block gave up waiting for its tables
+ * (its part of the output is then not written).  Applies to the later calls of the calling
+ * thread; NULL (the default) switches reporting off.  (No counterpart in the paper.) */
+int pvq_encode_status(uint32_t* d_status);
 
 /* ---- for callers that cannot allocate device memory ---------------------------------- */
 

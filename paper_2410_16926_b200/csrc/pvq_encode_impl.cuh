@@ -456,7 +456,10 @@ __global__ void __launch_bounds__(512) encode_kernel(const __grid_constant__ Bat
         const MatrixArgs& m0 = a.m[loc.mi];
         load_raw<N, BF16>(m0.x, static_cast<size_t>(loc.row0 + loc.rl) * m0.ld + static_cast<size_t>(loc.g) * N, pre);
     }
-    if (!bulk_stage_wait(stage)) return;  // the tables never arrived: leave rather than spin
+    if (!bulk_stage_wait(stage)) {  // the tables never arrived: report and leave rather than spin
+        if (a.status && threadIdx.x == 0) atomicOr(a.status, PVQ_STATUS_STAGING_TIMEOUT);
+        return;
+    }
     __syncthreads();                      // index words cleared
 #ifdef PVQ_DEBUG
     debug_begin(tabA, tabA + sm.enc_bytes + (FUSED ? sm.walk_bytes : 0u), tabA + sm.wbuf_off, YS,

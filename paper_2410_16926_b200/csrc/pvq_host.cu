@@ -222,6 +222,15 @@ extern "C" size_t pvq_scale_row_stride(int64_t G, int scale_bits) {
     return (bytes + 3u) & ~static_cast<size_t>(3u);
 }
 
+// ------------------------------------------------------ status word of the encode-side calls
+
+static thread_local uint32_t* g_encode_status = nullptr;
+
+extern "C" int pvq_encode_status(uint32_t* d_status) {
+    g_encode_status = d_status;
+    return PVQ_OK;
+}
+
 // ------------------------------------------------------ bounds-checked build
 
 static thread_local uint32_t* g_debug_status = nullptr;
@@ -330,6 +339,7 @@ int run_batch(const pvq_matrix_desc* descs, int count, int need, int dtype, int 
     a.c_one = 1u;
     a.c_minus_one = 0xffffffffu;
     a.debug_status = g_debug_status;
+    if (kind != 1 && !a.status) a.status = g_encode_status;  // the encode-side calls take no status argument
     if (amp_mode != 0 && amp_mode != 1) return PVQ_ERR_INVALID_ARG;
     a.amp_mode = amp_mode;
     if (rot_block != 0) {

@@ -72,6 +72,7 @@ def lib():
         L.pvq_rotate_roundtrip.argtypes = [vp, i32, i64, i64, i64, i32, vp, i32, i32, i32, vp, vp, vp, vp, i64, vp]
         L.pvq_decode_static_table.argtypes = [vp, vp, vp, i64, i64, i32, i32, i32, vp, vp, i64, vp, vp]
         L.pvq_debug_status.argtypes = [vp]
+        L.pvq_encode_status.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -80,7 +81,7 @@ EXPORTS = ["pvq_strerror", "pvq_last_cuda_error", "pvq_index_bits", "pvq_max_pul
            "pvq_count_table_bytes", "pvq_scale_row_stride", "pvq_build_count_table",
            "pvq_build_scale_codebook", "pvq_encode", "pvq_decode", "pvq_roundtrip", "pvq_encode_batched",
            "pvq_decode_batched", "pvq_decode_static_table", "pvq_rotate_encode", "pvq_rotate_roundtrip", "pvq_encode_amp",
-           "pvq_debug_status"]
+           "pvq_debug_status", "pvq_encode_status"]
 
 
 def _check(status, where):
@@ -110,6 +111,12 @@ def _dtype_code(x):
     if x.dtype == torch.bfloat16:
         return DTYPE_BF16
     raise TypeError("input must be float32 or bfloat16")
+
+
+def encode_status(word):
+    """The status word of the encode-side calls of this thread (an int32 device tensor of one
+    element, or None): a staging time-out is reported there."""
+    _check(lib().pvq_encode_status(_ptr(word, torch.int32)), "pvq_encode_status")
 
 
 def debug_status(word):

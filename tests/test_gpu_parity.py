@@ -234,6 +234,25 @@ def test_encode_decode_parity(N, bits, rows, cols, b, kind):
     check_decode(cd, enc_dev, enc_np)
 
 
+def test_encode_status_word_stays_clear():
+    # the encode-side calls report a staging time-out in the word of pvq_encode_status; on a
+    # healthy run it stays zero and the results are those of a run without it
+    rng = np.random.default_rng(77)
+    x_np = inputs.f32_to_bf16_bits((rng.standard_normal((19, 2048)) * 0.02).astype(np.float32))
+    cd = Codec(32, 96, 64, 4)
+    word = torch.zeros(1, dtype=torch.int32, device=DEV)
+    pvq.encode_status(word)
+    try:
+        check_encode(cd, x_np, "bf16")
+        out = pvq.roundtrip(to_device(x_np, "bf16"), cd.N, cd.K, cd.b, cd.table, cd.edges, cd.levels)
+        torch.cuda.synchronize()
+    finally:
+        pvq.encode_status(None)
+    assert int(word.item()) == 0
+    enc = po.encode(x_np, cd.N, cd.K, cd.b, cd.edges_np, W=cd.W)
+    assert np.array_equal(bf16_bits(out), po.decode(*enc, cd.N, cd.K, cd.b, cd.levels_np)[0])
+
+
 def test_heavy_tails_and_outliers():
     rng = np.random.default_rng(42)
     x = (rng.standard_t(2.0, size=(24, 1024)) * 0.05).astype(np.float32)
