@@ -50,7 +50,16 @@
  *                        the encoder's tables, rows by position, K+2 entries per row for
  *                        k = -1..K, of the cumulative counts V(n,k) = sum_{j<=k} N(n,j)
  *                        (App. C.2) modulo 2^(32 W): V(n,k) + V(n,k-1), then 2 V(n,k),
- *                        then V(n,k).
+ *                        then V(n,k);
+ *                        for N <= 64 and W <= 6: the decoder's widest table as doubles
+ *                        (values from 2^53 up replaced by 2^53), V(N-1,K) + V(N-1,K-1), and,
+ *                        where they fit, the encoder's tables in telescoped form (one read
+ *                        per position);
+ *                        for W <= 4 and K <= 127, where it fits shared memory: the tables
+ *                        of the decoder that finds each coordinate by one threshold
+ *                        search (a 16-byte header with N and K, one 16-byte record per
+ *                        row, the rows' bucket tables, the thresholds and the
+ *                        increments of the running value).
  *                      Callers treat everything after the first section as opaque.
  *   edges      float   2^b - 1 ascending bin edges of u.
  *   levels     float   2^b values sqrt(PPF((q + 1/2) / 2^b)): the factor that
@@ -84,6 +93,9 @@ typedef enum {
  * nothing (a bounded wait; not expected to happen).  Decoding reports it in its d_status, the
  * encode-side calls in the word of pvq_encode_status. */
 #define PVQ_STATUS_STAGING_TIMEOUT 2u
+/* bit 2 of the decode status word: the table given to the call was not built for this (N,K)
+ * (its header says so); nothing was decoded. */
+#define PVQ_STATUS_TABLE_MISMATCH 4u
 
 typedef void* pvq_stream_t; /* a cudaStream_t */
 

@@ -186,6 +186,15 @@ int launch_decode_n(BatchArgs& a, int W, cudaStream_t stream) {
 }  // namespace
 
 int launch_decode(const BatchArgs& args, int N, int W, cudaStream_t stream) {
+    // codes of up to four words and 127 pulses: one threshold search per position, where
+    // the tables for it are part of the blob; everything else walks
+    if (W <= 4 && args.K <= 127) {
+        const SearchLayout& S = search_layout_for(N, args.K);
+        if (S.present) {
+            const int st = launch_decode_search(args, N, W, S, stream);
+            if (st != PVQ_ERR_UNSUPPORTED) return st;
+        }
+    }
     BatchArgs a = args;
     switch (N) {
         case 8: return launch_decode_n<8, 2>(a, W, stream);

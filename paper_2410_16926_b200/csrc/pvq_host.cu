@@ -155,6 +155,99 @@ int code_words_for(int N, int K) {
     return W;
 }
 
+// The leading 24 bits of v >= 1 as the bits of an fp32 (what search_key computes on the device).
+static uint32_t key_bits(const BigU& v) {
+    const int e = v.bit_length() - 1;
+    uint32_t mant = 0;  // bits e .. e-23 of v
+    for (int b = 0; b < 24; ++b) {
+        const int pos = e - b;
+        const uint32_t bit = pos >= 0 ? (v.w[pos >> 5] >> (pos & 31)) & 1u : 0u;
+        mant = (mant << 1) | bit;
+    }
+    return (static_cast<uint32_t>(e + 127) << 23) | (mant & 0x7fffffu);
+}
+
+// Layout of the search section (SearchLayout): the thresholds of every row are computed
+// exactly, and each row gets the smallest number of key bits that puts every threshold in a
+// bucket of its own.
+const SearchLayout& search_layout_for(int N, int K) {
+    static std::mutex mu;
+    static std::map<std::pair<int, int>, SearchLayout> memo;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find({N, K});
+    if (it != memo.end()) return it->second;
+    SearchLayout& S = memo[{N, K}];
+    std::memset(&S, 0, sizeof S);
+    int W = 0;
+    {
+        const int bits = index_bits_exact(N, K);
+        W = bits < 0 ? 0 : std::max(1, (bits + 31) / 32);
+    }
+    if (W < 1 || W > 4 || K > 127 || K < 1 || N > kSearchMaxRows || N < 2) return S;
+    // keys of T_n[m], m = 0..2K, n = 0..N-1
+    const int M = 2 * K + 1;
+    std::vector<uint32_t> keys(static_cast<size_t>(N) * M);
+    std::vector<int> need(static_cast<size_t>(N));  // words that hold the row's largest threshold, N(n+1,K)
+    {
+        CountColumn c(N);  // col[n] = N(n,k)
+        std::vector<BigU> V(static_cast<size_t>(N)), Vprev(static_cast<size_t>(N));
+        for (int k = 0; k <= K; ++k) {
+            if (k > 0 && !c.advance()) return S;
+            for (int n = 0; n < N; ++n) {
+                Vprev[n] = V[n];
+                V[n].add(c.col[static_cast<size_t>(n)]);
+                BigU u = V[n], v2 = V[n];
+                u.add(Vprev[n]);
+                v2.add(V[n]);
+                keys[static_cast<size_t>(n) * M + 2 * k] = key_bits(u);
+                if (k < K) keys[static_cast<size_t>(n) * M + 2 * k + 1] = key_bits(v2);
+                if (k == K) need[n] = std::max(1, (u.bit_length() + 31) / 32);
+            }
+        }
+        // N(N,K) = U(N-1,K) must stay below 2^(32 W): q = N(N,K) - code is computed in W words
+        BigU top = V[N - 1];
+        top.add(Vprev[N - 1]);
+        if (top.bit_length() > 32 * W) return S;
+    }
+    const uint32_t key_one = 0x3f800000u;
+    uint32_t boff = 0;
+    for (int n = 0; n < N; ++n) {
+        const uint32_t* kr = keys.data() + static_cast<size_t>(n) * M;
+        const int last = n == 0 ? 1 : M - 1;  // row 0 (no dimension left) has the thresholds 1 and 2 only
+        int sh = -1;
+        for (int f = 0; f <= 23 && sh < 0; ++f) {
+            const int s = 23 - f;
+            bool distinct = true;
+            for (int m = 1; m <= last && distinct; ++m) distinct = (kr[m] >> s) != (kr[m - 1] >> s);
+            if (distinct) sh = s;
+        }
+        if (sh < 0) return S;
+        S.rows.shift[n] = static_cast<uint8_t>(sh);
+        S.rows.b_off[n] = boff;
+        S.rows.b_len[n] = (kr[last] >> sh) - (key_one >> sh) + 1u;
+        boff += S.rows.b_len[n];
+    }
+    if (N % 4 != 0) return S;
+    uint32_t teoff = 0;
+    for (int n = N - 1; n >= 0; --n) {  // a block of four rows takes the width of its top row
+        const int w = need[static_cast<size_t>(n | 3)];
+        S.rows.words[n] = static_cast<uint8_t>(w);
+        S.count[w] += 1;
+        S.rows.te_off[n] = teoff;
+        teoff += static_cast<uint32_t>(2 * K + 2) * search_entry_words(w) * 4u;
+    }
+    S.rec_off = kSearchHeader;
+    S.b_off = S.rec_off + static_cast<uint32_t>(N) * 16u;
+    S.t_off = (S.b_off + boff + 15u) & ~15u;
+    S.te_bytes = (teoff + 15u) & ~15u;
+    S.e_off = S.t_off + S.te_bytes;
+    S.total = (S.e_off + S.te_bytes + 127u) & ~127u;
+    if (S.total > kSearchLimit) return S;
+    S.off = (table_layout(N, K, W).total + 127u) & ~127u;
+    S.present = true;
+    return S;
+}
+
 }  // namespace pvq
 
 using namespace pvq;
@@ -213,7 +306,8 @@ extern "C" int pvq_code_words(int N, int K, int* W_out) {
 extern "C" size_t pvq_count_table_bytes(int N, int K) {
     int W = code_words_for(N, K);
     if (W == 0 || N < 1 || K < 1) return 0;
-    return table_layout(N, K, W).total;
+    const SearchLayout& S = search_layout_for(N, K);
+    return S.present ? static_cast<size_t>(S.off) + S.total : table_layout(N, K, W).total;
 }
 
 extern "C" size_t pvq_scale_row_stride(int64_t G, int scale_bits) {

@@ -53,6 +53,8 @@ struct BatchArgs {
     const float* rot_signs;  // +-1, rot_block of them
     int rot_block;           // power of two, a multiple of N, dividing every cols
     uint32_t* debug_status;  // bounds-checked build: where violations are reported (pvq_debug_status); else null
+    // decode by threshold search (SearchLayout): the section's place in the blob and its bytes
+    uint32_t srch_off, srch_bytes;
 };
 
 // Layout of the table blob.  Section 0 is the count table as the paper defines it,
@@ -176,9 +178,67 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
     return L;
 }
 
+// ---- tables of the decoder that searches (csrc/pvq_decode_search.cu) ------------------------
+//
+// With q = N(n+1,k) - r (r the part of the code not yet explained, n dimensions after the
+// current position, k pulses left) the coordinate of Algorithm 3 follows from where q falls
+// among the thresholds of row n,
+//     T_n[2k'] = U(n,k') = V(n,k') + V(n,k'-1),    T_n[2k'+1] = 2 V(n,k'),    k' = 0..K
+// (V(n,k) = sum_{j<=k} N(n,j), App. C.2): with m the first index whose threshold is >= q,
+// k' = m >> 1 pulses remain after the position, |y| = k - k', y > 0 iff m is odd, and the q of
+// the next position is q + E_n[m], E_n[m] = U(n-1,k') - T_n[m] (the encoder's telescoped
+// tables).  m is found without a loop: a key of q (its leading 24 bits as an fp32, see
+// search_key) shifted right by a per-row amount numbers a bucket, the row's byte table gives
+// the first threshold index that can be right for that bucket, and the shift is chosen
+// (on the host, from the exact thresholds) so that no two thresholds of a row share a
+// bucket: one multi-word compare with that threshold settles m.
+//
+// Values shrink from row to row (q <= N(n+1,K) at row n), so the rows are narrower towards
+// the end of the vector: a row's thresholds and increments are stored, and its arithmetic is
+// done, in the fewest words that hold N(n+1,K); rows are classed in aligned blocks of four
+// (a block takes the width of its top row), so that the decoder works through four
+// positions at a time in one width.
+//
+// The section follows the sections of TableLayout in the blob (128-byte aligned) and is
+// staged as one piece:
+//     header    32 bytes: magic, N, K, bytes of the section, then the number of rows whose
+//               arithmetic is done in 4, 3, 2 and 1 words (the widest rows are the top ones)
+//     records   one 16-byte record per row n: byte offsets (from the section's start) of the
+//               row of T, of the row of E, of the row's bucket table minus its first bucket
+//               number, and the shift
+//     buckets   the rows' byte tables, one after the other
+//     T, E      rows of 2K+2 entries (thresholds m = 0..2K; E modulo 2^(32 words)) of 1, 2 or
+//               4 words (three-word rows use four-word entries)
+constexpr int kSearchMaxRows = 64;
+constexpr uint32_t kSearchMagic = 0x53515650u;
+constexpr uint32_t kSearchHeader = 32u;
+constexpr uint32_t kSearchLimit = 184u * 1024u;  // the section has to leave room for the output slots
+
+__host__ __device__ constexpr int search_entry_words(int words) { return words == 3 ? 4 : words; }
+
+struct SearchRows {  // what the builder needs per row
+    uint32_t b_off[kSearchMaxRows];   // of the row's bucket table inside `buckets`
+    uint32_t b_len[kSearchMaxRows];   // its entries
+    uint32_t te_off[kSearchMaxRows];  // of the row inside T (and inside E)
+    uint8_t shift[kSearchMaxRows];    // bucket number = (key >> shift) - (key(1) >> shift)
+    uint8_t words[kSearchMaxRows];    // words the row's arithmetic is done in
+};
+
+struct SearchLayout {
+    bool present;
+    int count[5];         // count[w]: rows done in w words
+    uint32_t off;         // of the section in the blob
+    uint32_t rec_off, b_off, t_off, e_off;  // of its parts, from the section's start
+    uint32_t te_bytes;    // of T, and of E
+    uint32_t total;       // bytes of the section (a multiple of 128)
+    SearchRows rows;
+};
+
 // host helpers (pvq_host.cu)
 int set_cuda_error(cudaError_t e);  // records e, returns PVQ_ERR_CUDA
 int code_words_for(int N, int K);   // W, or 0 when it cannot be computed
+// the search section for (N,K), memoised; present == false where the decoder walks instead
+const SearchLayout& search_layout_for(int N, int K);
 bool is_aligned(const void* p, size_t a);
 
 // What a launcher needs to know about the current device and a kernel at a given block size
@@ -193,6 +253,7 @@ int prepare_kernel(const void* kern, int threads, size_t smem, int* blocks_per_s
 
 // launchers (one per kernel family); all return a pvq_status
 int launch_decode(const BatchArgs& args, int N, int W, cudaStream_t stream);
+int launch_decode_search(const BatchArgs& args, int N, int W, const SearchLayout& S, cudaStream_t stream);
 // large groups / wide codes (N = 128 or more than 6 words): tables in global memory
 int launch_big(const BatchArgs& args, int dtype, int N, int W, bool decode, cudaStream_t stream);  // args.fused: round trip
 int launch_encode(const BatchArgs& args, int dtype, int N, int W, bool fused, cudaStream_t stream);  // rotates when args.rot_block != 0
@@ -243,6 +304,7 @@ __device__ __forceinline__ int find_matrix(const BatchArgs& a, unsigned tile) {
 struct DebugCtx {
     uint32_t tab_lo, tab_hi;                      // shared addresses: the staged tables
     uint32_t slot_base, slot_stride, slot_bytes;  // output slots: thread t owns [base + t * stride, + bytes)
+    uint32_t slot_chain, slot_end;                // ... and the same range every slot_chain bytes up to slot_end (0: no)
     uint32_t* status;
 };
 __shared__ DebugCtx s_debug;
@@ -256,6 +318,7 @@ __device__ __forceinline__ void debug_begin(uint32_t tab_lo, uint32_t tab_hi, ui
         s_debug.slot_base = slot_base;
         s_debug.slot_stride = slot_stride;
         s_debug.slot_bytes = slot_bytes;
+        s_debug.slot_chain = s_debug.slot_end = 0u;
         s_debug.status = status;
     }
     __syncthreads();
@@ -270,7 +333,11 @@ __device__ __forceinline__ bool debug_table_ok(uint32_t addr, uint32_t bytes) {
 }
 __device__ __forceinline__ bool debug_slot_ok(uint32_t addr, uint32_t bytes) {
     const uint32_t lo = s_debug.slot_base + threadIdx.x * s_debug.slot_stride;
-    const bool ok = addr >= lo && addr + bytes <= lo + s_debug.slot_bytes;
+    bool ok = addr >= lo;
+    if (s_debug.slot_chain != 0u)
+        ok = ok && (addr - lo) % s_debug.slot_chain + bytes <= s_debug.slot_bytes && addr + bytes <= s_debug.slot_end;
+    else
+        ok = ok && addr + bytes <= lo + s_debug.slot_bytes;
     if (!ok) debug_flag(PVQ_DEBUG_SLOT_WRITE);
     return ok;
 }

@@ -3,6 +3,7 @@
 // or per (N,G,b).
 #include "mp_uint.cuh"
 #include "pvq_internal.cuh"
+#include "pvq_search.cuh"
 
 namespace pvq {
 
@@ -274,6 +275,79 @@ __global__ void derive_fast_tables_kernel(int N, int K, int Wc, uint32_t* __rest
     }
 }
 
+// The search section (SearchLayout), block n = row n, thread m = threshold m.  Runs after
+// derive_tables_kernel: thresholds and increments come from the cumulative tables U and 2V.
+// The bucket table of a row holds, for every bucket, how many thresholds lie in earlier
+// buckets: thread m writes its index into the buckets after that of threshold m-1 up to
+// its own.
+__global__ void __launch_bounds__(256) derive_search_tables_kernel(int N, int K, int Wc, uint32_t* __restrict__ blob,
+                                                                   const __grid_constant__ SearchLayout S) {
+    __shared__ uint32_t bucket_of[256];
+    const TableLayout L = table_layout(N, K, Wc);
+    const int TW = L.top_words;  // words per entry of the cumulative tables
+    const int n = blockIdx.x, m = threadIdx.x;
+    const int i = N - 1 - n;     // the position whose row of the cumulative tables this is
+    const int k = m >> 1;
+    const int last = n == 0 ? 1 : 2 * K;  // thresholds of the row: 0..last
+    const int RW = S.rows.words[n];       // words of this row's arithmetic
+    const int EW = search_entry_words(RW);
+    uint8_t* sec = reinterpret_cast<uint8_t*>(blob) + S.off;
+    const uint32_t* U = blob + L.enc_off[0] / 4;   // (i, col + 1), K + 2 entries a row
+    const uint32_t* V2 = blob + L.enc_off[1] / 4;
+    uint32_t t[4] = {0u, 0u, 0u, 0u};
+    if (m <= 2 * K) {
+        const uint32_t* src = ((m & 1) ? V2 : U) + (static_cast<size_t>(i) * (K + 2) + k + 1) * TW;
+        for (int w = 0; w < Wc; ++w) t[w] = src[w];
+    }
+    if (m < 2 * K + 2) {
+        const size_t at = (S.rows.te_off[n] + static_cast<size_t>(m) * EW * 4u) / 4u;
+        uint32_t* T = reinterpret_cast<uint32_t*>(sec + S.t_off) + at;
+        uint32_t* E = reinterpret_cast<uint32_t*>(sec + S.e_off) + at;
+        // E = U(n-1, k) - T, modulo 2^(32 RW); U(-1, .) = 0
+        const uint32_t* un = U + (static_cast<size_t>(i + 1) * (K + 2) + k + 1) * TW;
+        long long borrow = 0;
+        for (int w = 0; w < EW; ++w) {
+            const long long a = (n >= 1 && w < Wc && m <= 2 * K) ? static_cast<long long>(un[w]) : 0;
+            const long long d = a - static_cast<long long>(w < Wc ? t[w] : 0u) + borrow;
+            borrow = d >> 32;  // 0 or -1
+            T[w] = w < RW ? t[w] : 0u;
+            E[w] = w < RW ? static_cast<uint32_t>(d) : 0u;
+        }
+    }
+    const uint32_t sh = S.rows.shift[n];
+    bucket_of[m] = m <= last ? (search_key(t, Wc) >> sh) - (kSearchKeyOfOne >> sh) : 0u;
+    __syncthreads();
+    if (m <= last) {
+        uint8_t* B = sec + S.b_off + S.rows.b_off[n];
+        const uint32_t hi = bucket_of[m];
+        const uint32_t lo = m == 0 ? 0u : bucket_of[m - 1] + 1u;
+        for (uint32_t b = lo; b <= hi && b < S.rows.b_len[n]; ++b) B[b] = static_cast<uint8_t>(m);
+    }
+    if (m == 0) {
+        uint32_t* rec = reinterpret_cast<uint32_t*>(sec + S.rec_off) + 4 * n;
+        rec[0] = S.t_off + S.rows.te_off[n];
+        rec[1] = S.e_off + S.rows.te_off[n];
+        rec[2] = S.b_off + S.rows.b_off[n] - (kSearchKeyOfOne >> sh);
+        rec[3] = sh;
+        if (n == 0) {
+            uint32_t* head = reinterpret_cast<uint32_t*>(sec);
+            head[0] = kSearchMagic;
+            head[1] = static_cast<uint32_t>(N);
+            head[2] = static_cast<uint32_t>(K);
+            head[3] = S.total;
+            for (int w = 4; w >= 1; --w) head[8 - w] = static_cast<uint32_t>(S.count[w]);
+        }
+    }
+}
+
+static int launch_search_tables(int N, int K, int Wc, uint32_t* d_table, cudaStream_t s) {
+    const SearchLayout& S = search_layout_for(N, K);
+    if (!S.present) return PVQ_OK;
+    derive_search_tables_kernel<<<N, 256, 0, s>>>(N, K, Wc, d_table, S);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
+}
+
 template <int W>
 static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStream_t s) {
     const int threads = ((K + 1 + 31) / 32) * 32;
@@ -294,7 +368,8 @@ static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStrea
         derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table);
         if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
         derive_fast_tables_kernel<<<16, 256, 0, s>>>(N, K, Wc, d_table);
-        e = cudaGetLastError();
+        if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
+        return launch_search_tables(N, K, Wc, d_table, s);
     }
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }

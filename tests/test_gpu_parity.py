@@ -9,6 +9,8 @@ from oracle import beta_codebook as bc
 from oracle import pvq_oracle as po
 from paper_2410_16926_b200 import inputs, pvq
 
+import blob_sections as bs
+
 pytestmark = pytest.mark.gpu
 
 DEV = "cuda"
@@ -100,36 +102,6 @@ def test_count_table_word_for_word(N, K):
     assert np.array_equal(as_u32(pvq.count_table_view(t, N, K)), ref)
 
 
-def _blob_layout(N, K, W):
-    """Byte offsets of the sections that follow the count table (see include/pvq.h)."""
-    up = lambda v: (v + 127) & ~127
-    rowlen = (K + 2) & ~1
-    top = W if W <= 2 else (4 if W <= 4 else (6 if W <= 6 else (8 if W <= 8 else (12 if W <= 12 else (W + 3) & ~3))))
-    bound_words = 16 if W <= 12 else 64
-    off = up(N * (K + 1) * W * 4)
-    lay = {"bound": off, "bound_words": bound_words, "rowlen": rowlen, "top": top}
-    off += up(bound_words * 4)
-    for name, words in (("walk_top", top), ("walk2", 2 if top > 2 else 0), ("walk1", 1 if top > 1 else 0)):
-        lay[name] = (off, words)
-        off += up(N * rowlen * words * 4)
-    for name in ("enc_u", "enc_2v", "enc_v"):
-        lay[name] = off
-        off += up(N * (K + 2) * top * 4)
-    lay["walkd"] = lay["start"] = lay["cenc0"] = lay["cenc1"] = None
-    if N <= 64 and W <= 6:            # the sections of the shared-memory kernels
-        lay["walkd"] = off
-        off += up(N * rowlen * 8)
-        lay["start"] = off
-        off += 128
-        crow = 32 if K + 1 <= 32 else (64 if K + 1 <= 64 else 128)
-        cb = N * crow * top * 4
-        if W <= 4 and K + 1 <= 128 and 2 * cb <= 160 * 1024:
-            lay["cenc0"], lay["cenc1"], lay["crow"] = off, off + cb, crow
-            off += 2 * cb
-    lay["total"] = off
-    return lay
-
-
 @pytest.mark.parametrize("N,K", [(8, 16), (16, 18), (32, 22), (32, 50), (32, 105), (64, 96), (64, 26), (128, 40),
                                  (64, 230), (128, 300), (256, 200)])
 def test_table_blob_sections(N, K):
@@ -137,10 +109,12 @@ def test_table_blob_sections(N, K):
     W = pvq.code_words(N, K)
     blob = as_u32(pvq.build_count_table(N, K))
     torch.cuda.synchronize()
-    lay = _blob_layout(N, K, W)
-    assert blob.size * 4 == lay["total"] == pvq.count_table_bytes(N, K)
-    full = po.count_table(N, K, W)                      # rows n = 0..N
+    lay = bs.blob_layout(N, K, W)
+    full = po.count_table(N, K, W + 1)                  # rows n = 0..N
     val = [[po.code_to_int(full[n, k]) for k in range(K + 1)] for n in range(N + 1)]
+    srch = bs.section(val, N, K, W, lay["total"])
+    want_bytes = lay["total"] if srch is None else srch["off"] + srch["total"]
+    assert blob.size * 4 == want_bytes == pvq.count_table_bytes(N, K)
     mask = (1 << (32 * W)) - 1
     words = lambda v, nw: [(v >> (32 * w)) & 0xFFFFFFFF for w in range(nw)]
     bwn = lay["bound_words"]
@@ -188,6 +162,23 @@ def test_table_blob_sections(N, K):
                 for k in range(K + 1):
                     sub = U(n, k) if name == "cenc0" else 2 * sum(val[n][:k + 1])
                     assert list(sec[i, k]) == words((U(n - 1, k) - sub) & mask, top), (name, i, k)
+    if srch is not None:
+        # the decoder's search section: header, row records, bucket tables, thresholds, increments
+        sec = blob[srch["off"] // 4: (srch["off"] + srch["total"]) // 4]
+        assert list(sec[:8]) == [bs.MAGIC, N, K, srch["total"]] + srch["counts"]
+        raw = sec.view(np.uint8)
+        for n in range(N):
+            rec = sec[(srch["rec_off"] + 16 * n) // 4: (srch["rec_off"] + 16 * n) // 4 + 4]
+            sh, ew, at = srch["shifts"][n], srch["ewords"][n], srch["te_offs"][n]
+            want = [srch["t_off"] + at, srch["e_off"] + at,
+                    (srch["b_off"] + srch["offs"][n] - (bs.KEY_OF_ONE >> sh)) & 0xFFFFFFFF, sh]
+            assert list(rec) == want, ("record", n)
+            b0 = srch["b_off"] + srch["offs"][n]
+            assert list(raw[b0: b0 + srch["lens"][n]]) == srch["tables"][n], ("buckets", n)
+            for name, vals in (("t_off", srch["T"]), ("e_off", srch["E"])):
+                row = sec[(srch[name] + at) // 4: (srch[name] + at) // 4 + (2 * K + 2) * ew].reshape(2 * K + 2, ew)
+                for m in range(2 * K + 1):
+                    assert list(row[m]) == words(vals[n][m], ew), (name, n, m)
 
 
 @pytest.mark.parametrize("N,G,b", [(32, 16, 8), (32, 128, 4), (32, 448, 8), (64, 448, 6), (32, 128, 8),

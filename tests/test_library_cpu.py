@@ -45,6 +45,59 @@ def test_pulse_selection_matches_oracle(N, bits):
     assert pvq.count_table_bytes(N, K) >= N * (K + 1) * W * 4      # the count table is the blob's first section
 
 
+@pytest.mark.parametrize("N,K", [(8, 6), (8, 40), (16, 18), (16, 40), (32, 22), (32, 30), (32, 50), (32, 105),
+                                 (32, 127), (64, 26), (64, 31), (64, 96), (128, 40), (32, 1), (16, 127)])
+def test_blob_size_counts_the_search_section(N, K):
+    """The host lays out the search section from exact thresholds: its size is the one a plain
+    Python computation from the oracle's count table gives (shifts, bucket-table lengths)."""
+    import blob_sections as bs
+    from oracle import pvq_pyref as pr
+    W = pvq.code_words(N, K)
+    lay = bs.blob_layout(N, K, W)
+    srch = bs.section(pr.count_table(N, K), N, K, W, lay["total"])
+    want = lay["total"] if srch is None else srch["off"] + srch["total"]
+    assert pvq.count_table_bytes(N, K) == want
+    if (N, K) in ((32, 50), (32, 22), (16, 18), (64, 31)):
+        assert srch is not None
+    if (N, K) in ((64, 96), (128, 40), (32, 127)):
+        assert srch is None
+
+
+@pytest.mark.parametrize("N,K", [(4, 3), (4, 5), (4, 8), (8, 3)])
+def test_search_recipe_is_algorithm_3_exhaustively(N, K):
+    """Decoding by one threshold search per position (the tables of the blob's search section,
+    here built in Python) gives the point of Algorithm 3 for every code of small pyramids."""
+    import blob_sections as bs
+    from oracle import pvq_pyref as pr
+    count = pr.count_table(N, K)
+    sec = bs.section(count, N, K, 1, 0)
+    assert sec is not None
+    for code in range(count[N][K]):
+        y, ok = pr.deenumerate_code(code, N, K)
+        assert ok and bs.decode_with(sec, count, code, N, K) == y
+
+
+@pytest.mark.parametrize("N,K,W", [(32, 50, 3), (32, 22, 2), (16, 40, 2), (8, 60, 2), (64, 31, 4)])
+def test_search_recipe_is_algorithm_3_on_random_codes(N, K, W):
+    import random
+    import blob_sections as bs
+    from oracle import pvq_pyref as pr
+    count = pr.count_table(N, K)
+    sec = bs.section(count, N, K, W, 0)
+    assert sec is not None
+    rnd = random.Random(N * 1000 + K)
+    total = count[N][K]
+    for code in [0, 1, total - 1, total // 2] + [rnd.randrange(total) for _ in range(200)]:
+        y, ok = pr.deenumerate_code(code, N, K)
+        assert ok and bs.decode_with(sec, count, code, N, K) == y
+    # the most lopsided points: all pulses on one coordinate, either sign
+    for pos in (0, N // 2, N - 1):
+        for sign in (1, -1):
+            y = [0] * N
+            y[pos] = sign * K
+            assert bs.decode_with(sec, count, pr.enumerate_point(y, K), N, K) == y
+
+
 def test_index_bits_small_cases():
     # N(2,7) = 28 -> 5 bits; N(1,k) = 2 -> 1 bit; N(n,0) = 1 -> 0 bits
     assert pvq.index_bits(2, 7) == 5
