@@ -43,15 +43,9 @@ __device__ __forceinline__ uint4 load_record(uint32_t addr) {
 __device__ __forceinline__ uint32_t load_bucket(uint32_t addr) {
     uint32_t v;
 #ifdef PVQ_DEBUG
-    {
-        const bool ok = addr >= s_debug.tab_lo && addr < s_debug.tab_hi;
-        if (!ok) {
-            debug_flag(PVQ_DEBUG_TABLE_READ);
-            return 0u;
-        }
-    }
+    if (!debug_table_ok(addr, 4)) return 0u;
 #endif
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
 
@@ -112,9 +106,14 @@ __device__ __forceinline__ void store_y4(uint32_t addr, uint32_t val) {
 // `rec` is the shared address of the record of the first of the four rows (the rows of the
 // following positions have the records before it); a record is read once for all chains.
 // The four y_i + 128 of chain j go to the word at y + j * ychain.
+//
+// Per position: the key of q selects a bucket; its entry is m0 and the low key bits of the
+// threshold T[m0]; q's own low key bits being larger means q > T[m0], smaller means q <= T[m0]
+// (a bucket without a threshold holds all ones there).  Equal bits leave it open: then, and
+// that is rare, the threads of the warp whose bits were equal compare q with T[m0] in full.
 template <int W, int PW, int GP>
-__device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP], uint32_t rec, uint32_t y,
-                                              uint32_t ychain) {
+__device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP], uint32_t rec, uint32_t t_before_e,
+                                              uint32_t y, uint32_t ychain) {
     constexpr int EB = search_entry_words(PW) * 4;  // bytes of an entry of T and E
     uint32_t acc[GP];
     mp<PW> v[GP];  // the low PW words of q: the rest is zero by now
@@ -126,15 +125,29 @@ __device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP],
     }
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
-        const uint4 r = load_record(rec - static_cast<uint32_t>(s) * 16u);
-        uint32_t m0[GP], m[GP];
-        mp<PW> t[GP], e[GP];
+        const uint4 r = load_record(rec - static_cast<uint32_t>(s) * 16u);  // 32 - shift, E row, buckets, shift
+        uint32_t key[GP], entry[GP], m[GP];
+        mp<PW> e[GP];
+        bool open = false;
 #pragma unroll
-        for (int j = 0; j < GP; ++j) m0[j] = load_bucket(r.z + (search_key<PW>(v[j].w) >> r.w));
+        for (int j = 0; j < GP; ++j) {
+            key[j] = search_key<PW>(v[j].w);
+            entry[j] = load_bucket(r.z + ((key[j] >> r.w) << 2));
+        }
 #pragma unroll
-        for (int j = 0; j < GP; ++j) t[j] = load_entry<PW>(r.x + m0[j] * EB);
+        for (int j = 0; j < GP; ++j) {
+            const uint32_t x = key[j] << r.x;  // the key bits below the shift, left-aligned like the entry's
+            m[j] = (entry[j] & 0xffu) + (x > entry[j] ? 1u : 0u);
+            open = open || (entry[j] - x < 256u);
+        }
+        if (__any_sync(kFull, open)) {
 #pragma unroll
-        for (int j = 0; j < GP; ++j) m[j] = bump_if_less<PW>(m0[j], t[j], v[j]);
+            for (int j = 0; j < GP; ++j) {
+                const uint32_t m0 = entry[j] & 0xffu;
+                if (entry[j] - (key[j] << r.x) < 256u)
+                    m[j] = bump_if_less<PW>(m0, load_entry<PW>(r.y - t_before_e + m0 * EB), v[j]);
+            }
+        }
 #pragma unroll
         for (int j = 0; j < GP; ++j) e[j] = load_entry<PW>(r.y + m[j] * EB);
 #pragma unroll
@@ -158,26 +171,26 @@ __device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP],
 // The points of GP codes: q = N(N,K) - code on entry.  `recs` is the shared address of the
 // row records (absolute shared addresses by now), cnt[w] the number of rows done in w words.
 template <int N, int W, int GP>
-__device__ __forceinline__ void search_codes(mp<W> (&q)[GP], int K, uint32_t recs, const int (&cnt)[5], uint32_t y,
-                                             uint32_t ychain) {
+__device__ __forceinline__ void search_codes(mp<W> (&q)[GP], int K, uint32_t recs, uint32_t t_before_e,
+                                             const int (&cnt)[5], uint32_t y, uint32_t ychain) {
     uint32_t k[GP];
 #pragma unroll
     for (int j = 0; j < GP; ++j) k[j] = static_cast<uint32_t>(K);
     uint32_t rec = recs + static_cast<uint32_t>(N - 1) * 16u;
     if constexpr (W >= 4) {
 #pragma unroll 1
-        for (int b = 0; b < cnt[4]; b += 4, rec -= 64u, y += 4u) search_block4<W, 4, GP>(q, k, rec, y, ychain);
+        for (int b = 0; b < cnt[4]; b += 4, rec -= 64u, y += 4u) search_block4<W, 4, GP>(q, k, rec, t_before_e, y, ychain);
     }
     if constexpr (W >= 3) {
 #pragma unroll 1
-        for (int b = 0; b < cnt[3]; b += 4, rec -= 64u, y += 4u) search_block4<W, 3, GP>(q, k, rec, y, ychain);
+        for (int b = 0; b < cnt[3]; b += 4, rec -= 64u, y += 4u) search_block4<W, 3, GP>(q, k, rec, t_before_e, y, ychain);
     }
     if constexpr (W >= 2) {
 #pragma unroll 1
-        for (int b = 0; b < cnt[2]; b += 4, rec -= 64u, y += 4u) search_block4<W, 2, GP>(q, k, rec, y, ychain);
+        for (int b = 0; b < cnt[2]; b += 4, rec -= 64u, y += 4u) search_block4<W, 2, GP>(q, k, rec, t_before_e, y, ychain);
     }
 #pragma unroll 1
-    for (int b = 0; b < cnt[1]; b += 4, rec -= 64u, y += 4u) search_block4<W, 1, GP>(q, k, rec, y, ychain);
+    for (int b = 0; b < cnt[1]; b += 4, rec -= 64u, y += 4u) search_block4<W, 1, GP>(q, k, rec, t_before_e, y, ychain);
 }
 
 // GP groups per thread: a warp takes GP consecutive tiles of 32 groups in one pass.
@@ -233,7 +246,6 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
     }
     if (threadIdx.x < N) {  // the records' offsets become shared addresses
         uint32_t* rec = reinterpret_cast<uint32_t*>(smem + kSearchHeader) + 4 * threadIdx.x;
-        rec[0] += sbase;
         rec[1] += sbase;
         rec[2] += sbase;
     }
@@ -308,7 +320,7 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
             }
             mp_sub_borrow<W>(q[j], bound, c);  // 1 <= q <= N(N,K)
         }
-        search_codes<N, W, GP>(q, K, recs, cnt, shared_addr(yslots), ychain);
+        search_codes<N, W, GP>(q, K, recs, a.srch_t_before_e, cnt, shared_addr(yslots), ychain);
 #pragma unroll
         for (int j = 0; j < GP; ++j)
             if (active[j])
@@ -331,6 +343,7 @@ int launch_search_t(BatchArgs& a, const SearchLayout& S, cudaStream_t stream) {
     a.total_tiles = tiles;
     a.srch_off = S.off;
     a.srch_bytes = S.total;
+    a.srch_t_before_e = S.e_off - S.t_off;
     DeviceInfo di;
     int st = device_info(&di);
     if (st != PVQ_OK) return st;

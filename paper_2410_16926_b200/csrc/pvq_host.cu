@@ -221,7 +221,7 @@ const SearchLayout& search_layout_for(int N, int K) {
             for (int m = 1; m <= last && distinct; ++m) distinct = (kr[m] >> s) != (kr[m - 1] >> s);
             if (distinct) sh = s;
         }
-        if (sh < 0) return S;
+        if (sh < 1) return S;  // the low key bits have to leave a bucket entry's low byte free
         S.rows.shift[n] = static_cast<uint8_t>(sh);
         S.rows.b_off[n] = boff;
         S.rows.b_len[n] = (kr[last] >> sh) - (key_one >> sh) + 1u;
@@ -238,7 +238,7 @@ const SearchLayout& search_layout_for(int N, int K) {
     }
     S.rec_off = kSearchHeader;
     S.b_off = S.rec_off + static_cast<uint32_t>(N) * 16u;
-    S.t_off = (S.b_off + boff + 15u) & ~15u;
+    S.t_off = (S.b_off + 4u * boff + 15u) & ~15u;
     S.te_bytes = (teoff + 15u) & ~15u;
     S.e_off = S.t_off + S.te_bytes;
     S.total = (S.e_off + S.te_bytes + 127u) & ~127u;

@@ -55,6 +55,7 @@ struct BatchArgs {
     uint32_t* debug_status;  // bounds-checked build: where violations are reported (pvq_debug_status); else null
     // decode by threshold search (SearchLayout): the section's place in the blob and its bytes
     uint32_t srch_off, srch_bytes;
+    uint32_t srch_t_before_e;  // bytes from a row of T to the same row of E
 };
 
 // Layout of the table blob.  Section 0 is the count table as the paper defines it,
@@ -187,11 +188,14 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
 // (V(n,k) = sum_{j<=k} N(n,j), App. C.2): with m the first index whose threshold is >= q,
 // k' = m >> 1 pulses remain after the position, |y| = k - k', y > 0 iff m is odd, and the q of
 // the next position is q + E_n[m], E_n[m] = U(n-1,k') - T_n[m] (the encoder's telescoped
-// tables).  m is found without a loop: a key of q (its leading 24 bits as an fp32, see
-// search_key) shifted right by a per-row amount numbers a bucket, the row's byte table gives
-// the first threshold index that can be right for that bucket, and the shift is chosen
-// (on the host, from the exact thresholds) so that no two thresholds of a row share a
-// bucket: one multi-word compare with that threshold settles m.
+// tables).  m is found without a loop.  A key of q (its leading 24 bits as an fp32, see
+// search_key) shifted right by a per-row amount numbers a bucket; the shift is chosen (on the
+// host, from the exact thresholds) so that no two thresholds of a row share a bucket.  The
+// bucket's entry holds m0, the number of thresholds in earlier buckets, and the key bits
+// below the shift of the one threshold that can lie in the bucket: q is beyond that threshold
+// iff its own low key bits are larger, and only when they are equal and the threshold has more
+// than 24 bits (the two agree in their leading 24 bits) does the multi-word compare with
+// T_n[m0] have to decide.
 //
 // Values shrink from row to row (q <= N(n+1,K) at row n), so the rows are narrower towards
 // the end of the vector: a row's thresholds and increments are stored, and its arithmetic is
@@ -203,10 +207,13 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
 // staged as one piece:
 //     header    32 bytes: magic, N, K, bytes of the section, then the number of rows whose
 //               arithmetic is done in 4, 3, 2 and 1 words (the widest rows are the top ones)
-//     records   one 16-byte record per row n: byte offsets (from the section's start) of the
-//               row of T, of the row of E, of the row's bucket table minus its first bucket
-//               number, and the shift
-//     buckets   the rows' byte tables, one after the other
+//     records   one 16-byte record per row n: 32 - shift, the byte offsets (from the section's
+//               start) of the row of E and of the row's bucket table minus four times its
+//               first bucket number, and the shift; the row of T is t_off - e_off from that of E
+//     buckets   the rows' tables, one after the other, 4 bytes a bucket: m0 in the low byte,
+//               in the top bits the low `shift` key bits of T_n[m0] if T_n[m0] lies in the
+//               bucket, else all ones in bits 8..31 (no q of the bucket is beyond T_n[m0]);
+//               bit 8 is set when T_n[m0] < 2^24, where equal keys mean equal numbers
 //     T, E      rows of 2K+2 entries (thresholds m = 0..2K; E modulo 2^(32 words)) of 1, 2 or
 //               4 words (three-word rows use four-word entries)
 constexpr int kSearchMaxRows = 64;

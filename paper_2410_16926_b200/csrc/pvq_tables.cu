@@ -278,8 +278,8 @@ __global__ void derive_fast_tables_kernel(int N, int K, int Wc, uint32_t* __rest
 // The search section (SearchLayout), block n = row n, thread m = threshold m.  Runs after
 // derive_tables_kernel: thresholds and increments come from the cumulative tables U and 2V.
 // The bucket table of a row holds, for every bucket, how many thresholds lie in earlier
-// buckets: thread m writes its index into the buckets after that of threshold m-1 up to
-// its own.
+// buckets, and the low key bits of the threshold in the bucket, if any: thread m writes the
+// buckets after that of threshold m-1 up to its own.
 __global__ void __launch_bounds__(256) derive_search_tables_kernel(int N, int K, int Wc, uint32_t* __restrict__ blob,
                                                                    const __grid_constant__ SearchLayout S) {
     __shared__ uint32_t bucket_of[256];
@@ -314,20 +314,25 @@ __global__ void __launch_bounds__(256) derive_search_tables_kernel(int N, int K,
             E[w] = w < RW ? static_cast<uint32_t>(d) : 0u;
         }
     }
-    const uint32_t sh = S.rows.shift[n];
-    bucket_of[m] = m <= last ? (search_key(t, Wc) >> sh) - (kSearchKeyOfOne >> sh) : 0u;
+    const uint32_t sh = S.rows.shift[n];  // 1..23
+    const uint32_t key = search_key(t, Wc);
+    bucket_of[m] = m <= last ? (key >> sh) - (kSearchKeyOfOne >> sh) : 0u;
     __syncthreads();
     if (m <= last) {
-        uint8_t* B = sec + S.b_off + S.rows.b_off[n];
+        uint32_t* B = reinterpret_cast<uint32_t*>(sec + S.b_off) + S.rows.b_off[n];
         const uint32_t hi = bucket_of[m];
         const uint32_t lo = m == 0 ? 0u : bucket_of[m - 1] + 1u;
-        for (uint32_t b = lo; b <= hi && b < S.rows.b_len[n]; ++b) B[b] = static_cast<uint8_t>(m);
+        // a threshold below 2^24 is its key: equal key bits then mean equal numbers, and bit 8
+        // of the entry says so (it keeps the decoder from comparing in full)
+        const uint32_t exact = key < 0x4b800000u ? 0x100u : 0u;
+        for (uint32_t b = lo; b <= hi && b < S.rows.b_len[n]; ++b)
+            B[b] = (b == hi ? (key << (32u - sh)) | exact : 0xffffff00u) | static_cast<uint32_t>(m);
     }
     if (m == 0) {
         uint32_t* rec = reinterpret_cast<uint32_t*>(sec + S.rec_off) + 4 * n;
-        rec[0] = S.t_off + S.rows.te_off[n];
+        rec[0] = 32u - sh;
         rec[1] = S.e_off + S.rows.te_off[n];
-        rec[2] = S.b_off + S.rows.b_off[n] - (kSearchKeyOfOne >> sh);
+        rec[2] = S.b_off + 4u * (S.rows.b_off[n] - (kSearchKeyOfOne >> sh));
         rec[3] = sh;
         if (n == 0) {
             uint32_t* head = reinterpret_cast<uint32_t*>(sec);

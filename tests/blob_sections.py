@@ -3,8 +3,11 @@
 With V(n,k) = sum_{j<=k} N(n,j) (App. C.2) the thresholds of row n are
 T_n[2k] = V(n,k) + V(n,k-1) and T_n[2k+1] = 2 V(n,k); the increment that goes with threshold m
 is E_n[m] = T_{n-1}[2 (m >> 1)] - T_n[m] (T_{-1} = 0).  A row's bucket table maps the leading
-bits of a value q to the number of thresholds that lie in earlier buckets, and the row takes the
-fewest leading bits for which no two of its thresholds share a bucket.  Rows are stored in the
+bits of a value q to the number m0 of thresholds that lie in earlier buckets, and the row takes
+the fewest leading bits for which no two of its thresholds share a bucket.  A bucket's entry is
+m0 in its low byte and, above it, the key bits below the bucket number of the threshold that lies
+in the bucket, left-aligned (all ones when the bucket has none); bit 8 marks a threshold below
+2^24, which its key represents exactly.  Rows are stored in the
 fewest 32-bit words that hold their largest threshold, classed in aligned blocks of four rows (a
 block takes the width of its top row); three-word rows use four-word entries.  Plain Python
 integers throughout; nothing here comes from the library.
@@ -98,11 +101,15 @@ def section(count, N, K, W, blob_bytes_before):
                 break
         else:
             return None
+        if sh < 1:
+            return None
         base = KEY_OF_ONE >> sh
         length = ids[-1] - base + 1
         tab = []
         for m, b in enumerate(ids):
-            tab += [m] * (b - base + 1 - len(tab))
+            tab += [0xFFFFFF00 | m] * (b - base - len(tab))            # buckets without a threshold
+            exact = 0x100 if T[n][m] < 1 << 24 else 0                  # equal keys are equal numbers there
+            tab.append(((keys[m] << (32 - sh)) & 0xFFFFFFFF) | exact | m)  # the bucket of threshold m
         assert len(tab) == length
         shifts.append(sh)
         lens.append(length)
@@ -111,7 +118,7 @@ def section(count, N, K, W, blob_bytes_before):
         boff += length
     rec_off = 32
     b_off = rec_off + 16 * N
-    t_off = (b_off + boff + 15) & ~15
+    t_off = (b_off + 4 * boff + 15) & ~15
     te_bytes = (teoff + 15) & ~15
     e_off = t_off + te_bytes
     total = (e_off + te_bytes + 127) & ~127
@@ -129,16 +136,24 @@ def section(count, N, K, W, blob_bytes_before):
                 te_bytes=te_bytes, total=total, shifts=shifts, lens=lens, offs=offs, tables=tables, T=T, E=E)
 
 
-def decode_with(sec, count, code, N, K):
-    """The point of `code`, found the way the section is meant to be used."""
+def decode_with(sec, count, code, N, K, ties=None):
+    """The point of `code`, found the way the section is meant to be used; `ties` (a list) collects
+    the positions where the key bits could not decide."""
     q = count[N][K] - code
     k, y = K, []
     for i in range(N):
         n = N - 1 - i
         sh = sec["shifts"][n]
-        m = sec["tables"][n][(key_bits(q) >> sh) - (KEY_OF_ONE >> sh)]
-        if sec["T"][n][m] < q:
-            m += 1
+        key = key_bits(q)
+        entry = sec["tables"][n][(key >> sh) - (KEY_OF_ONE >> sh)]
+        x = (key << (32 - sh)) & 0xFFFFFFFF
+        m0 = entry & 0xFF
+        m = m0 + (1 if x > entry else 0)
+        if (entry - x) & 0xFFFFFFFF < 256:          # same leading 24 bits as the threshold: compare in full
+            m = m0 + (1 if sec["T"][n][m0] < q else 0)
+            if ties is not None:
+                ties.append(i)
+        assert sec["T"][n][m] >= q and (m == 0 or sec["T"][n][m - 1] < q)
         kp = m >> 1
         y.append(k - kp if m & 1 else kp - k)
         q += (sec["T"][n - 1][2 * kp] if n >= 1 else 0) - sec["T"][n][m]

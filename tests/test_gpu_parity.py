@@ -166,15 +166,14 @@ def test_table_blob_sections(N, K):
         # the decoder's search section: header, row records, bucket tables, thresholds, increments
         sec = blob[srch["off"] // 4: (srch["off"] + srch["total"]) // 4]
         assert list(sec[:8]) == [bs.MAGIC, N, K, srch["total"]] + srch["counts"]
-        raw = sec.view(np.uint8)
         for n in range(N):
             rec = sec[(srch["rec_off"] + 16 * n) // 4: (srch["rec_off"] + 16 * n) // 4 + 4]
             sh, ew, at = srch["shifts"][n], srch["ewords"][n], srch["te_offs"][n]
-            want = [srch["t_off"] + at, srch["e_off"] + at,
-                    (srch["b_off"] + srch["offs"][n] - (bs.KEY_OF_ONE >> sh)) & 0xFFFFFFFF, sh]
+            want = [32 - sh, srch["e_off"] + at,
+                    (srch["b_off"] + 4 * (srch["offs"][n] - (bs.KEY_OF_ONE >> sh))) & 0xFFFFFFFF, sh]
             assert list(rec) == want, ("record", n)
-            b0 = srch["b_off"] + srch["offs"][n]
-            assert list(raw[b0: b0 + srch["lens"][n]]) == srch["tables"][n], ("buckets", n)
+            b0 = srch["b_off"] // 4 + srch["offs"][n]
+            assert list(sec[b0: b0 + srch["lens"][n]]) == srch["tables"][n], ("buckets", n)
             for name, vals in (("t_off", srch["T"]), ("e_off", srch["E"])):
                 row = sec[(srch[name] + at) // 4: (srch[name] + at) // 4 + (2 * K + 2) * ew].reshape(2 * K + 2, ew)
                 for m in range(2 * K + 1):
@@ -390,6 +389,57 @@ def test_decode_of_codes_the_encoder_did_not_make(N, K):
     flat[2 * third::32] = sflat[2 * third::32]
     flat[-1] = big
     flat[0] = 0
+    sidx = rng.integers(0, 256, size=(rows, int(pvq.scale_row_stride(G, b))), dtype=np.uint8)
+    rnorm = (rng.random(rows).astype(np.float32) + 0.5)
+    enc_np = (codes, sidx, rnorm)
+    enc_dev = (torch.from_numpy(codes.view(np.int32)).to(DEV), torch.from_numpy(sidx).to(DEV),
+               torch.from_numpy(rnorm).to(DEV))
+    check_decode(cd, enc_dev, enc_np)
+
+
+@pytest.mark.parametrize("N,K", [(32, 50), (32, 22), (16, 27), (8, 40), (64, 31), (32, 105)])
+def test_decode_of_codes_on_the_search_thresholds(N, K):
+    """Codes whose running value sits on a threshold of the searching decoder, or next to one:
+    points y = (a_0, ..., a_p, rest) where the rest is the first or the last point of its
+    pyramid put the value of position p + 1 exactly on, or one beyond, a threshold, which the
+    leading 24 bits cannot tell apart; also the neighbours of such codes."""
+    from oracle import pvq_pyref as pr
+    rows, G, b = 4, 64, 8
+    cd = Codec(N, 0, G, b, K=K)
+    W = cd.W
+    count = pr.count_table(N, K)
+    total = count[N][K]
+    rng = np.random.default_rng(77 * N + K)
+    want = rows * G
+    ints = []
+    while len(ints) < want:
+        # a random prefix, then all remaining pulses on one late coordinate (first / last points of
+        # the sub-pyramids behind the prefix), either sign
+        p = int(rng.integers(0, N - 1))
+        y = [0] * N
+        left = K
+        for i in range(p):
+            if left == 0:
+                break
+            v = int(rng.integers(0, min(left, 4) + 1))
+            y[i] = v if rng.integers(0, 2) else -v
+            left -= v
+        pos = int(rng.choice([p, N - 1]))
+        y[pos] += left if rng.integers(0, 2) else -left
+        if sum(abs(v) for v in y) != K:
+            continue
+        c = pr.enumerate_point(y, K)
+        for d in (0, -1, 1):
+            if 0 <= c + d < total:
+                ints.append(c + d)
+    codes = np.array([po.int_to_code(c, W) for c in ints[:want]], dtype=np.uint32).reshape(rows, G, W)
+    if cd.W <= 4 and K <= 127:
+        sec = bs.section(count, N, K, W, 0)
+        if sec is not None:   # these inputs do reach the full compare
+            ties = []
+            for c in ints[:want]:
+                bs.decode_with(sec, count, c, N, K, ties)
+            assert len(ties) > want // 4
     sidx = rng.integers(0, 256, size=(rows, int(pvq.scale_row_stride(G, b))), dtype=np.uint8)
     rnorm = (rng.random(rows).astype(np.float32) + 0.5)
     enc_np = (codes, sidx, rnorm)
