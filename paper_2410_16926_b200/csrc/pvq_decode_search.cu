@@ -30,168 +30,6 @@ namespace {
 
 constexpr int kSearchThreads = 1024;
 
-__device__ __forceinline__ uint4 load_record(uint32_t addr) {
-    uint4 v;
-#ifdef PVQ_DEBUG
-    if (!debug_table_ok(addr, 16)) return make_uint4(0u, 0u, 0u, 0u);
-#endif
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
-
-__device__ __forceinline__ uint32_t load_bucket(uint32_t addr) {
-    uint32_t v;
-#ifdef PVQ_DEBUG
-    if (!debug_table_ok(addr, 4)) return 0u;
-#endif
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-
-// m0 + (t < q): minus the borrow of t - q, which the last link of the chain leaves as 0 or -1
-template <int W>
-__device__ __forceinline__ uint32_t bump_if_less(uint32_t m0, const mp<W>& t, const mp<W>& q) {
-    uint32_t m;
-    if constexpr (W == 1) {
-        asm("{\n\t.reg .u32 d;\n\t"
-            "sub.cc.u32 d, %2, %3;\n\t"
-            "subc.u32 d, 0, 0;\n\t"
-            "sub.u32 %0, %1, d;\n\t}"
-            : "=r"(m)
-            : "r"(m0), "r"(t.w[0]), "r"(q.w[0]));
-    } else if constexpr (W == 2) {
-        asm("{\n\t.reg .u32 d;\n\t"
-            "sub.cc.u32 d, %2, %4;\n\t"
-            "subc.cc.u32 d, %3, %5;\n\t"
-            "subc.u32 d, 0, 0;\n\t"
-            "sub.u32 %0, %1, d;\n\t}"
-            : "=r"(m)
-            : "r"(m0), "r"(t.w[0]), "r"(t.w[1]), "r"(q.w[0]), "r"(q.w[1]));
-    } else if constexpr (W == 3) {
-        asm("{\n\t.reg .u32 d;\n\t"
-            "sub.cc.u32 d, %2, %5;\n\t"
-            "subc.cc.u32 d, %3, %6;\n\t"
-            "subc.cc.u32 d, %4, %7;\n\t"
-            "subc.u32 d, 0, 0;\n\t"
-            "sub.u32 %0, %1, d;\n\t}"
-            : "=r"(m)
-            : "r"(m0), "r"(t.w[0]), "r"(t.w[1]), "r"(t.w[2]), "r"(q.w[0]), "r"(q.w[1]), "r"(q.w[2]));
-    } else {
-        static_assert(W == 4, "codes of up to four words");
-        asm("{\n\t.reg .u32 d;\n\t"
-            "sub.cc.u32 d, %2, %6;\n\t"
-            "subc.cc.u32 d, %3, %7;\n\t"
-            "subc.cc.u32 d, %4, %8;\n\t"
-            "subc.cc.u32 d, %5, %9;\n\t"
-            "subc.u32 d, 0, 0;\n\t"
-            "sub.u32 %0, %1, d;\n\t}"
-            : "=r"(m)
-            : "r"(m0), "r"(t.w[0]), "r"(t.w[1]), "r"(t.w[2]), "r"(t.w[3]), "r"(q.w[0]), "r"(q.w[1]), "r"(q.w[2]),
-              "r"(q.w[3]));
-    }
-    return m;
-}
-
-// Four bytes of a thread's slot at once.
-__device__ __forceinline__ void store_y4(uint32_t addr, uint32_t val) {
-#ifdef PVQ_DEBUG
-    if (!debug_slot_ok(addr, 4)) return;
-#endif
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(val) : "memory");
-}
-
-// Four positions of GP codes (GP independent chains of dependent table reads, so that one
-// thread keeps several reads in flight), in PW-word arithmetic on rows stored PW words wide.
-// `rec` is the shared address of the record of the first of the four rows (the rows of the
-// following positions have the records before it); a record is read once for all chains.
-// The four y_i + 128 of chain j go to the word at y + j * ychain.
-//
-// Per position: the key of q selects a bucket; its entry is m0 and the low key bits of the
-// threshold T[m0]; q's own low key bits being larger means q > T[m0], smaller means q <= T[m0]
-// (a bucket without a threshold holds all ones there).  Equal bits leave it open: then, and
-// that is rare, the threads of the warp whose bits were equal compare q with T[m0] in full.
-template <int W, int PW, int GP>
-__device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP], uint32_t rec, uint32_t t_before_e,
-                                              uint32_t y, uint32_t ychain) {
-    constexpr int EB = search_entry_words(PW) * 4;  // bytes of an entry of T and E
-    uint32_t acc[GP];
-    mp<PW> v[GP];  // the low PW words of q: the rest is zero by now
-#pragma unroll
-    for (int j = 0; j < GP; ++j) {
-        acc[j] = 0u;
-#pragma unroll
-        for (int w = 0; w < PW; ++w) v[j].w[w] = q[j].w[w];
-    }
-#pragma unroll
-    for (int s = 0; s < 4; ++s) {
-        const uint4 r = load_record(rec - static_cast<uint32_t>(s) * 16u);  // 32 - shift, E row, buckets, shift
-        uint32_t key[GP], entry[GP], m[GP];
-        mp<PW> e[GP];
-        bool open = false;
-#pragma unroll
-        for (int j = 0; j < GP; ++j) {
-            key[j] = search_key<PW>(v[j].w);
-            entry[j] = load_bucket(r.z + ((key[j] >> r.w) << 2));
-        }
-#pragma unroll
-        for (int j = 0; j < GP; ++j) {
-            const uint32_t x = key[j] << r.x;  // the key bits below the shift, left-aligned like the entry's
-            m[j] = (entry[j] & 0xffu) + (x > entry[j] ? 1u : 0u);
-            open = open || (entry[j] - x < 256u);
-        }
-        if (__any_sync(kFull, open)) {
-#pragma unroll
-            for (int j = 0; j < GP; ++j) {
-                const uint32_t m0 = entry[j] & 0xffu;
-                if (entry[j] - (key[j] << r.x) < 256u)
-                    m[j] = bump_if_less<PW>(m0, load_entry<PW>(r.y - t_before_e + m0 * EB), v[j]);
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < GP; ++j) e[j] = load_entry<PW>(r.y + m[j] * EB);
-#pragma unroll
-        for (int j = 0; j < GP; ++j) {
-            mp_add<PW>(v[j], e[j]);
-            const uint32_t kp = m[j] >> 1;  // pulses left after this position
-            const int mag = static_cast<int>(k[j] - kp);
-            const uint32_t val = static_cast<uint32_t>((m[j] & 1u) ? 128 + mag : 128 - mag);
-            acc[j] = __funnelshift_r(acc[j], val, 8);  // the new byte enters at the top
-            k[j] = kp;
-        }
-    }
-#pragma unroll
-    for (int j = 0; j < GP; ++j) {
-        store_y4(y + static_cast<uint32_t>(j) * ychain, acc[j]);
-#pragma unroll
-        for (int w = 0; w < PW; ++w) q[j].w[w] = v[j].w[w];
-    }
-}
-
-// The points of GP codes: q = N(N,K) - code on entry.  `recs` is the shared address of the
-// row records (absolute shared addresses by now), cnt[w] the number of rows done in w words.
-template <int N, int W, int GP>
-__device__ __forceinline__ void search_codes(mp<W> (&q)[GP], int K, uint32_t recs, uint32_t t_before_e,
-                                             const int (&cnt)[5], uint32_t y, uint32_t ychain) {
-    uint32_t k[GP];
-#pragma unroll
-    for (int j = 0; j < GP; ++j) k[j] = static_cast<uint32_t>(K);
-    uint32_t rec = recs + static_cast<uint32_t>(N - 1) * 16u;
-    if constexpr (W >= 4) {
-#pragma unroll 1
-        for (int b = 0; b < cnt[4]; b += 4, rec -= 64u, y += 4u) search_block4<W, 4, GP>(q, k, rec, t_before_e, y, ychain);
-    }
-    if constexpr (W >= 3) {
-#pragma unroll 1
-        for (int b = 0; b < cnt[3]; b += 4, rec -= 64u, y += 4u) search_block4<W, 3, GP>(q, k, rec, t_before_e, y, ychain);
-    }
-    if constexpr (W >= 2) {
-#pragma unroll 1
-        for (int b = 0; b < cnt[2]; b += 4, rec -= 64u, y += 4u) search_block4<W, 2, GP>(q, k, rec, t_before_e, y, ychain);
-    }
-#pragma unroll 1
-    for (int b = 0; b < cnt[1]; b += 4, rec -= 64u, y += 4u) search_block4<W, 1, GP>(q, k, rec, t_before_e, y, ychain);
-}
-
 // GP groups per thread: a warp takes GP consecutive tiles of 32 groups in one pass.
 template <int N, int W, int GP>
 __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
@@ -205,16 +43,21 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
     // stage the search section with the bulk-copy engine; waited for below
     __shared__ uint64_t stage_bar;
     const BulkStage stage = bulk_stage_begin(&stage_bar);
+    // (records and bucket tables, then the increments E where the blob has the thresholds T)
+    const uint8_t* section = reinterpret_cast<const uint8_t*>(a.table) + a.srch_off;
+    const uint32_t staged = a.srch_bytes - a.srch_t_before_e;
     if (threadIdx.x == 0) {
-        bulk_stage_expect(stage, a.srch_bytes);
-        bulk_stage_copy(stage, smem, reinterpret_cast<const uint8_t*>(a.table) + a.srch_off, a.srch_bytes);
+        bulk_stage_expect(stage, staged);
+        bulk_stage_copy(stage, smem, section, a.srch_t_off);
+        bulk_stage_copy(stage, smem + a.srch_t_off, section + a.srch_t_off + a.srch_t_before_e, staged - a.srch_t_off);
     }
+    // global address of a row of T = t_rows + shared address of the row of E
+    const uint8_t* t_rows = section - sbase;
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    // slots: chain j of thread t at (j * blockDim.x + t) * YS behind the tables (srch_bytes is a
-    // multiple of 128)
-    uint8_t* yslots = smem + a.srch_bytes + threadIdx.x * YS;
+    // slots: chain j of thread t at (j * blockDim.x + t) * YS behind the tables (a multiple of 16 bytes)
+    uint8_t* yslots = smem + staged + threadIdx.x * YS;
     const uint32_t ychain = blockDim.x * YS;
 
     // N(N,K): codes at or above it are invalid
@@ -226,33 +69,16 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
         if (a.status && threadIdx.x == 0) atomicOr(a.status, PVQ_STATUS_STAGING_TIMEOUT);
         return;
     }
-    {  // a table built for another (N,K) would send the look-ups anywhere: refuse it
-        const uint32_t* head = reinterpret_cast<const uint32_t*>(smem);
-        if (head[0] != kSearchMagic || head[1] != static_cast<uint32_t>(N) || head[2] != static_cast<uint32_t>(K) ||
-            head[3] != a.srch_bytes) {
-            if (a.status && threadIdx.x == 0) atomicOr(a.status, PVQ_STATUS_TABLE_MISMATCH);
-            return;
-        }
-    }
     int cnt[5];
-#pragma unroll
-    for (int w = 1; w <= 4; ++w) cnt[w] = static_cast<int>(reinterpret_cast<const uint32_t*>(smem)[8 - w]);
-    cnt[0] = 0;
-    if (cnt[1] + cnt[2] + cnt[3] + cnt[4] != N || ((cnt[1] | cnt[2] | cnt[3] | cnt[4]) & 3) != 0 ||
-        (W < 4 && cnt[4] != 0) || (W < 3 && cnt[3] != 0) || (W < 2 && cnt[2] != 0)) {
+    if (!search_section_begin<N, W>(smem, a.srch_bytes, a.srch_t_before_e, K, cnt)) {  // not the table of this (N,K): refuse it
         if (a.status && threadIdx.x == 0) atomicOr(a.status, PVQ_STATUS_TABLE_MISMATCH);
         return;
     }
-    if (threadIdx.x < N) {  // the records' offsets become shared addresses
-        uint32_t* rec = reinterpret_cast<uint32_t*>(smem + kSearchHeader) + 4 * threadIdx.x;
-        rec[1] += sbase;
-        rec[2] += sbase;
-    }
 #ifdef PVQ_DEBUG
-    debug_begin(sbase, sbase + a.srch_bytes, sbase + a.srch_bytes, YS, N, a.debug_status);
+    debug_begin(sbase, sbase + staged, sbase + staged, YS, N, a.debug_status);
     if (threadIdx.x == 0) {
         s_debug.slot_chain = ychain;
-        s_debug.slot_end = sbase + a.srch_bytes + GP * ychain;
+        s_debug.slot_end = sbase + staged + GP * ychain;
     }
 #endif
     __syncthreads();
@@ -319,7 +145,7 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
             }
             mp_sub_borrow<W>(q[j], bound, c);  // 1 <= q <= N(N,K)
         }
-        search_codes<N, W, GP>(q, K, recs, a.srch_t_before_e, cnt, shared_addr(yslots), ychain);
+        search_codes<N, W, GP>(q, K, recs, t_rows, cnt, shared_addr(yslots), ychain);
 #pragma unroll
         for (int j = 0; j < GP; ++j)
             if (active[j])
@@ -342,7 +168,9 @@ int launch_search_t(BatchArgs& a, const SearchLayout& S, cudaStream_t stream) {
     a.total_tiles = tiles;
     a.srch_off = S.off;
     a.srch_bytes = S.total;
+    a.srch_t_off = S.t_off;
     a.srch_t_before_e = S.e_off - S.t_off;
+    const size_t staged = S.total - (S.e_off - S.t_off);
     DeviceInfo di;
     int st = device_info(&di);
     if (st != PVQ_OK) return st;
@@ -354,12 +182,16 @@ int launch_search_t(BatchArgs& a, const SearchLayout& S, cudaStream_t stream) {
     int threads = 0;
     size_t smem = 0;
     double best_score = -1.0;
-    for (int t = kMaxThreads; t >= kMaxThreads / 2; t -= 32) {
-        const size_t bytes = static_cast<size_t>(S.total) + static_cast<size_t>(t) * YS * GP;
+    for (int t = kMaxThreads; t >= 128; t -= 32) {
+        const size_t bytes = staged + static_cast<size_t>(t) * YS * GP;
         if (bytes > static_cast<size_t>(di.smem_max)) continue;
         const double slots = static_cast<double>(di.sms) * (t / 32) * GP;
         const double rounds = std::ceil(tiles / slots);
-        const double score = tiles / (rounds * slots) * (1.0 - 0.004 * (kMaxThreads - t) / 32);
+        // a launch of one round: the smallest block that still makes it one round (the work
+        // spreads over more SMs); otherwise the fullest rounds among the larger blocks
+        if (rounds > 1.0 && t < kMaxThreads / 2) break;
+        const double score = rounds > 1.0 ? tiles / (rounds * slots) * (1.0 - 0.004 * (kMaxThreads - t) / 32)
+                                          : 2.0 + (kMaxThreads - t);
         if (score > best_score) {
             best_score = score;
             threads = t;

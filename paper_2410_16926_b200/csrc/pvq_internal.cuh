@@ -55,6 +55,7 @@ struct BatchArgs {
     uint32_t* debug_status;  // bounds-checked build: where violations are reported (pvq_debug_status); else null
     // decode by threshold search (SearchLayout): the section's place in the blob and its bytes
     uint32_t srch_off, srch_bytes;
+    uint32_t srch_t_off;       // where the thresholds T start in the section; they stay in global memory
     uint32_t srch_t_before_e;  // bytes from a row of T to the same row of E
 };
 
