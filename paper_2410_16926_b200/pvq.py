@@ -19,6 +19,8 @@ LIB_PATH = os.environ.get("PVQ_B200_LIB") or os.path.join(_HERE, "libpvq_b200.so
 DTYPE_F32 = 0
 DTYPE_BF16 = 1
 STATUS_INVALID_CODE = 1
+STATUS_STAGING_TIMEOUT = 2
+STATUS_TABLE_MISMATCH = 4
 
 _lib = None
 

@@ -448,6 +448,26 @@ def test_decode_of_codes_on_the_search_thresholds(N, K):
     check_decode(cd, enc_dev, enc_np)
 
 
+def test_decode_refuses_a_table_built_for_other_parameters():
+    """The searching decoder's look-ups follow what the table says, so it checks the header of
+    its section first: with the table of another K nothing is decoded and the status says so."""
+    N, G, b, rows = 32, 64, 8, 4
+    cd = Codec(N, 0, G, b, K=50)
+    assert pvq.code_words(N, 49) == cd.W
+    assert pvq.count_table_bytes(N, 49) <= pvq.count_table_bytes(N, 50)
+    rng = np.random.default_rng(3)
+    codes = torch.from_numpy(rng.integers(0, 1 << 20, size=(rows, G, cd.W), dtype=np.int64).astype(np.int32)).to(DEV)
+    sidx = torch.zeros((rows, int(pvq.scale_row_stride(G, b))), dtype=torch.uint8, device=DEV)
+    rnorm = torch.ones(rows, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out, check = guarded((rows, G * N), torch.bfloat16, 7.0)
+    pvq.decode(codes, sidx, rnorm, N, 49, b, cd.table, cd.levels, status=status, out=out)   # cd.table is for K = 50
+    torch.cuda.synchronize()
+    check()
+    assert int(status.item()) == pvq.STATUS_TABLE_MISMATCH
+    assert bool((out == 7.0).all())
+
+
 def test_fused_roundtrip_equals_encode_then_decode():
     for (N, bits, rows, cols, b, kind) in [(32, 64, 40, 4096, 8, "bf16"), (16, 40, 9, 208, 4, "f32"),
                                            (64, 192, 5, 3584, 6, "bf16")]:
