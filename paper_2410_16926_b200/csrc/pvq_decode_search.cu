@@ -31,7 +31,7 @@ namespace {
 constexpr int kSearchThreads = 1024;
 
 // GP groups per thread: a warp takes GP consecutive tiles of 32 groups in one pass.
-template <int N, int W, int GP>
+template <int N, int W, int GP, int PLANE>
 __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
     decode_search_kernel(const __grid_constant__ BatchArgs a) {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
             }
             mp_sub_borrow<W>(q[j], bound, c);  // 1 <= q <= N(N,K)
         }
-        search_codes<N, W, GP>(q, K, recs, t_rows, cnt, shared_addr(yslots), ychain);
+        search_codes<N, W, GP, PLANE>(q, K, recs, t_rows, cnt, shared_addr(yslots), ychain);
 #pragma unroll
         for (int j = 0; j < GP; ++j)
             if (active[j])
@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
     if (bad && a.status) atomicOr(a.status, PVQ_STATUS_INVALID_CODE);
 }
 
-template <int N, int W, int GP>
+template <int N, int W, int GP, int PLANE>
 int launch_search_t(BatchArgs& a, const SearchLayout& S, cudaStream_t stream) {
     constexpr int YS = N + 4;
     constexpr int kMaxThreads = kSearchThreads / (GP > 2 ? 2 : 1);
@@ -178,7 +178,7 @@ int launch_search_t(BatchArgs& a, const SearchLayout& S, cudaStream_t stream) {
     // per resident warp; among the block sizes that fit, take the one whose rounds are
     // fullest, with a preference for more warps (they hide the latency of the dependent
     // table reads).
-    auto kern = decode_search_kernel<N, W, GP>;
+    auto kern = decode_search_kernel<N, W, GP, PLANE>;
     int threads = 0;
     size_t smem = 0;
     double best_score = -1.0;
@@ -215,7 +215,12 @@ int launch_search_t(BatchArgs& a, const SearchLayout& S, cudaStream_t stream) {
 // two: 333 us, four at half the threads: 455 us).
 template <int N, int W>
 int launch_search_g(BatchArgs& a, const SearchLayout& S, cudaStream_t stream) {
-    return launch_search_t<N, W, 2>(a, S, stream);
+    switch (S.plane) {  // entries per word plane of the section's rows
+        case 64: return launch_search_t<N, W, 2, 64>(a, S, stream);
+        case 128: return launch_search_t<N, W, 2, 128>(a, S, stream);
+        case 256: return launch_search_t<N, W, 2, 256>(a, S, stream);
+        default: return PVQ_ERR_UNSUPPORTED;
+    }
 }
 
 template <int N, int WMAX>

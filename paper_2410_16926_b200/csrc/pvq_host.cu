@@ -228,13 +228,14 @@ const SearchLayout& search_layout_for(int N, int K) {
         boff += S.rows.b_len[n];
     }
     if (N % 4 != 0) return S;
+    S.plane = search_plane_of(K);
     uint32_t teoff = 0;
     for (int n = N - 1; n >= 0; --n) {  // a block of four rows takes the width of its top row
         const int w = need[static_cast<size_t>(n | 3)];
         S.rows.words[n] = static_cast<uint8_t>(w);
         S.count[w] += 1;
         S.rows.te_off[n] = teoff;
-        teoff += static_cast<uint32_t>(2 * K + 2) * search_entry_words(w) * 4u;
+        teoff += static_cast<uint32_t>(S.plane) * w * 4u;
     }
     S.rec_off = kSearchHeader;
     S.b_off = S.rec_off + static_cast<uint32_t>(N) * 16u;

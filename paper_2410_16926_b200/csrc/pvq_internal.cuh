@@ -215,14 +215,17 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
 //               in the top bits the low `shift` key bits of T_n[m0] if T_n[m0] lies in the
 //               bucket, else all ones in bits 8..31 (no q of the bucket is beyond T_n[m0]);
 //               bit 8 is set when T_n[m0] < 2^24, where equal keys mean equal numbers
-//     T, E      rows of 2K+2 entries (thresholds m = 0..2K; E modulo 2^(32 words)) of 1, 2 or
-//               4 words (three-word rows use four-word entries)
+//     T, E      rows of `plane` entries (64, 128 or 256: the first that holds the thresholds
+//               m = 0..2K; E modulo 2^(32 words)), word by word: a row of w words is w planes
+//               of `plane` 32-bit words, plane j holding word j of every entry.  The threads
+//               of a warp read entries a few indices apart, which word planes put in
+//               different banks (entries of 16 bytes would collide in groups of eight).
 constexpr int kSearchMaxRows = 64;
 constexpr uint32_t kSearchMagic = 0x53515650u;
 constexpr uint32_t kSearchHeader = 32u;
 constexpr uint32_t kSearchLimit = 184u * 1024u;  // the section has to leave room for the output slots
 
-__host__ __device__ constexpr int search_entry_words(int words) { return words == 3 ? 4 : words; }
+__host__ __device__ constexpr int search_plane_of(int K) { return 2 * K + 2 <= 64 ? 64 : (2 * K + 2 <= 128 ? 128 : 256); }
 
 struct SearchRows {  // what the builder needs per row
     uint32_t b_off[kSearchMaxRows];   // of the row's bucket table inside `buckets`
@@ -235,6 +238,7 @@ struct SearchRows {  // what the builder needs per row
 struct SearchLayout {
     bool present;
     int count[5];         // count[w]: rows done in w words
+    int plane;            // entries per word plane of a row of T or E
     uint32_t off;         // of the section in the blob
     uint32_t rec_off, b_off, t_off, e_off;  // of its parts, from the section's start
     uint32_t te_bytes;    // of T, and of E

@@ -118,6 +118,18 @@ __device__ __forceinline__ bool search_section_begin(uint8_t* sec, uint32_t byte
     return true;
 }
 
+// Entry of PW words of a row stored word plane by word plane (PLANE entries a plane): word w
+// sits PLANE words behind word w - 1.  `addr` is the shared address of word 0.
+template <int PW, int PLANE>
+__device__ __forceinline__ mp<PW> load_planes(uint32_t addr) {
+    mp<PW> t;  // the plane offsets go into the loads as immediates
+    t.w[0] = load_entry<1, 0>(addr).w[0];
+    if constexpr (PW > 1) t.w[1] = load_entry<1, PLANE * 4>(addr).w[0];
+    if constexpr (PW > 2) t.w[2] = load_entry<1, 2 * PLANE * 4>(addr).w[0];
+    if constexpr (PW > 3) t.w[3] = load_entry<1, 3 * PLANE * 4>(addr).w[0];
+    return t;
+}
+
 // Four bytes of a thread's slot at once.
 __device__ __forceinline__ void store_y4(uint32_t addr, uint32_t val) {
 #ifdef PVQ_DEBUG
@@ -127,7 +139,7 @@ __device__ __forceinline__ void store_y4(uint32_t addr, uint32_t val) {
 }
 
 // Four positions of GP codes (GP independent chains of dependent table reads, so that one
-// thread keeps several reads in flight), in PW-word arithmetic on rows stored PW words wide.
+// thread keeps several reads in flight), in PW-word arithmetic on rows of PW word planes.
 // `rec` is the shared address of the record of the first of the four rows (the rows of the
 // following positions have the records before it); a record is read once for all chains.
 // `t_rows` plus the shared address of a row of E is the global address of the same row of T.
@@ -137,10 +149,9 @@ __device__ __forceinline__ void store_y4(uint32_t addr, uint32_t val) {
 // threshold T[m0]; q's own low key bits being larger means q > T[m0], smaller means q <= T[m0]
 // (a bucket without a threshold holds all ones there).  Equal bits leave it open: then, and
 // that is rare, the threads of the warp whose bits were equal compare q with T[m0] in full.
-template <int W, int PW, int GP>
+template <int W, int PW, int GP, int PLANE>
 __device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP], uint32_t rec, const uint8_t* t_rows,
                                               uint32_t y, uint32_t ychain) {
-    constexpr int EB = search_entry_words(PW) * 4;  // bytes of an entry of T and E
     uint32_t acc[GP];  // the four threshold indices m, a byte each, first position lowest
     mp<PW> v[GP];      // the low PW words of q: the rest is zero by now
 #pragma unroll
@@ -172,16 +183,16 @@ __device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP],
                 const uint32_t m0 = entry[j] & 0xffu;
                 if (entry[j] - (key[j] << r.x) < 256u) {
                     // the row of T in global memory lies where the row of E lies in shared memory
-                    const uint32_t* tp = reinterpret_cast<const uint32_t*>(t_rows + r.y + m0 * EB);
+                    const uint32_t* tp = reinterpret_cast<const uint32_t*>(t_rows + r.y + m0 * 4u);
                     mp<PW> t;
 #pragma unroll
-                    for (int w = 0; w < PW; ++w) t.w[w] = tp[w];
+                    for (int w = 0; w < PW; ++w) t.w[w] = tp[w * PLANE];
                     m[j] = bump_if_less<PW>(m0, t, v[j]);
                 }
             }
         }
 #pragma unroll
-        for (int j = 0; j < GP; ++j) e[j] = load_entry<PW>(r.y + m[j] * EB);
+        for (int j = 0; j < GP; ++j) e[j] = load_planes<PW, PLANE>(r.y + (m[j] << 2));
 #pragma unroll
         for (int j = 0; j < GP; ++j) {
             mp_add<PW>(v[j], e[j]);
@@ -209,7 +220,7 @@ __device__ __forceinline__ void search_block4(mp<W> (&q)[GP], uint32_t (&k)[GP],
 
 // The points of GP codes: q = N(N,K) - code on entry.  `recs` is the shared address of the
 // row records (absolute shared addresses by now), cnt[w] the number of rows done in w words.
-template <int N, int W, int GP>
+template <int N, int W, int GP, int PLANE>
 __device__ __forceinline__ void search_codes(mp<W> (&q)[GP], int K, uint32_t recs, const uint8_t* t_rows,
                                              const int (&cnt)[5], uint32_t y, uint32_t ychain) {
     uint32_t k[GP];
@@ -218,18 +229,18 @@ __device__ __forceinline__ void search_codes(mp<W> (&q)[GP], int K, uint32_t rec
     uint32_t rec = recs + static_cast<uint32_t>(N - 1) * 16u;
     if constexpr (W >= 4) {
 #pragma unroll 1
-        for (int b = 0; b < cnt[4]; b += 4, rec -= 64u, y += 4u) search_block4<W, 4, GP>(q, k, rec, t_rows, y, ychain);
+        for (int b = 0; b < cnt[4]; b += 4, rec -= 64u, y += 4u) search_block4<W, 4, GP, PLANE>(q, k, rec, t_rows, y, ychain);
     }
     if constexpr (W >= 3) {
 #pragma unroll 1
-        for (int b = 0; b < cnt[3]; b += 4, rec -= 64u, y += 4u) search_block4<W, 3, GP>(q, k, rec, t_rows, y, ychain);
+        for (int b = 0; b < cnt[3]; b += 4, rec -= 64u, y += 4u) search_block4<W, 3, GP, PLANE>(q, k, rec, t_rows, y, ychain);
     }
     if constexpr (W >= 2) {
 #pragma unroll 1
-        for (int b = 0; b < cnt[2]; b += 4, rec -= 64u, y += 4u) search_block4<W, 2, GP>(q, k, rec, t_rows, y, ychain);
+        for (int b = 0; b < cnt[2]; b += 4, rec -= 64u, y += 4u) search_block4<W, 2, GP, PLANE>(q, k, rec, t_rows, y, ychain);
     }
 #pragma unroll 1
-    for (int b = 0; b < cnt[1]; b += 4, rec -= 64u, y += 4u) search_block4<W, 1, GP>(q, k, rec, t_rows, y, ychain);
+    for (int b = 0; b < cnt[1]; b += 4, rec -= 64u, y += 4u) search_block4<W, 1, GP, PLANE>(q, k, rec, t_rows, y, ychain);
 }
 
 }  // namespace pvq

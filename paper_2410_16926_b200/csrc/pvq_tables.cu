@@ -289,8 +289,7 @@ __global__ void __launch_bounds__(256) derive_search_tables_kernel(int N, int K,
     const int i = N - 1 - n;     // the position whose row of the cumulative tables this is
     const int k = m >> 1;
     const int last = n == 0 ? 1 : 2 * K;  // thresholds of the row: 0..last
-    const int RW = S.rows.words[n];       // words of this row's arithmetic
-    const int EW = search_entry_words(RW);
+    const int RW = S.rows.words[n];       // words of this row's arithmetic: its planes
     uint8_t* sec = reinterpret_cast<uint8_t*>(blob) + S.off;
     const uint32_t* U = blob + L.enc_off[0] / 4;   // (i, col + 1), K + 2 entries a row
     const uint32_t* V2 = blob + L.enc_off[1] / 4;
@@ -300,18 +299,18 @@ __global__ void __launch_bounds__(256) derive_search_tables_kernel(int N, int K,
         for (int w = 0; w < Wc; ++w) t[w] = src[w];
     }
     if (m < 2 * K + 2) {
-        const size_t at = (S.rows.te_off[n] + static_cast<size_t>(m) * EW * 4u) / 4u;
+        const size_t at = S.rows.te_off[n] / 4u + static_cast<size_t>(m);  // word 0; word w is w planes further
         uint32_t* T = reinterpret_cast<uint32_t*>(sec + S.t_off) + at;
         uint32_t* E = reinterpret_cast<uint32_t*>(sec + S.e_off) + at;
         // E = U(n-1, k) - T, modulo 2^(32 RW); U(-1, .) = 0
         const uint32_t* un = U + (static_cast<size_t>(i + 1) * (K + 2) + k + 1) * TW;
         long long borrow = 0;
-        for (int w = 0; w < EW; ++w) {
+        for (int w = 0; w < RW; ++w) {
             const long long a = (n >= 1 && w < Wc && m <= 2 * K) ? static_cast<long long>(un[w]) : 0;
             const long long d = a - static_cast<long long>(w < Wc ? t[w] : 0u) + borrow;
             borrow = d >> 32;  // 0 or -1
-            T[w] = w < RW ? t[w] : 0u;
-            E[w] = w < RW ? static_cast<uint32_t>(d) : 0u;
+            T[static_cast<size_t>(w) * S.plane] = t[w];
+            E[static_cast<size_t>(w) * S.plane] = static_cast<uint32_t>(d);
         }
     }
     const uint32_t sh = S.rows.shift[n];  // 1..23

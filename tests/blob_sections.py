@@ -9,7 +9,8 @@ m0 in its low byte and, above it, the key bits below the bucket number of the th
 in the bucket, left-aligned (all ones when the bucket has none); bit 8 marks a threshold below
 2^24, which its key represents exactly.  Rows are stored in the
 fewest 32-bit words that hold their largest threshold, classed in aligned blocks of four rows (a
-block takes the width of its top row); three-word rows use four-word entries.  Plain Python
+block takes the width of its top row), and word plane by word plane: a row of w words is w planes
+of `plane` words (64, 128 or 256, the first that holds 2K+2), plane j holding word j of every entry.  Plain Python
 integers throughout; nothing here comes from the library.
 """
 
@@ -84,11 +85,11 @@ def section(count, N, K, W, blob_bytes_before):
         return None
     need = [max(1, (T[n][2 * K].bit_length() + 31) // 32) for n in range(N)]
     words = [need[n | 3] for n in range(N)]
-    ewords = [4 if w == 3 else w for w in words]
+    plane = 64 if 2 * K + 2 <= 64 else (128 if 2 * K + 2 <= 128 else 256)
     te_offs, teoff = [0] * N, 0
     for n in range(N - 1, -1, -1):              # the widest rows come first
         te_offs[n] = teoff
-        teoff += (2 * K + 2) * ewords[n] * 4
+        teoff += plane * words[n] * 4
     shifts, lens, offs, tables = [], [], [], []
     boff = 0
     for n in range(N):
@@ -131,7 +132,7 @@ def section(count, N, K, W, blob_bytes_before):
             nxt = T[n - 1][2 * (m >> 1)] if n >= 1 else 0
             row.append((nxt - T[n][m]) & ((1 << (32 * words[n])) - 1))
         E.append(row)
-    return dict(off=(blob_bytes_before + 127) & ~127, words=words, ewords=ewords, te_offs=te_offs,
+    return dict(off=(blob_bytes_before + 127) & ~127, words=words, plane=plane, te_offs=te_offs,
                 counts=[words.count(w) for w in (4, 3, 2, 1)], rec_off=rec_off, b_off=b_off, t_off=t_off, e_off=e_off,
                 te_bytes=te_bytes, total=total, shifts=shifts, lens=lens, offs=offs, tables=tables, T=T, E=E)
 

@@ -168,16 +168,16 @@ def test_table_blob_sections(N, K):
         assert list(sec[:8]) == [bs.MAGIC, N, K, srch["total"]] + srch["counts"]
         for n in range(N):
             rec = sec[(srch["rec_off"] + 16 * n) // 4: (srch["rec_off"] + 16 * n) // 4 + 4]
-            sh, ew, at = srch["shifts"][n], srch["ewords"][n], srch["te_offs"][n]
+            sh, nw, at, plane = srch["shifts"][n], srch["words"][n], srch["te_offs"][n], srch["plane"]
             want = [32 - sh, srch["e_off"] + at,
                     (srch["b_off"] + 4 * (srch["offs"][n] - (bs.KEY_OF_ONE >> sh))) & 0xFFFFFFFF, sh]
             assert list(rec) == want, ("record", n)
             b0 = srch["b_off"] // 4 + srch["offs"][n]
             assert list(sec[b0: b0 + srch["lens"][n]]) == srch["tables"][n], ("buckets", n)
             for name, vals in (("t_off", srch["T"]), ("e_off", srch["E"])):
-                row = sec[(srch[name] + at) // 4: (srch[name] + at) // 4 + (2 * K + 2) * ew].reshape(2 * K + 2, ew)
+                row = sec[(srch[name] + at) // 4: (srch[name] + at) // 4 + plane * nw].reshape(nw, plane)   # word planes
                 for m in range(2 * K + 1):
-                    assert list(row[m]) == words(vals[n][m], ew), (name, n, m)
+                    assert list(row[:, m]) == words(vals[n][m], nw), (name, n, m)
 
 
 @pytest.mark.parametrize("N,G,b", [(32, 16, 8), (32, 128, 4), (32, 448, 8), (64, 448, 6), (32, 128, 8),
