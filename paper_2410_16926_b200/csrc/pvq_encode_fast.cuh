@@ -117,7 +117,7 @@ __device__ __forceinline__ void index_step(float avs, float t, float one, uint32
     constexpr int EB = TW * 4;
     // 2^23 + |y_i| moved to where one unit in the last place is 1/EB: the low bits of the
     // float are then |y_i| * EB, the bytes to move along the row
-    constexpr int SH = EB == 16 ? 4 : (EB == 8 ? 3 : 2);
+    constexpr int SH = 2;  // the rows are stored word plane by word plane: an entry's word 0 is 4 bytes from the next entry's
     constexpr uint32_t kBaseBits = static_cast<uint32_t>(127 + 23 - SH) << 23;   // bits of 2^(23-SH)
     const float tq = __fadd_rn(t, one);                                          // 2^23 + |y_i|
     const float shifted = __fsub_rn(tq, kMagic - static_cast<float>(1 << (23 - SH)));  // 2^(23-SH) + |y_i|, exact
@@ -131,10 +131,13 @@ __device__ __forceinline__ void index_step(float avs, float t, float one, uint32
     const float mf = __fsub_rn(tq, kMagic);  // |y_i|
     const float offs = __fmul_rn(flag_gt(__fmul_rn(mf, avs), 0.0f), __int_as_float(N * CROW * EB));
     const uint32_t addr = __float_as_uint(__fadd_rn(__uint_as_float(A), offs));
-    const mp<TW> ent = load_entry<TW, I * CROW * EB>(addr);
+    // word w of the entry sits CROW words behind word w - 1 (threads of a warp read
+    // neighbouring columns: different banks)
     mp<W> add;
-#pragma unroll
-    for (int w = 0; w < W; ++w) add.w[w] = ent.w[w];
+    add.w[0] = load_entry<1, I * CROW * EB>(addr).w[0];
+    if constexpr (W > 1) add.w[1] = load_entry<1, I * CROW * EB + CROW * 4>(addr).w[0];
+    if constexpr (W > 2) add.w[2] = load_entry<1, I * CROW * EB + 2 * CROW * 4>(addr).w[0];
+    if constexpr (W > 3) add.w[3] = load_entry<1, I * CROW * EB + 3 * CROW * 4>(addr).w[0];
     mp_add<W>(c, add);  // modulo 2^(32 W)
     A += __float_as_uint(shifted) - kBaseBits;
 }

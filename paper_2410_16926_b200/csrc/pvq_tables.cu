@@ -252,10 +252,11 @@ __global__ void derive_fast_tables_kernel(int N, int K, int Wc, uint32_t* __rest
     for (int e = tid; e < centries; e += nthr) {
         const int i = e / L.crow;
         const int k = e - i * L.crow;
-        uint32_t* c0 = blob + L.cenc_off[0] / 4 + static_cast<size_t>(e) * TW;
-        uint32_t* c1 = blob + L.cenc_off[1] / 4 + static_cast<size_t>(e) * TW;
+        // a row is TW planes of crow words: word w of entry k at (i * TW + w) * crow + k
+        uint32_t* c0 = blob + L.cenc_off[0] / 4 + static_cast<size_t>(i) * TW * L.crow + k;
+        uint32_t* c1 = blob + L.cenc_off[1] / 4 + static_cast<size_t>(i) * TW * L.crow + k;
         if (k > K) {  // the rest of the row
-            for (int w = 0; w < TW; ++w) c0[w] = c1[w] = 0u;
+            for (int w = 0; w < TW; ++w) c0[w * L.crow] = c1[w * L.crow] = 0u;
             continue;
         }
         const uint32_t* un = U + (static_cast<size_t>(i + 1) * (K + 2) + k + 1) * TW;  // U(n-1, k): next position
@@ -269,8 +270,8 @@ __global__ void derive_fast_tables_kernel(int N, int K, int Wc, uint32_t* __rest
             b0 = d0 >> 32;  // 0 or -1
             b1 = d1 >> 32;
             const bool in = w < Wc;  // modulo 2^(32 Wc): the words above stay zero
-            c0[w] = in ? static_cast<uint32_t>(d0) : 0u;
-            c1[w] = in ? static_cast<uint32_t>(d1) : 0u;
+            c0[w * L.crow] = in ? static_cast<uint32_t>(d0) : 0u;
+            c1[w * L.crow] = in ? static_cast<uint32_t>(d1) : 0u;
         }
     }
 }

@@ -155,13 +155,13 @@ def test_table_blob_sections(N, K):
     if lay["cenc0"] is not None:
         for name, off in (("cenc0", lay["cenc0"]), ("cenc1", lay["cenc1"])):
             crow = lay["crow"]
-            sec = blob[off // 4: off // 4 + N * crow * top].reshape(N, crow, top)
-            assert not sec[:, K + 1:].any()
+            sec = blob[off // 4: off // 4 + N * crow * top].reshape(N, top, crow)      # rows of `top` word planes
+            assert not sec[:, :, K + 1:].any()
             for i in range(N):
                 n = N - 1 - i
                 for k in range(K + 1):
                     sub = U(n, k) if name == "cenc0" else 2 * sum(val[n][:k + 1])
-                    assert list(sec[i, k]) == words((U(n - 1, k) - sub) & mask, top), (name, i, k)
+                    assert list(sec[i, :, k]) == words((U(n - 1, k) - sub) & mask, top), (name, i, k)
     if srch is not None:
         # the decoder's search section: header, row records, bucket tables, thresholds, increments
         sec = blob[srch["off"] // 4: (srch["off"] + srch["total"]) // 4]
