@@ -121,7 +121,7 @@ __device__ __forceinline__ void index_step(float avs, float t, float one, uint32
     constexpr uint32_t kBaseBits = static_cast<uint32_t>(127 + 23 - SH) << 23;   // bits of 2^(23-SH)
     const float tq = __fadd_rn(t, one);                                          // 2^23 + |y_i|
     const float shifted = __fsub_rn(tq, kMagic - static_cast<float>(1 << (23 - SH)));  // 2^(23-SH) + |y_i|, exact
-    // y_i > 0 reads cenc[1], N rows further on.  "|y_i| > 0 and the sign bit of x_i clear" is
+    // y_i > 0 reads cenc[1], N rows and the skew further on.  "|y_i| > 0 and the sign bit of x_i clear" is
     // "|y_i| a_i > 0" with the sign of x_i on a_i: a position with a_i = 0 never gets a pulse
     // (d = sum e_i + (K - sum a_i), the last term far below 1 in magnitude and every e_i below 1,
     // so d does not exceed the number of non-zero residuals), and the point (K, 0, ..., 0) of a
@@ -129,7 +129,7 @@ __device__ __forceinline__ void index_step(float avs, float t, float one, uint32
     // flag (1.0f or 0.0f) times the distance between the tables, and its sum with the address,
     // are exact on integers this small held as subnormal floats.
     const float mf = __fsub_rn(tq, kMagic);  // |y_i|
-    const float offs = __fmul_rn(flag_gt(__fmul_rn(mf, avs), 0.0f), __int_as_float(N * CROW * EB));
+    const float offs = __fmul_rn(flag_gt(__fmul_rn(mf, avs), 0.0f), __int_as_float(N * CROW * EB + static_cast<int>(kCencSkew)));
     const uint32_t addr = __float_as_uint(__fadd_rn(__uint_as_float(A), offs));
     // word w of the entry sits CROW words behind word w - 1 (threads of a warp read
     // neighbouring columns: different banks)
@@ -265,8 +265,8 @@ __global__ void __launch_bounds__(kFastThreadsMax, 2) encode_fast_kernel(const _
     __shared__ uint64_t stage_bar;
     const BulkStage stage = bulk_stage_begin(&stage_bar);
     if (tid == 0) {
-        bulk_stage_expect(stage, 2u * L.cenc_bytes + (FUSED ? walk_tables_stage_bytes(L, sm.walk_phases) : 0u));
-        bulk_stage_copy(stage, smem, reinterpret_cast<const uint8_t*>(a.table) + L.cenc_off[0], 2u * L.cenc_bytes);
+        bulk_stage_expect(stage, 2u * L.cenc_bytes + kCencSkew + (FUSED ? walk_tables_stage_bytes(L, sm.walk_phases) : 0u));
+        bulk_stage_copy(stage, smem, reinterpret_cast<const uint8_t*>(a.table) + L.cenc_off[0], 2u * L.cenc_bytes + kCencSkew);
         if constexpr (FUSED) walk_tables_stage(stage, smem + sm.walk_off, a.table, L, sm.walk_phases);
     }
     WalkTables wt;
@@ -535,7 +535,7 @@ static int launch_encode_fast_c(BatchArgs& a, cudaStream_t stream) {
     FastSmem sm;
     // room behind the tables: a column offset is a sum of N small integers that cannot leave
     // [0, K] for finite input; should it ever, the read still falls inside the block's memory
-    sm.tab_bytes = static_cast<uint32_t>(2 * N * CROW + N + 2) * EB;  // == 2 * cenc_bytes + slack
+    sm.tab_bytes = static_cast<uint32_t>(2 * N * CROW + N + 2) * EB + kCencSkew;  // == 2 * cenc_bytes + the skew + slack
     sm.ss_off = (sm.tab_bytes + 15u) & ~15u;
     sm.ss_floats = ss_floats;
     sm.edges_off = sm.ss_off + 2u * static_cast<uint32_t>(ss_floats) * 4u;

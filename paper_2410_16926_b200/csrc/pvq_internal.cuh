@@ -93,7 +93,9 @@ struct BatchArgs {
 //   cenc[0..1]  the encoder's tables in telescoped form (present for codes of up to 4 words and
 //               up to 127 pulses when both fit 160 KB), rows by position i, `crow` entries of
 //               `top_words` words for k = 0..K (zeros beyond K), crow = 32, 64 or 128, the
-//               first that holds K+1; cenc[1] follows cenc[0] directly.  Modulo 2^(32 W):
+//               first that holds K+1, stored word plane by word plane (a row is `top_words`
+//               planes of crow words, plane j holding word j of every entry); cenc[1] follows
+//               cenc[0] after kCencSkew bytes.  Modulo 2^(32 W):
 //                 cenc[0]  U(n-1,k) - U(n,k)      for y_i <= 0
 //                 cenc[1]  U(n-1,k) - 2 V(n,k)    for y_i > 0
 //               with n = N-1-i and U(-1, .) = 0.  The contribution of position i to the code,
@@ -125,6 +127,9 @@ struct TableLayout {
 };
 
 constexpr uint32_t kCencLimit = 160u * 1024u;  // both telescoped encoder tables have to fit this
+// cenc[1] starts half a row of banks (64 bytes) off a multiple of 128 behind cenc[0]: threads of a
+// warp that read the same column of the two tables then hit different banks
+constexpr uint32_t kCencSkew = 64u;
 
 __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
     TableLayout L;
@@ -170,10 +175,9 @@ __host__ __device__ inline TableLayout table_layout(int N, int K, int W) {
         if (W <= 4 && K + 1 <= 128 && 2u * cb <= kCencLimit) {
             L.crow = crow;
             L.cenc_bytes = cb;
-            for (int p = 0; p < 2; ++p) {
-                L.cenc_off[p] = off;
-                off += cb;  // a multiple of 128
-            }
+            L.cenc_off[0] = off;
+            L.cenc_off[1] = off + cb + kCencSkew;
+            off += 2u * cb + 128u;  // cb is a multiple of 128
         }
     }
     L.total = off;

@@ -39,8 +39,8 @@ def blob_layout(N, K, W):
         crow = 32 if K + 1 <= 32 else (64 if K + 1 <= 64 else 128)
         cb = N * crow * top * 4
         if W <= 4 and K + 1 <= 128 and 2 * cb <= 160 * 1024:
-            lay["cenc0"], lay["cenc1"], lay["crow"] = off, off + cb, crow
-            off += 2 * cb
+            lay["cenc0"], lay["cenc1"], lay["crow"] = off, off + cb + 64, crow      # 64 bytes between the two
+            off += 2 * cb + 128
     lay["total"] = off
     return lay
 
