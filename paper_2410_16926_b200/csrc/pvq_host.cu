@@ -155,6 +155,26 @@ int code_words_for(int N, int K) {
     return W;
 }
 
+bool count_fills_its_words(int N, int K) {  // memoised like code_words_for: the count takes a while for large (N,K)
+    static std::mutex mu;
+    static std::map<std::pair<int, int>, bool> memo;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = memo.find({N, K});
+    if (it != memo.end()) return it->second;
+    bool fills = false;
+    if (N >= 1 && N <= 4096 && K >= 0 && K <= 65535) {
+        CountColumn c(N);
+        bool ok = true;
+        for (int k = 0; k < K && ok; ++k) ok = c.advance();
+        if (ok) {
+            const BigU& v = c.col[static_cast<size_t>(N)];
+            fills = v.is_pow2() && v.bit_length() > 32 && (v.bit_length() - 1) % 32 == 0;
+        }
+    }
+    memo[{N, K}] = fills;
+    return fills;
+}
+
 // The leading 24 bits of v >= 1 as the bits of an fp32 (what search_key computes on the device).
 static uint32_t key_bits(const BigU& v) {
     const int e = v.bit_length() - 1;

@@ -253,6 +253,7 @@ struct SearchLayout {
 // host helpers (pvq_host.cu)
 int set_cuda_error(cudaError_t e);  // records e, returns PVQ_ERR_CUDA
 int code_words_for(int N, int K);   // W, or 0 when it cannot be computed
+bool count_fills_its_words(int N, int K);  // N(N,K) == 2^(32 W) exactly: the one count that needs W + 1 words
 // the search section for (N,K), memoised; present == false where the decoder walks instead
 const SearchLayout& search_layout_for(int N, int K);
 bool is_aligned(const void* p, size_t a);

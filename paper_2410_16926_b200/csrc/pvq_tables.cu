@@ -72,67 +72,102 @@ __global__ void __launch_bounds__(1024) count_table_kernel(int N, int K, int Wc,
     }
 }
 
-// The same table for more pulses than a block has threads (K up to kMaxPulses).  One block;
-// thread t owns the `chunk` consecutive columns from t * chunk.  Row n is the inclusive prefix
-// sum over k of a_k = N(n-1,k) + N(n-1,k-1), read back from the row the block has just
-// written: each thread sums its chunk, the block scans the threads' totals in shared memory,
-// and a second pass over the chunk writes the row.  Still no inter-block barrier.
+// The same table for more pulses than a block has threads (K up to kMaxPulses), built by many
+// blocks (App. C.2 / Algorithm 4 spreads a row over blocks and puts a barrier between rows).
+// Row n is the inclusive prefix sum over k of a_k = N(n-1,k) + N(n-1,k-1), read back from the
+// row before it.  Thread t of the launch owns the `chunk` consecutive columns from t * chunk.
+// Two launches per row, the launch boundary being the barrier between blocks (every wait is
+// the stream's: nothing spins):
+//   count_row_sums_kernel   every block sums the a_k of its columns and writes the total;
+//   count_row_write_kernel  every block scans the totals of the blocks before it, scans its
+//                           threads' sums once more, and writes its columns of the row.
+// The block totals go to a scratch area inside the blob that a later set-up kernel overwrites.
+
+// Inclusive scan over the block's threads of one W-word value each, through `buf`
+// (blockDim.x entries of W words); on return buf[t] holds thread t's result as well.
 template <int W>
-__global__ void __launch_bounds__(1024) count_table_chunked_kernel(int N, int K, int Wc, int chunk,
-                                                                   uint32_t* __restrict__ table) {
-    extern __shared__ uint32_t tot[];  // blockDim.x entries of W words
+__device__ __forceinline__ void block_scan_inclusive(mp<W>& v, uint32_t* buf) {
     const int t = threadIdx.x;
-    const int KP = K + 1;
-    const int k0 = t * chunk;
-    const int k1 = k0 + chunk < KP ? k0 + chunk : KP;
-    auto load = [Wc](const uint32_t* row, int k) {
-        mp<W> v;
 #pragma unroll
-        for (int w = 0; w < W; ++w) v.w[w] = w < Wc ? row[static_cast<size_t>(k) * Wc + w] : 0u;
-        return v;
-    };
-    for (int k = k0; k < k1; ++k)  // row 0: N(0,0) = 1, N(0,k>=1) = 0
-        for (int w = 0; w < Wc; ++w) table[static_cast<size_t>(k) * Wc + w] = (k == 0 && w == 0) ? 1u : 0u;
+    for (int w = 0; w < W; ++w) buf[t * W + w] = v.w[w];
     __syncthreads();
-    for (int n = 1; n < N; ++n) {
-        const uint32_t* prev = table + static_cast<size_t>(n - 1) * KP * Wc;
-        uint32_t* cur = table + static_cast<size_t>(n) * KP * Wc;
-        mp<W> run;
-        mp_zero(run);
-        for (int k = k0; k < k1; ++k) {
-            mp_add<W>(run, load(prev, k));
-            if (k > 0) mp_add<W>(run, load(prev, k - 1));
-        }
-        // inclusive scan of the threads' totals
-        mp<W> v = run;
-#pragma unroll
-        for (int w = 0; w < W; ++w) tot[t * W + w] = v.w[w];
+    for (int off = 1; off < static_cast<int>(blockDim.x); off <<= 1) {
+        mp<W> o;
+        mp_zero(o);
+        if (t >= off) o = mp_load<W>(buf + (t - off) * W);
         __syncthreads();
-        for (int off = 1; off < static_cast<int>(blockDim.x); off <<= 1) {
-            mp<W> o;
-            mp_zero(o);
-            if (t >= off) o = mp_load<W>(tot + (t - off) * W);
-            __syncthreads();
-            mp_add<W>(v, o);
+        mp_add<W>(v, o);
 #pragma unroll
-            for (int w = 0; w < W; ++w) tot[t * W + w] = v.w[w];
-            __syncthreads();
+        for (int w = 0; w < W; ++w) buf[t * W + w] = v.w[w];
+        __syncthreads();
+    }
+}
+
+// sum of a_k over the columns [k0, k1) of a thread
+template <int W>
+__device__ __forceinline__ mp<W> chunk_sum(const uint32_t* __restrict__ prev, int Wc, int k0, int k1) {
+    mp<W> run;
+    mp_zero(run);
+    for (int k = k0; k < k1; ++k) {
+        for (int j = (k > 0 ? k - 1 : k); j <= k; ++j) {
+            mp<W> v;
+#pragma unroll
+            for (int w = 0; w < W; ++w) v.w[w] = w < Wc ? prev[static_cast<size_t>(j) * Wc + w] : 0u;
+            mp_add<W>(run, v);
         }
-        mp_zero(run);
-        if (t > 0) run = mp_load<W>(tot + (t - 1) * W);  // everything left of this chunk
-        for (int k = k0; k < k1; ++k) {
-            mp_add<W>(run, load(prev, k));
-            if (k > 0) mp_add<W>(run, load(prev, k - 1));
-            for (int w = 0; w < Wc; ++w) cur[static_cast<size_t>(k) * Wc + w] = run.w[w];
-        }
-        __syncthreads();  // the row is complete (and the totals free) before the next one starts
+    }
+    return run;
+}
+
+__global__ void count_row0_kernel(int K, int Wc, uint32_t* __restrict__ table) {
+    const size_t words = static_cast<size_t>(K + 1) * Wc;  // row 0: N(0,0) = 1, N(0,k>=1) = 0
+    for (size_t i = blockIdx.x * blockDim.x + threadIdx.x; i < words; i += static_cast<size_t>(gridDim.x) * blockDim.x)
+        table[i] = i == 0 ? 1u : 0u;
+}
+
+template <int W>
+__global__ void __launch_bounds__(256) count_row_sums_kernel(const uint32_t* __restrict__ prev, int KP, int Wc, int chunk,
+                                                             uint32_t* __restrict__ block_totals) {
+    extern __shared__ uint32_t buf[];  // blockDim.x entries of W words
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int k0 = min(t * chunk, KP), k1 = min(k0 + chunk, KP);
+    mp<W> v = chunk_sum<W>(prev, Wc, k0, k1);
+    block_scan_inclusive<W>(v, buf);
+    if (threadIdx.x == blockDim.x - 1) {
+#pragma unroll
+        for (int w = 0; w < W; ++w) block_totals[blockIdx.x * W + w] = v.w[w];
+    }
+}
+
+template <int W>
+__global__ void __launch_bounds__(256) count_row_write_kernel(const uint32_t* __restrict__ prev, uint32_t* __restrict__ cur,
+                                                              int KP, int Wc, int chunk,
+                                                              const uint32_t* __restrict__ block_totals) {
+    extern __shared__ uint32_t buf[];
+    // everything in the blocks before this one (gridDim.x <= blockDim.x: one total per thread)
+    mp<W> base;
+    mp_zero(base);
+    if (threadIdx.x < gridDim.x) base = mp_load<W>(block_totals + threadIdx.x * W);
+    block_scan_inclusive<W>(base, buf);
+    mp_zero(base);
+    if (blockIdx.x > 0) base = mp_load<W>(buf + (blockIdx.x - 1) * W);
+    __syncthreads();  // buf is reused below
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    const int k0 = min(t * chunk, KP), k1 = min(k0 + chunk, KP);
+    mp<W> v = chunk_sum<W>(prev, Wc, k0, k1);
+    block_scan_inclusive<W>(v, buf);
+    if (threadIdx.x > 0) mp_add<W>(base, mp_load<W>(buf + (threadIdx.x - 1) * W));  // the threads before this one
+    for (int k = k0; k < k1; ++k) {
+        mp_add<W>(base, chunk_sum<W>(prev, Wc, k, k + 1));
+        for (int w = 0; w < Wc; ++w) cur[static_cast<size_t>(k) * Wc + w] = base.w[w];
     }
 }
 
 // The other sections of the blob (TableLayout): the same numbers re-laid for the decode walk,
 // narrow copies saturated at their width, and N(N,K) itself.
+// with_enc == 0: the encoder's cumulative tables are written by derive_enc_tables_kernel instead.
 template <int W>
-__global__ void derive_tables_kernel(int N, int K, int Wc, uint32_t* __restrict__ blob) {
+__global__ void derive_tables_kernel(int N, int K, int Wc, uint32_t* __restrict__ blob, int with_enc) {
     const TableLayout L = table_layout(N, K, Wc);
     if (L.rowlen == 0) return;
     const int KP = K + 1;
@@ -166,7 +201,7 @@ __global__ void derive_tables_kernel(int N, int K, int Wc, uint32_t* __restrict_
         }
     }
     // encoder tables: one thread per position runs the prefix sum V(n,k) = V(n,k-1) + N(n,k)
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < N; i += gridDim.x * blockDim.x) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; with_enc && i < N; i += gridDim.x * blockDim.x) {
         const uint32_t* row = blob + static_cast<size_t>(N - 1 - i) * KP * Wc;
         const int TW = L.top_words;
         uint32_t* eu = blob + L.enc_off[0] / 4 + static_cast<size_t>(i) * (K + 2) * TW;
@@ -370,7 +405,7 @@ static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStrea
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error(e);
     if (table_layout(N, K, Wc).rowlen != 0) {
-        derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table);
+        derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table, 1);
         if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
         derive_fast_tables_kernel<<<16, 256, 0, s>>>(N, K, Wc, d_table);
         if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
@@ -379,22 +414,97 @@ static int launch_count_table(int N, int K, int Wc, uint32_t* d_table, cudaStrea
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 
+// The encoder's cumulative tables entry by entry, for tables too large for the one-thread-per-row
+// prefix sums of derive_tables_kernel.  With V(n,k) = sum_{j<=k} N(n,j):
+//   U(n,k) = V(n,k) + V(n,k-1) = N(n+1,k)     (the recurrence of Sec. 2.4 summed over k)
+//   N(n,k) = V(n,k) - V(n,k-1),  so  2 V(n,k) = N(n+1,k) + N(n,k)
+// Row n + 1 is the next row of the count table, for n = N-1 the row `row_n` that the builder
+// ran one row further (N(N,k), modulo 2^(32 Wc): top_overflow says that N(N,K) is exactly
+// 2^(32 Wc), the one value that does not fit).
+template <int W>
+__global__ void derive_enc_tables_kernel(int N, int K, int Wc, uint32_t* __restrict__ blob,
+                                         const uint32_t* __restrict__ row_n, int top_overflow) {
+    const TableLayout L = table_layout(N, K, Wc);
+    const int TW = L.top_words;
+    const int KP = K + 1;
+    const long long entries = static_cast<long long>(N) * (K + 2);
+    for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < entries;
+         e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int i = static_cast<int>(e / (K + 2));
+        const int c = static_cast<int>(e - static_cast<long long>(i) * (K + 2)) - 1;  // -1..K
+        const int n = N - 1 - i;
+        uint32_t* eu = blob + L.enc_off[0] / 4 + static_cast<size_t>(e) * TW;
+        uint32_t* e2 = blob + L.enc_off[1] / 4 + static_cast<size_t>(e) * TW;
+        uint32_t* ev = blob + L.enc_off[2] / 4 + static_cast<size_t>(e) * TW;
+        const uint32_t* up = c < 0 ? nullptr : (n + 1 < N ? blob + (static_cast<size_t>(n + 1) * KP + c) * Wc
+                                                         : row_n + static_cast<size_t>(c) * Wc);
+        const uint32_t* np = c < 0 ? nullptr : blob + (static_cast<size_t>(n) * KP + c) * Wc;
+        unsigned long long carry = 0;
+        uint32_t sum[W + 1];  // U + N = 2 V, one word more than an entry
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+            const unsigned long long a = (up && w < Wc) ? up[w] : 0u, b = (np && w < Wc) ? np[w] : 0u;
+            const unsigned long long t = a + b + carry;
+            sum[w] = static_cast<uint32_t>(t);
+            carry = t >> 32;
+        }
+        sum[W] = static_cast<uint32_t>(carry);
+        // the word above the entry: a carry out of Wc words sits in sum[Wc]; the lost top bit of U adds one
+        uint32_t above = Wc < W ? sum[Wc] : sum[W];
+        if (top_overflow && i == 0 && c == K) above += 1u;
+        for (int w = 0; w < TW; ++w) {
+            const bool in = w < Wc;
+            const uint32_t hi = w + 1 < Wc ? sum[w + 1 < W ? w + 1 : W] : above;  // the word above word w of 2 V
+            eu[w] = (in && up) ? up[w] : 0u;
+            e2[w] = in ? sum[w < W ? w : W] : 0u;
+            ev[w] = in ? (sum[w < W ? w : W] >> 1) | (hi << 31) : 0u;
+        }
+    }
+}
+
 template <int W>
 static int launch_count_table_chunked(int N, int K, int Wc, uint32_t* d_table, cudaStream_t s) {
-    const int threads = 1024;
-    const int chunk = (K + 1 + threads - 1) / threads;
+    const TableLayout L = table_layout(N, K, Wc);
+    DeviceInfo di;
+    int st = device_info(&di);
+    if (st != PVQ_OK) return st;
+    const int threads = 256;
+    const int KP = K + 1;
+    const int chunk = (KP + di.sms * threads - 1) / (di.sms * threads);  // at most one block per SM
+    const int blocks = (KP + chunk * threads - 1) / (chunk * threads);   // <= threads, as the write kernel needs
     const size_t smem = static_cast<size_t>(threads) * W * sizeof(uint32_t);
-    cudaError_t e = cudaFuncSetAttribute(count_table_chunked_kernel<W>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         static_cast<int>(smem));
+    constexpr size_t kScratchRowOffset = 32768;  // behind the totals (at most 256 blocks of 32 words)
+    // the block totals: at the start of the decoder's first table, which derive_tables_kernel fills below
+    if (L.rowlen == 0 || static_cast<size_t>(blocks) * W * 4u > L.walk_bytes[0] || blocks > threads)
+        return PVQ_ERR_UNSUPPORTED;
+    uint32_t* totals = d_table + L.walk_off[0] / 4;
+    count_row0_kernel<<<16, 256, 0, s>>>(K, Wc, d_table);
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return set_cuda_error(e);
-    count_table_chunked_kernel<W><<<1, threads, smem, s>>>(N, K, Wc, chunk, d_table);
-    if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
-    if (table_layout(N, K, Wc).rowlen != 0) {
-        derive_tables_kernel<W><<<16, 256, 0, s>>>(N, K, Wc, d_table);
+    for (int n = 1; n < N; ++n) {
+        const uint32_t* prev = d_table + static_cast<size_t>(n - 1) * KP * Wc;
+        uint32_t* cur = d_table + static_cast<size_t>(n) * KP * Wc;
+        count_row_sums_kernel<W><<<blocks, threads, smem, s>>>(prev, KP, Wc, chunk, totals);
+        count_row_write_kernel<W><<<blocks, threads, smem, s>>>(prev, cur, KP, Wc, chunk, totals);
         if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
-        derive_fast_tables_kernel<<<16, 256, 0, s>>>(N, K, Wc, d_table);
-        e = cudaGetLastError();
     }
+    // One row more, N(N,k), behind the totals in the same scratch area: with it the encoder's
+    // cumulative tables follow entry by entry.  (Where the area is too small the set-up kernel
+    // below runs its own prefix sums.)
+    const size_t row_bytes = static_cast<size_t>(KP) * Wc * 4u;
+    const bool enc_by_entry = kScratchRowOffset + row_bytes <= L.walk_bytes[0];
+    if (enc_by_entry) {
+        const uint32_t* prev = d_table + static_cast<size_t>(N - 1) * KP * Wc;
+        uint32_t* row_n = totals + kScratchRowOffset / 4;
+        count_row_sums_kernel<W><<<blocks, threads, smem, s>>>(prev, KP, Wc, chunk, totals);
+        count_row_write_kernel<W><<<blocks, threads, smem, s>>>(prev, row_n, KP, Wc, chunk, totals);
+        derive_enc_tables_kernel<W><<<4 * di.sms, 256, 0, s>>>(N, K, Wc, d_table, row_n, count_fills_its_words(N, K) ? 1 : 0);
+        if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
+    }
+    derive_tables_kernel<W><<<4 * di.sms, 256, 0, s>>>(N, K, Wc, d_table, enc_by_entry ? 0 : 1);
+    if ((e = cudaGetLastError()) != cudaSuccess) return set_cuda_error(e);
+    derive_fast_tables_kernel<<<16, 256, 0, s>>>(N, K, Wc, d_table);
+    e = cudaGetLastError();
     return e == cudaSuccess ? PVQ_OK : set_cuda_error(e);
 }
 
@@ -457,7 +567,8 @@ extern "C" int pvq_build_count_table(int N, int K, uint32_t* d_table, size_t byt
     if (!is_aligned(d_table, 16)) return PVQ_ERR_ALIGNMENT;
     if (bytes < pvq_count_table_bytes(N, K)) return PVQ_ERR_TABLE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (K > 1023) {  // more pulses than threads of a block: the chunked builder, in 8, 16 or 32 words
+    // more pulses than threads of a block, or rows of 32 KB and more: the multi-block builder, in 8, 16 or 32 words
+    if (K > 1023 || static_cast<long long>(K + 1) * W >= 8192) {
         if (W <= 8) return launch_count_table_chunked<8>(N, K, W, d_table, s);
         if (W <= 16) return launch_count_table_chunked<16>(N, K, W, d_table, s);
         return launch_count_table_chunked<32>(N, K, W, d_table, s);

@@ -103,7 +103,7 @@ def test_count_table_word_for_word(N, K):
 
 
 @pytest.mark.parametrize("N,K", [(8, 16), (16, 18), (32, 22), (32, 50), (32, 105), (64, 96), (64, 26), (128, 40),
-                                 (64, 230), (128, 300), (256, 200)])
+                                 (64, 230), (128, 300), (256, 200), (16, 1136), (32, 1100)])
 def test_table_blob_sections(N, K):
     """Every rearranged section of the table blob holds the numbers of the count table."""
     W = pvq.code_words(N, K)
