@@ -93,7 +93,8 @@ def check_decode(cd, enc_dev, enc_np):
 
 @pytest.mark.parametrize("N,K", [(8, 6), (8, 40), (16, 18), (32, 22), (32, 50), (64, 96), (32, 1), (128, 187),
                                  (64, 405), (128, 386), (128, 782), (256, 369), (256, 760),
-                                 (16, 1136), (32, 1858), (64, 3359), (128, 1576), (128, 6378), (32, 1024)])
+                                 (16, 1136), (32, 1858), (64, 3359), (128, 1576), (128, 6378), (32, 1024),
+                                 (1, 1100), (2, 1500), (3, 2047), (8, 8191)])
 def test_count_table_word_for_word(N, K):
     W = pvq.code_words(N, K)
     t = pvq.build_count_table(N, K)
