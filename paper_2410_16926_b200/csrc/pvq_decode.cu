@@ -15,7 +15,7 @@ namespace pvq {
 
 namespace {
 
-constexpr int kDecThreads = 512;
+constexpr int kDecThreads = 768;
 
 template <int N, int W, typename YT>
 __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_constant__ BatchArgs a) {
