@@ -179,7 +179,10 @@ int pvq_encode(const void* d_x, int dtype, int64_t rows, int64_t cols, int64_t l
  *   d_out      rows x cols bf16, leading dimension ld_out (elements, multiple of 8),
  *              16-byte aligned.
  *   d_status   optional device word; PVQ_STATUS_INVALID_CODE is OR-ed into it when a code
- *              is >= N(N,K) (that group decodes to zeros).  May be NULL. */
+ *              is >= N(N,K) (that group decodes to zeros), PVQ_STATUS_TABLE_MISMATCH when
+ *              d_table was built for other (N,K) (nothing is written then),
+ *              PVQ_STATUS_STAGING_TIMEOUT when a block gave up waiting for its tables.
+ *              May be NULL. */
 int pvq_decode(const uint32_t* d_codes, const uint8_t* d_scale_idx, const float* d_row_norm,
                int64_t rows, int64_t cols, int N, int K, int scale_bits, const uint32_t* d_table,
                const float* d_levels, void* d_out, int64_t ld_out, uint32_t* d_status,
