@@ -94,8 +94,9 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
         while (mi + 1 < a.count && tile0 >= a.m[mi + 1].tile_begin) ++mi;
         int mj[GP];
         unsigned row[GP], g[GP];
-        float amp[GP];
-        bool active[GP];
+        float rnorm[GP];
+        unsigned sbits[GP];
+        bool active[GP], active_valid[GP];
         mp<W> q[GP];
         int mcur = mi;
 #pragma unroll
@@ -109,6 +110,7 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
             const unsigned g0 = (tile - m.tile_begin) * 32u;             // first group of the tile
             const unsigned gi = g0 + lane;
             active[j] = tile < a.total_tiles && gi < ngroups;
+            active_valid[j] = active[j];
             // row and group-in-row: one division per tile, the threads follow from the first group
             row[j] = g0 / G;
             g[j] = g0 - row[j] * G + lane;
@@ -123,24 +125,22 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
             }
             mp<W> c;
             mp_zero(c);
-            amp[j] = 0.0f;
+            sbits[j] = 0u;
+            rnorm[j] = 0.0f;
             if (active[j]) {
                 c = mp_load<W>(m.codes + static_cast<size_t>(gi) * W);
+                // the bytes that hold the amplitude index, bits [g*b, g*b + b) of the row's LSB-first
+                // stream, and the row norm: asked for now, used after the search
+                const uint8_t* srow = m.scale_idx + static_cast<size_t>(row[j]) * m.sstride;
+                const unsigned bit = g[j] * b;
+                sbits[j] = srow[bit >> 3];
+                if ((bit & 7u) + b > 8u) sbits[j] |= static_cast<unsigned>(srow[(bit >> 3) + 1]) << 8;
+                if (b != 16u) rnorm[j] = m.row_norm[row[j]];
                 mp<W> tmp;
-                const bool valid = mp_sub_borrow<W>(tmp, c, bound);
-                if (!valid) {  // decodes to zeros: search code 0, whose point has no negative entry
+                if (!mp_sub_borrow<W>(tmp, c, bound)) {  // invalid: decodes to zeros (search code 0, whose point has no negative entry)
                     bad = true;
+                    active_valid[j] = false;
                     mp_zero(c);
-                } else {
-                    // amplitude index: bits [g*b, g*b + b) of the row's LSB-first stream
-                    const uint8_t* srow = m.scale_idx + static_cast<size_t>(row[j]) * m.sstride;
-                    const unsigned bit = g[j] * b;
-                    unsigned bits = srow[bit >> 3];
-                    if ((bit & 7u) + b > 8u) bits |= static_cast<unsigned>(srow[(bit >> 3) + 1]) << 8;
-                    const unsigned qi = (bits >> (bit & 7u)) & ((1u << b) - 1u);
-                    // 16 bits: the amplitude itself as binary16; else the quantile level times the row norm
-                    amp[j] = b == 16u ? __half2float(__ushort_as_half(static_cast<unsigned short>(qi)))
-                                      : __fmul_rn(m.row_norm[row[j]], m.levels[qi]);
                 }
             }
             mp_sub_borrow<W>(q[j], bound, c);  // 1 <= q <= N(N,K)
@@ -148,9 +148,17 @@ __global__ void __launch_bounds__(kSearchThreads / (GP > 2 ? 2 : 1), 1)
         search_codes<N, W, GP, PLANE>(q, K, recs, t_rows, cnt, shared_addr(yslots), ychain);
 #pragma unroll
         for (int j = 0; j < GP; ++j)
-            if (active[j])
-                emit_group<N, int8_t>(a.m[mj[j]], reinterpret_cast<const int8_t*>(yslots + j * ychain), amp[j], row[j],
-                                      g[j]);
+            if (active[j]) {
+                const MatrixArgs& m = a.m[mj[j]];
+                float amp = 0.0f;  // an invalid code decodes to zeros
+                if (active_valid[j]) {
+                    const unsigned qi = (sbits[j] >> ((g[j] * b) & 7u)) & ((1u << b) - 1u);
+                    // 16 bits: the amplitude itself as binary16; else the quantile level times the row norm
+                    amp = b == 16u ? __half2float(__ushort_as_half(static_cast<unsigned short>(qi)))
+                                   : __fmul_rn(rnorm[j], m.levels[qi]);
+                }
+                emit_group<N, int8_t>(m, reinterpret_cast<const int8_t*>(yslots + j * ychain), amp, row[j], g[j]);
+            }
     }
     if (bad && a.status) atomicOr(a.status, PVQ_STATUS_INVALID_CODE);
 }
