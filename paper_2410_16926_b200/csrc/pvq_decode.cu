@@ -81,28 +81,36 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_kernel(const __grid_con
 
         mp<W> c;
         mp_zero(c);
-        float amp = 0.0f;
+        unsigned sbits = 0u;
+        float rnorm = 0.0f;
+        bool valid = false;
         if (active) {
             c = mp_load<W>(m.codes + static_cast<size_t>(gi) * W);
+            // the bytes that hold the amplitude index, bits [g*b, g*b + b) of the row's LSB-first
+            // stream, and the row norm: asked for now, used after the walk
+            const uint8_t* srow = m.scale_idx + static_cast<size_t>(row) * m.sstride;
+            const unsigned bit = g * b;
+            sbits = srow[bit >> 3];
+            if ((bit & 7u) + b > 8u) sbits |= static_cast<unsigned>(srow[(bit >> 3) + 1]) << 8;
+            if (b != 16u) rnorm = m.row_norm[row];
             mp<W> tmp;
-            const bool valid = bound_wide || mp_sub_borrow<W>(tmp, c, bound);
+            valid = bound_wide || mp_sub_borrow<W>(tmp, c, bound);
             if (!valid) {  // decodes to zeros: walk code 0, whose point has no negative entry
                 bad = true;
                 mp_zero(c);
-            } else {
-                // amplitude index: bits [g*b, g*b + b) of the row's LSB-first stream
-                const uint8_t* srow = m.scale_idx + static_cast<size_t>(row) * m.sstride;
-                const unsigned bit = g * b;
-                unsigned bits = srow[bit >> 3];
-                if ((bit & 7u) + b > 8u) bits |= static_cast<unsigned>(srow[(bit >> 3) + 1]) << 8;
-                const unsigned q = (bits >> (bit & 7u)) & ((1u << b) - 1u);
-                // 16 bits: the amplitude itself as binary16; else the quantile level times the row norm
-                amp = b == 16u ? __half2float(__ushort_as_half(static_cast<unsigned short>(q)))
-                               : __fmul_rn(m.row_norm[row], m.levels[q]);
             }
         }
         walk_code<N, W, YT>(c, wt, K, yslots);
-        if (active) emit_group<N, YT>(m, yslots, amp, row, g);
+        if (active) {
+            float amp = 0.0f;
+            if (valid) {
+                const unsigned q = (sbits >> ((g * b) & 7u)) & ((1u << b) - 1u);
+                // 16 bits: the amplitude itself as binary16; else the quantile level times the row norm
+                amp = b == 16u ? __half2float(__ushort_as_half(static_cast<unsigned short>(q)))
+                               : __fmul_rn(rnorm, m.levels[q]);
+            }
+            emit_group<N, YT>(m, yslots, amp, row, g);
+        }
     }
     if (bad && a.status) atomicOr(a.status, PVQ_STATUS_INVALID_CODE);
 }
