@@ -449,6 +449,39 @@ def test_decode_of_codes_on_the_search_thresholds(N, K):
     check_decode(cd, enc_dev, enc_np)
 
 
+@pytest.mark.parametrize("N,K", [(8, 1), (8, 2), (8, 3), (8, 17), (8, 64), (8, 100), (8, 127), (16, 1), (16, 5), (16, 33),
+                                 (16, 64), (16, 90), (16, 127), (32, 1), (32, 2), (32, 7), (32, 31), (32, 32), (32, 63),
+                                 (32, 64), (32, 77), (32, 104), (64, 1), (64, 2), (64, 9), (64, 20), (64, 31)])
+def test_decode_across_pulse_counts(N, K):
+    """Random codes, the first and the last code, and codes at the edges of the first coordinate's
+    blocks, over pulse counts from one to the most that a byte per coordinate and four words per
+    code allow: every table shape of the searching decoder (plane sizes, row widths, shifts)."""
+    from oracle import pvq_pyref as pr
+    rows, G, b = 3, 64, 8
+    cd = Codec(N, 0, G, b, K=K)
+    W = cd.W
+    if W > 4:
+        pytest.skip("more than four words: decoded by the walk, covered elsewhere")
+    count = pr.count_table(N, K)
+    total = count[N][K]
+    rng = np.random.default_rng(5000 * N + K)
+    codes = _random_codes(rng, total, (rows, G), W)
+    flat = codes.reshape(-1, W)
+    # block ends of position 0: N(N-1,K), then + 2 N(N-1,K-j) ... (Algorithm 3's subtractions), and their neighbours
+    edge, special = count[N - 1][K], [0, total - 1]
+    for j in range(1, K + 1):
+        special += [edge - 1, edge, min(edge + 1, total - 1)]
+        edge += 2 * count[N - 1][K - j]
+    for i, c in enumerate(special[:flat.shape[0]]):
+        flat[i] = po.int_to_code(max(0, min(c, total - 1)), W)
+    sidx = rng.integers(0, 256, size=(rows, int(pvq.scale_row_stride(G, b))), dtype=np.uint8)
+    rnorm = (rng.random(rows).astype(np.float32) + 0.5)
+    enc_np = (codes, sidx, rnorm)
+    enc_dev = (torch.from_numpy(codes.view(np.int32)).to(DEV), torch.from_numpy(sidx).to(DEV),
+               torch.from_numpy(rnorm).to(DEV))
+    check_decode(cd, enc_dev, enc_np)
+
+
 def test_decode_refuses_a_table_built_for_other_parameters():
     """The searching decoder's look-ups follow what the table says, so it checks the header of
     its section first: with the table of another K nothing is decoded and the status says so."""
